@@ -1,0 +1,368 @@
+"""CPU oracle for the late-scale step of VAR next-scale prediction under FasterVAR.
+
+TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, obviously-correct numpy
+restatement of what the GPU library computes.  It is imported by the tests, by
+the smoke check and by the benchmark's CPU-baseline leg, and by nothing else;
+it shares no code with the CUDA path and never calls it.
+
+Arithmetic is fp64 (numpy) on bf16-representable inputs, except the row score
+that decides the index set, which is taken in fp32 -- the precision the GPU
+kernel decides it in -- so that both sides take the integer decision alike.
+
+What the paper fixes and this file follows:
+  * row score  p_i = ||F^(i)||^2 / ||F||_F^2            (Sec. 3.3, RTR paragraph)
+  * index set I: the r most important rows, |I| = r       (Sec. 3.3; Algorithm 1)
+  * random projection  F_r = Q^T F,  Q in R^{M x r}, Q_ij ~ N(0, 1/r)
+                                                          (Sec. 3.3 RP; Algorithm 1)
+  * cached output upsampled, F^{o,cache}_{k-1} = Up(F^o_{k-1})   (Eq. "upcache")
+  * restoration F^o_k := {F^o_r rows at I} U {cache rows elsewhere} (Eq. "redefine")
+  * CFG = 0 in the fidelity-refinement stage = null-prompt branch only
+                                                          (Sec. 3.2; Algorithm 1)
+  * rank schedule: ratio of min(M, d) per block chunk and late scale
+                                                          (Eq. "low_rank_percent"; App. A.1 table)
+The paper gives no internals for "the VAR block"; the block below (AdaLN
+shift/scale/gate, multi-head attention over a multi-scale KV cache, tanh-GELU
+FFN, optional cross-attention) is the synthetic definition both sides use.
+
+Parity pins live in tests/test_oracle_*.py.  The composite RP -> blocks -> RTR
+numerics have no worked example in the paper: parity unpinned for the composite
+beyond the invariants tested there (r = M equals the dense block, restoration
+row identities, linearity and norm preservation of the projection).
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+# --------------------------------------------------------------------------- elementary pieces
+
+
+def gelu_tanh(x: np.ndarray) -> np.ndarray:
+    """tanh-approximated GELU: x/2 * (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))."""
+    return 0.5 * x * (1.0 + np.tanh(math.sqrt(2.0 / math.pi) * (x + 0.044715 * x ** 3)))
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def layer_norm(x: np.ndarray, eps: float) -> np.ndarray:
+    """LayerNorm over the last axis, no affine, biased variance."""
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps)
+
+
+def ada_vectors(cond: np.ndarray, w_ada: np.ndarray, b_ada: np.ndarray) -> np.ndarray:
+    """AdaLN vectors of one block for one batch element: W_ada SiLU(c) + b_ada, as
+    6 rows [shift1, scale1, gate1, shift2, scale2, gate2] of width C."""
+    C = cond.shape[-1]
+    return (w_ada @ silu(cond) + b_ada).reshape(6, C)
+
+
+def modulate(x: np.ndarray, shift: np.ndarray, scale: np.ndarray, eps: float) -> np.ndarray:
+    return layer_norm(x, eps) * (1.0 + scale) + shift
+
+
+def softmax_rows(s: np.ndarray) -> np.ndarray:
+    s = s - s.max(axis=-1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, n_heads: int) -> np.ndarray:
+    """Multi-head attention of queries q [n][C] over keys K [L][C] and values V [L][C];
+    heads are contiguous slices of width C / n_heads; no mask; scores scaled by 1/sqrt(D)."""
+    n, C = q.shape
+    D = C // n_heads
+    out = np.empty_like(q)
+    for h in range(n_heads):
+        sl = slice(h * D, (h + 1) * D)
+        p = softmax_rows(q[:, sl] @ K[:, sl].T / math.sqrt(D))
+        out[:, sl] = p @ V[:, sl]
+    return out
+
+
+# --------------------------------------------------------------------------- the method's own steps
+
+
+def row_scores(X: np.ndarray, dtype=np.float32) -> np.ndarray:
+    """s_i = sum_c X[i,c]^2 (numerator of the row probability; Sec. 3.3 RTR)."""
+    Xd = np.asarray(X, dtype=dtype)
+    return np.sum(Xd * Xd, axis=-1, dtype=dtype)
+
+
+def row_probabilities(X: np.ndarray) -> np.ndarray:
+    """p_i = ||X^(i)||^2 / ||X||_F^2 (Sec. 3.3 RTR)."""
+    s = row_scores(X, np.float64)
+    return s / s.sum()
+
+
+def select_top_r(scores: np.ndarray, r: int) -> np.ndarray:
+    """Indices of the r highest-scoring rows, returned ascending.
+    Order: score descending, then index ascending; NaN ranks as +inf; -0 equals +0."""
+    s = np.asarray(scores, dtype=np.float32).copy()
+    s[np.isnan(s)] = np.inf
+    s = s + np.float32(0.0)                      # -0 -> +0
+    M = s.shape[0]
+    order = sorted(range(M), key=lambda i: (-float(s[i]), i))
+    return np.array(sorted(order[:r]), dtype=np.int32)
+
+
+def random_projection(Q: np.ndarray, X: np.ndarray) -> np.ndarray:
+    """F_r = Q^T X: [r][C] from Q [M][r] and X [M][C] (Algorithm 1, RP step)."""
+    return Q.T @ X
+
+
+def upsample_bilinear(F: np.ndarray, hw_in, hw_out) -> np.ndarray:
+    """Up(.) on a row-major (h, w) token grid, per channel: bilinear, half-pixel
+    centres, source coordinate clamped at 0, neighbours clamped at the edge.
+    F is [h_in*w_in][C]; returns [h_out*w_out][C].  Equal sizes give the identity."""
+    h0, w0 = hw_in
+    h1, w1 = hw_out
+    C = F.shape[-1]
+    G = F.reshape(h0, w0, C)
+    out = np.empty((h1, w1, C), dtype=F.dtype)
+    for y in range(h1):
+        sy = max((y + 0.5) * h0 / h1 - 0.5, 0.0)
+        y0 = min(int(math.floor(sy)), h0 - 1)
+        y1 = min(y0 + 1, h0 - 1)
+        fy = sy - y0
+        for x in range(w1):
+            sx = max((x + 0.5) * w0 / w1 - 0.5, 0.0)
+            x0 = min(int(math.floor(sx)), w0 - 1)
+            x1 = min(x0 + 1, w0 - 1)
+            fx = sx - x0
+            top = (1.0 - fx) * G[y0, x0] + fx * G[y0, x1]
+            bot = (1.0 - fx) * G[y1, x0] + fx * G[y1, x1]
+            out[y, x] = (1.0 - fy) * top + fy * bot
+    return out.reshape(h1 * w1, C)
+
+
+def rtr_restore(F_r_out: np.ndarray, idx: np.ndarray, cache_up: np.ndarray) -> np.ndarray:
+    """Eq. "redefine": row idx[j] takes row j of the block output, every other row
+    takes the upsampled cached row."""
+    out = cache_up.copy()
+    out[idx] = F_r_out
+    return out
+
+
+def rank_from_keep_ratio(M: int, rho: float) -> int:
+    return max(1, min(M, int(math.floor(rho * M + 0.5))))
+
+
+def rank_from_table_ratio(M: int, C: int, ratio: float) -> int:
+    """r for a tabulated rank ratio: the ratio is of n = min(M, d) singular values
+    (Sec. 3.2, low-rank paragraph)."""
+    n = min(M, C)
+    return max(1, min(M, int(math.floor(ratio * n + 0.5))))
+
+
+def energy_rank(X: np.ndarray, alpha: float) -> int:
+    """r = min{ r : eta_r >= alpha }, eta_r = sum_{i<=r} sigma_i^2 / sum_i sigma_i^2
+    (Eq. "low_rank_percent")."""
+    sv = np.linalg.svd(np.asarray(X, dtype=np.float64), compute_uv=False)
+    eta = np.cumsum(sv ** 2) / np.sum(sv ** 2)
+    return int(np.searchsorted(eta, alpha - 1e-15) + 1)
+
+
+# Rank ratios per block chunk (rows) and late scale 40 / 48 / 64 (columns) of the
+# Infinity backbone at alpha = 0.96 (App. A.1, rank table; means only).
+INFINITY_RANK_RATIO = (
+    (0.016, 0.013, 0.008),
+    (0.136, 0.117, 0.054),
+    (0.210, 0.189, 0.083),
+    (0.250, 0.222, 0.066),
+    (0.256, 0.234, 0.056),
+    (0.198, 0.183, 0.029),
+    (0.157, 0.134, 0.038),
+    (0.191, 0.163, 0.055),
+)
+
+# --------------------------------------------------------------------------- the block
+
+
+def block_forward(x: np.ndarray, ada6: np.ndarray, w: Dict[str, np.ndarray], K_cache: np.ndarray,
+                  V_cache: np.ndarray, n_heads: int, eps: float, cross_kv=None,
+                  query_rows: Optional[np.ndarray] = None):
+    """One AdaLN transformer block on rows x [n][C].
+
+    Keys/values are the committed cache rows followed by this call's own rows (no
+    mask inside the scale).  Returns (x_out, k_new, v_new).  With query_rows the
+    output is computed for that subset of rows only (keys still come from all rows).
+    """
+    sh1, sc1, g1, sh2, sc2, g2 = ada6
+    C = x.shape[-1]
+    y = modulate(x, sh1, sc1, eps)
+    qkv = y @ w["w_qkv"].T + w["b_qkv"]
+    q, k, v = qkv[:, :C], qkv[:, C:2 * C], qkv[:, 2 * C:]
+    K_all = np.concatenate([K_cache, k], axis=0)
+    V_all = np.concatenate([V_cache, v], axis=0)
+    if query_rows is not None:
+        x = x[query_rows]
+        q = q[query_rows]
+    a = attention(q, K_all, V_all, n_heads)
+    x = x + g1 * (a @ w["w_o"].T + w["b_o"])
+    if cross_kv is not None:
+        Kc, Vc = cross_kv
+        yc = layer_norm(x, eps) * w["ln_c_gamma"]
+        qc = yc @ w["w_cq"].T
+        x = x + attention(qc, Kc, Vc, n_heads) @ w["w_co"].T
+    y = modulate(x, sh2, sc2, eps)
+    hdn = gelu_tanh(y @ w["w_fc1"].T + w["b_fc1"])
+    x = x + g2 * (hdn @ w["w_fc2"].T + w["b_fc2"])
+    return x, k, v
+
+
+# --------------------------------------------------------------------------- the step, with state
+
+
+class Policy:
+    """Per-call policy of a scale step (mirrors the C ABI's keep policy)."""
+
+    def __init__(self, mode: str = "dense", cfg_mode: str = "pair", keep_ratio: float = 1.0,
+                 rank_per_group: Optional[Sequence[int]] = None, forced_indices=None):
+        assert mode in ("dense", "lowrank_rtr", "skip")
+        assert cfg_mode in ("pair", "null_only")
+        self.mode, self.cfg_mode = mode, cfg_mode
+        self.keep_ratio, self.rank_per_group = keep_ratio, rank_per_group
+        self.forced_indices = forced_indices      # [B_eff][G] -> int array, or None
+
+
+class Oracle:
+    """State across scale steps: weights, hoisted conditioning, the multi-scale KV
+    cache per block and batch element, and the block-group outputs of the last
+    stepped scale."""
+
+    def __init__(self, weights: List[Dict[str, np.ndarray]], n_heads: int, blocks_per_group: int,
+                 scale_hw: Sequence, ln_eps: float = 1e-6, dtype=np.float64):
+        self.dt = dtype
+        self.w = [{k: np.asarray(v, dtype=dtype) for k, v in blk.items()} for blk in weights]
+        self.n_blocks = len(weights)
+        self.bpg = blocks_per_group
+        self.G = self.n_blocks // blocks_per_group
+        self.H = n_heads
+        self.hw = [tuple(x) for x in scale_hw]
+        self.eps = ln_eps
+        self.C = self.w[0]["w_o"].shape[0]
+        self.cross = "w_cq" in self.w[0]
+        self.reset()
+
+    def reset(self):
+        self.B = 0
+        self.ada = None
+        self.cross_kv = None
+        self.K = self.V = None
+        self.staged = None
+        self.group_cache = None          # [G][B] -> [M][C] of scale self.cache_scale
+        self.cache_scale = -1
+        self.proj: Dict = {}
+        self.last_indices = None
+
+    def set_cond(self, cond: np.ndarray, context: Optional[np.ndarray] = None):
+        cond = np.asarray(cond, dtype=self.dt)
+        self.B = cond.shape[0]
+        self.ada = [[ada_vectors(cond[b], w["w_ada"], w["b_ada"]) for b in range(self.B)] for w in self.w]
+        C = self.C
+        if self.cross:
+            ctx = np.asarray(context, dtype=self.dt)
+            self.cross_kv = []
+            for w in self.w:
+                per_b = []
+                for b in range(self.B):
+                    kv = ctx[b] @ w["w_ckv"].T
+                    per_b.append((kv[:, :C], kv[:, C:]))
+                self.cross_kv.append(per_b)
+        empty = np.zeros((0, C), dtype=self.dt)
+        self.K = [[empty for _ in range(self.B)] for _ in range(self.n_blocks)]
+        self.V = [[empty for _ in range(self.B)] for _ in range(self.n_blocks)]
+        self.staged = None
+
+    def set_projection(self, scale_idx: int, group: int, Q: np.ndarray):
+        self.proj[(scale_idx, group)] = np.asarray(Q, dtype=self.dt)
+
+    def load_kv(self, K: np.ndarray, V: np.ndarray):
+        """Stand-in earlier scales: K, V [n_blocks][B][L][C] become the committed cache."""
+        for blk in range(self.n_blocks):
+            for b in range(self.B):
+                self.K[blk][b] = np.asarray(K[blk][b], dtype=self.dt)
+                self.V[blk][b] = np.asarray(V[blk][b], dtype=self.dt)
+
+    def load_group_cache(self, scale_idx: int, cache: np.ndarray):
+        """Stand-in block-group outputs of scale scale_idx: [G][B][M][C]."""
+        self.group_cache = [[np.asarray(cache[g][b], dtype=self.dt) for b in range(self.B)]
+                            for g in range(self.G)]
+        self.cache_scale = scale_idx
+
+    def ranks(self, M: int, pol: Policy) -> List[int]:
+        if pol.mode == "dense":
+            return [M] * self.G
+        if pol.rank_per_group is not None:
+            return [int(r) for r in pol.rank_per_group]
+        return [rank_from_keep_ratio(M, pol.keep_ratio)] * self.G
+
+    def scale_step(self, tokens: np.ndarray, scale_idx: int, pol: Policy) -> Optional[np.ndarray]:
+        """One scale step.  tokens [B][M][C]; returns [B_eff][M][C] (None for skip)."""
+        if pol.mode == "skip":
+            return None
+        tokens = np.asarray(tokens, dtype=self.dt)
+        B, M, C = tokens.shape
+        assert B == self.B and M == self.hw[scale_idx][0] * self.hw[scale_idx][1]
+        elems = list(range(B)) if pol.cfg_mode == "pair" else list(range(1, B, 2))
+        ranks = self.ranks(M, pol)
+        new_cache = [[None] * B for _ in range(self.G)]
+        staged = [[None] * B for _ in range(self.n_blocks)]
+        indices = [[None] * self.G for _ in elems]
+        outs = []
+        for e, b in enumerate(elems):
+            X = tokens[b]
+            for g in range(self.G):
+                r = ranks[g]
+                blocks = range(g * self.bpg, (g + 1) * self.bpg)
+                if r >= M:                                 # dense: Q = I, I = all rows
+                    x = X
+                    idx = np.arange(M, dtype=np.int32)
+                else:
+                    if pol.forced_indices is not None:
+                        idx = np.asarray(pol.forced_indices[e][g], dtype=np.int32)
+                    else:
+                        idx = select_top_r(row_scores(X, np.float32), r)
+                    x = random_projection(self.proj[(scale_idx, g)], X)
+                for blk in blocks:
+                    ckv = self.cross_kv[blk][b] if self.cross else None
+                    x, k, v = block_forward(x, self.ada[blk][b], self.w[blk], self.K[blk][b],
+                                            self.V[blk][b], self.H, self.eps, ckv)
+                    staged[blk][b] = (k, v)
+                if r >= M:
+                    out = x
+                else:
+                    assert self.group_cache is not None and self.cache_scale >= 0
+                    up = upsample_bilinear(self.group_cache[g][b], self.hw[self.cache_scale],
+                                           self.hw[scale_idx])
+                    out = rtr_restore(x, idx, up)
+                indices[e][g] = idx
+                new_cache[g][b] = out
+                X = out
+            outs.append(X)
+        # elements not computed keep no cache entry for this scale
+        self.group_cache = new_cache
+        self.cache_scale = scale_idx
+        self.staged = (scale_idx, staged)
+        self.last_indices = indices
+        return np.stack(outs, axis=0)
+
+    def kv_append(self, scale_idx: int):
+        """Commit the rows the last step staged (per block: the r rows its group computed)."""
+        assert self.staged is not None and self.staged[0] == scale_idx
+        for blk in range(self.n_blocks):
+            for b in range(self.B):
+                if self.staged[1][blk][b] is not None:
+                    k, v = self.staged[1][blk][b]
+                    self.K[blk][b] = np.concatenate([self.K[blk][b], k], axis=0)
+                    self.V[blk][b] = np.concatenate([self.V[blk][b], v], axis=0)
+        self.staged = None
+
+    def cache_len(self, blk: int, b: int) -> int:
+        return self.K[blk][b].shape[0]
