@@ -1,0 +1,200 @@
+/*
+ * libfvar -- late-scale step of VAR next-scale prediction under FasterVAR, for NVIDIA B200 (sm_100a).
+ *
+ * One call, fvar_scale_step, runs a stack of AdaLN transformer blocks over the tokens of one
+ * scale; the current scale's rows attend over a multi-scale KV cache.  It runs either densely or
+ * under the paper's fidelity-refinement approximation: null-prompt-only CFG (Sec. 3.2, "Semantic
+ * irrelevance"), random projection of the M token rows to r rows (Sec. 3.3 "Random Projection";
+ * Algorithm 1), the block forward on r rows, and representative token restoration (Sec. 3.3
+ * "RTR", Eq. "upcache" and Eq. "redefine").
+ *
+ * Conventions
+ *   - "dev" pointers are device memory of the current CUDA device, "host" pointers are host memory.
+ *   - bf16 arrays are raw 16-bit patterns.  All matrices are row-major.
+ *   - Weight matrices are stored [out_features][in_features] (y = x W^T + b).
+ *   - The library never allocates or frees device memory and never synchronises unless a function
+ *     says so; all work is enqueued on the stream given to fvar_init.  The caller owns weights,
+ *     tokens, outputs, workspace and the stream, and keeps them alive while the context exists.
+ *   - Every function returns an fvar_status; nothing is thrown across this boundary.  Errors found
+ *     by a kernel (a bounded wait that ran out) are recorded in a device status word that
+ *     fvar_poll_status reads after the caller has synchronised.
+ *   - A CFG pair is two adjacent batch elements: element 2p is the prompt-conditioned branch,
+ *     element 2p+1 the null-prompt branch.
+ */
+#ifndef FVAR_H_
+#define FVAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fvar_ctx fvar_ctx;
+
+typedef enum {
+  FVAR_OK = 0,
+  FVAR_EINVAL = 1,       /* bad argument */
+  FVAR_ENOMEM = 2,       /* workspace too small */
+  FVAR_ESTATE = 3,       /* call out of order (see each function) */
+  FVAR_ECUDA = 4,        /* a CUDA runtime / driver call failed */
+  FVAR_ETIMEOUT = 5,     /* a bounded device-side wait ran out (fvar_poll_status) */
+  FVAR_EUNSUPPORTED = 6  /* shape outside what the kernels support */
+} fvar_status;
+
+enum { FVAR_DENSE = 0, FVAR_LOWRANK_RTR = 1, FVAR_SKIP = 2 };      /* fvar_keep_policy.mode     */
+enum { FVAR_CFG_PAIR = 0, FVAR_CFG_NULL_ONLY = 1 };                /* fvar_keep_policy.cfg_mode */
+
+/* Static shape of the block stack. */
+typedef struct {
+  int n_blocks;          /* transformer blocks                                                */
+  int blocks_per_group;  /* RP / RTR are applied per block group ("at the block level", Sec. 3.3) */
+  int width;             /* C (the paper's d); multiple of 64                                 */
+  int n_heads;           /* H                                                                 */
+  int head_dim;          /* D: 64 or 128; H * D == C                                          */
+  int ffn_dim;           /* F; multiple of 64                                                 */
+  int n_scales;
+  const int *scale_hw;   /* host, 2 * n_scales ints: h_k, w_k (h != w is legal)               */
+  int max_batch;         /* largest B given to fvar_set_cond                                  */
+  int has_cross_attn;    /* 1: blocks also cross-attend to ctx_len context tokens             */
+  int ctx_len;
+  int ctx_width;         /* multiple of 64                                                    */
+  float ln_eps;          /* LayerNorm epsilon (1e-6 in the reference workloads)               */
+} fvar_cfg;
+
+/* Per-block parameters: each member is a host array of n_blocks device pointers to bf16 data.
+ * w_qkv [3C][C], b_qkv [3C], w_o [C][C], b_o [C], w_fc1 [F][C], b_fc1 [F], w_fc2 [C][F], b_fc2 [C],
+ * w_ada [6C][C], b_ada [6C] (chunks shift1, scale1, gate1, shift2, scale2, gate2);
+ * cross-attention (NULL arrays when has_cross_attn == 0): w_cq [C][C], w_ckv [2C][ctx_width]
+ * (keys then values), w_co [C][C], ln_c_gamma [C]. */
+typedef struct {
+  const void *const *w_qkv, *const *b_qkv, *const *w_o, *const *b_o;
+  const void *const *w_fc1, *const *b_fc1, *const *w_fc2, *const *b_fc2;
+  const void *const *w_ada, *const *b_ada;
+  const void *const *w_cq, *const *w_ckv, *const *w_co, *const *ln_c_gamma;
+} fvar_weights;
+
+/* Per-call policy of a scale step. */
+typedef struct {
+  int mode;                   /* FVAR_DENSE | FVAR_LOWRANK_RTR | FVAR_SKIP                         */
+  int cfg_mode;               /* FVAR_CFG_PAIR: all B elements; FVAR_CFG_NULL_ONLY: elements 2p+1  */
+  const int *rank_per_group;  /* host, n_groups ints: r per block group; NULL -> keep_ratio        */
+  float keep_ratio;           /* r = floor(keep_ratio * M + 0.5) for every group                   */
+  const int *forced_indices;  /* dev, test hook: [n_groups][B_eff][r_max] ascending row indices that
+                                 replace the selection (r_max = largest r of the call); NULL in production */
+} fvar_keep_policy;
+
+/* Bytes of device workspace fvar_init needs for this shape (0 if the shape is invalid). */
+size_t fvar_workspace_bytes(const fvar_cfg *cfg);
+
+/* Create a context.  `workspace` (dev, 1024-byte aligned, >= fvar_workspace_bytes) holds the KV
+ * cache, the block-group output caches, projection matrices, index lists, activations and the
+ * status word; it is zeroed here (enqueued on `cuda_stream`, a cudaStream_t passed as void*).
+ * Builds the TMA descriptors of the weights.  FVAR_EINVAL / FVAR_EUNSUPPORTED on a bad shape,
+ * FVAR_ENOMEM if `bytes` is too small, FVAR_ECUDA if no sm_100 device is current. */
+fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *workspace, size_t bytes,
+                      void *cuda_stream, fvar_ctx **out);
+
+/* Hoisted conditioning (constant across scales): AdaLN vectors W_ada SiLU(c_b) + b_ada for every
+ * block and batch element, and the cross-attention keys/values of the context tokens.  Also empties
+ * the KV cache (a new generation starts).  cond dev bf16 [B][C]; context dev bf16
+ * [B][ctx_len][ctx_width] or NULL without cross-attention.  B <= max_batch. */
+fvar_status fvar_set_cond(fvar_ctx *ctx, int B, const void *cond, const void *context);
+
+/* Random-projection matrix Q of Sec. 3.3 (entries N(0, 1/r)) for one (scale, block group), given
+ * TRANSPOSED: Qt dev bf16 [r][M].  Copied into the workspace; shared by the whole batch.  Must be
+ * set before a FVAR_LOWRANK_RTR step whose group rank is r < M. */
+fvar_status fvar_set_projection(fvar_ctx *ctx, int scale_idx, int group, const void *Qt, int r);
+
+/* One scale step (Algorithm 1: the dense loop body, or the fidelity-refinement loop body RP -> blocks
+ * -> RTR).  tokens dev bf16 [B][M][C] with M = h_k * w_k; out dev bf16 [B_eff][M][C], B_eff = B
+ * (pair) or B/2 (null-only).  Stages this scale's K/V rows at the cache tail; they become visible
+ * to later scales only after fvar_kv_append.  A group with r == M runs the dense path (Q = I).
+ * FVAR_LOWRANK_RTR needs the previous stepped scale's group outputs (FVAR_ESTATE otherwise) and a
+ * projection for every group with r < M.  FVAR_SKIP enqueues nothing.  scale_idx must not decrease
+ * (FVAR_ESTATE); a FVAR_CFG_PAIR step after a FVAR_CFG_NULL_ONLY step is FVAR_ESTATE. */
+fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, const fvar_keep_policy *policy,
+                            void *out);
+
+/* Same step with HOST buffers: copies tokens host->dev, runs the step, copies out dev->host, and
+ * synchronises the stream before returning.  Pinned host memory makes the copies asynchronous. */
+fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int scale_idx,
+                                 const fvar_keep_policy *policy, void *out_host);
+
+/* Commit the rows staged by the last step of `scale_idx` (O(1), host only).  FVAR_ESTATE if that
+ * scale was not the last one stepped or was already appended. */
+fvar_status fvar_kv_append(fvar_ctx *ctx, int scale_idx);
+
+/* Row indices chosen by the last FVAR_LOWRANK_RTR step for `group`: copies [B_eff][r] int32 into
+ * idx_dev (device to device, stream-ordered) and stores r in *count_host. */
+fvar_status fvar_get_indices(fvar_ctx *ctx, int group, int *idx_dev, int *count_host);
+
+/* fp32 output of block group `group` at the last stepped scale: [B][M][C] floats copied to out_dev
+ * (rows of batch elements the step did not compute are unspecified). */
+fvar_status fvar_get_group_output(fvar_ctx *ctx, int group, float *out_dev);
+
+/* Stand-ins for earlier scales (tests, benchmarks): load committed K/V rows, K and V dev bf16
+ * [n_blocks][B][L][C], as the cache contents (cache length becomes L for every block), and load
+ * block-group outputs dev fp32 [n_groups][B][M][C] as those of scale `scale_idx`. */
+fvar_status fvar_load_kv(fvar_ctx *ctx, const void *K, const void *V, int L);
+fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cache);
+
+/* Committed cache rows of `block` (host value). */
+int fvar_cache_len(const fvar_ctx *ctx, int block);
+
+/* Number of kernels the library has launched on this context since fvar_init (host counter). */
+long long fvar_launch_count(const fvar_ctx *ctx);
+
+/* Synchronises the stream, reads the device status word and clears it.  FVAR_OK, FVAR_ETIMEOUT,
+ * or FVAR_ECUDA. */
+fvar_status fvar_poll_status(fvar_ctx *ctx);
+
+/* Empties the KV cache and the group caches (host state only; device memory is not cleared). */
+fvar_status fvar_reset(fvar_ctx *ctx);
+void fvar_destroy(fvar_ctx *ctx);
+/* Message of the last error on this context (or of the last failed fvar_init when ctx is NULL). */
+const char *fvar_last_error(const fvar_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------
+ * Kernel-level entry points: the individual steps of the path, callable on caller-owned device
+ * buffers.  `stream` is a cudaStream_t passed as void*.  They synchronise nothing.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Row score of Sec. 3.3 (RTR): s[b][i] = sum_c x[b][i][c]^2 (the numerator of p_i; the common
+ * denominator ||X||_F^2 does not change the order).  x dev fp32 [B][M][C], C % 4 == 0; scores dev fp32 [B][M]. */
+fvar_status fvar_row_scores(const float *x, int B, int M, int C, float *scores, void *stream);
+
+/* Index set I of Sec. 3.3 / Algorithm 1: per batch element the r highest-scoring rows, ascending.
+ * Order: score descending then index ascending; NaN ranks as +inf; -0 == +0.
+ * scores dev fp32 [B][M]; idx dev int32 [B][r]; inv dev int32 [B][M] (position j of row i in idx, or -1). */
+fvar_status fvar_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, void *stream);
+
+/* LayerNorm (no affine, biased variance) + AdaLN modulation: y = LN(x) * (1 + scale) + shift.
+ * x dev fp32 [R][C]; shift/scale dev fp32, row i uses the vectors at offset (i / rows_per_batch) *
+ * vec_stride floats; y dev bf16 [R][C].  C % 8 == 0, C <= 8192. */
+fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, const float *shift,
+                             const float *scale, long long vec_stride, float eps, void *y, void *stream);
+
+/* out[R][N] (fp32) = A[R][K] W[N][K]^T + bias[N] on the tensor cores (bf16 operands, fp32
+ * accumulation).  A, W, bias dev bf16 (bias may be NULL); K % 8 == 0; lda = ldw = K. */
+fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out,
+                           void *stream);
+
+/* softmax(q k^T / sqrt(D)) v per head over the first L rows of a cache in the library's layout:
+ * q dev bf16 [B][r][H*D]; Kc dev bf16 [B][H][L_cap][D]; Vt dev bf16 [B][H][D][L_cap] (values stored
+ * transposed); out dev bf16 [B][r][H*D].  D in {64, 128}; L_cap % 8 == 0; 1 <= L <= L_cap. */
+fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B, int H, int r, int D, int L,
+                           int L_cap, void *out, void *stream);
+
+/* Restoration fill of Eq. "redefine" with Eq. "upcache": for every row i of batch element b with
+ * inv[b][i] < 0, out[b][i] = Up(prev[b])[i], bilinear with half-pixel centres on the (h, w) grid.
+ * prev dev fp32 [B][h0*w0][C]; out dev fp32 [B][h1*w1][C]; rows with inv >= 0 are left untouched;
+ * inv == NULL fills every row.  C % 4 == 0. */
+fvar_status fvar_rtr_fill(const float *prev, int B, int h0, int w0, int h1, int w1, int C, const int *inv,
+                          float *out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FVAR_H_ */

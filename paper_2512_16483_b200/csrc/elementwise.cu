@@ -1,0 +1,424 @@
+// HBM-bound kernels of the path: row score, top-r selection with ballot prefix-sum compaction,
+// LayerNorm + AdaLN modulation, restoration fill (bilinear Up of the cached group output), and
+// the layout / type conversions between them.  All use 16-byte vector accesses.
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace fvar {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row score s_i = sum_c x[i][c]^2: one warp per row, float4 loads.
+__global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict__ x, long long rows, int C,
+                                                         float *__restrict__ scores) {
+  const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const float4 *p = reinterpret_cast<const float4 *>(x + row * C);
+  float acc = 0.f;
+  for (int i = lane; i < C / 4; i += 32) {
+    float4 v = __ldg(p + i);
+    acc = fmaf(v.x, v.x, acc);
+    acc = fmaf(v.y, v.y, acc);
+    acc = fmaf(v.z, v.z, acc);
+    acc = fmaf(v.w, v.w, acc);
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) scores[row] = acc;
+}
+
+cudaError_t launch_row_scores(const float *x, long long rows, int C, float *scores, cudaStream_t st) {
+  if (rows <= 0) return cudaSuccess;
+  row_scores_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(x, rows, C, scores);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Top-r selection.  One CTA per batch element.  The fp32 scores map to unsigned keys whose order
+// is the float order (NaN -> +inf, -0 -> +0); a 4-pass, 8-bit radix select finds the key of the
+// r-th largest; rows are then compacted in ascending index order: every key above the threshold,
+// plus the first (r - #above) rows whose key equals it.  Prefix sums use warp ballots.
+constexpr int kSelThreads = 1024;
+
+__device__ __forceinline__ unsigned score_key(float s) {
+  if (s != s) s = INFINITY;
+  s += 0.0f;                                    // -0 -> +0
+  const unsigned u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_topr_kernel(const float *__restrict__ scores, int M, int r,
+                                                                  int *__restrict__ idx, int *__restrict__ inv) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned s_prefix, s_need;
+  __shared__ int warp_gt[32], warp_eq[32];
+  __shared__ int base_gt, base_eq;
+  const int b = blockIdx.x;
+  const float *s = scores + static_cast<long long>(b) * M;
+  int *idx_b = idx + static_cast<long long>(b) * r;
+  int *inv_b = inv + static_cast<long long>(b) * M;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // radix select: after the loop, `prefix` is the key of the r-th largest and `need` is how many
+  // rows with exactly that key are taken
+  unsigned prefix = 0, mask = 0, need = static_cast<unsigned>(r);
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int i = tid; i < M; i += kSelThreads) {
+      const unsigned k = score_key(s[i]);
+      if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned acc = 0;
+      int d = 255;
+      for (; d > 0; --d) {
+        if (acc + hist[d] >= need) break;
+        acc += hist[d];
+      }
+      s_prefix = prefix | (static_cast<unsigned>(d) << shift);
+      s_need = need - acc;
+    }
+    __syncthreads();
+    prefix = s_prefix;
+    need = s_need;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const unsigned thr = prefix;
+
+  if (tid == 0) {
+    base_gt = 0;
+    base_eq = 0;
+  }
+  __syncthreads();
+  for (int start = 0; start < M; start += kSelThreads) {
+    const int i = start + tid;
+    const unsigned k = (i < M) ? score_key(s[i]) : 0u;
+    const bool gt = (i < M) && k > thr;
+    const bool eq = (i < M) && k == thr;
+    const unsigned bgt = __ballot_sync(0xffffffffu, gt), beq = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) {
+      warp_gt[warp] = __popc(bgt);
+      warp_eq[warp] = __popc(beq);
+    }
+    __syncthreads();
+    if (warp == 0) {                           // exclusive scan of the 32 per-warp counts
+      int g = warp_gt[lane], q = warp_eq[lane];
+      int gi = g, qi = q;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int tg = __shfl_up_sync(0xffffffffu, gi, o), tq = __shfl_up_sync(0xffffffffu, qi, o);
+        if (lane >= o) {
+          gi += tg;
+          qi += tq;
+        }
+      }
+      warp_gt[lane] = gi - g;
+      warp_eq[lane] = qi - q;
+    }
+    __syncthreads();
+    const unsigned below = (1u << lane) - 1u;
+    const int n_gt = base_gt + warp_gt[warp] + __popc(bgt & below);   // rows above thr before i
+    const int n_eq = base_eq + warp_eq[warp] + __popc(beq & below);   // rows equal to thr before i
+    if (i < M) {
+      const bool take = gt || (eq && n_eq < static_cast<int>(need));
+      const int pos = n_gt + min(n_eq, static_cast<int>(need));
+      if (take) idx_b[pos] = i;
+      inv_b[i] = take ? pos : -1;
+    }
+    __syncthreads();
+    if (tid == kSelThreads - 1) {
+      base_gt = n_gt + (gt ? 1 : 0);
+      base_eq = n_eq + (eq ? 1 : 0);
+    }
+    __syncthreads();
+  }
+}
+
+cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st) {
+  if (B <= 0) return cudaSuccess;
+  select_topr_kernel<<<B, kSelThreads, 0, st>>>(scores, M, r, idx, inv);
+  return cudaGetLastError();
+}
+
+// Test hook: take the caller's index lists instead of selecting.  Checks range and strict ascent;
+// a bad list sets a status bit and the offending entry is clamped into range.
+__global__ void copy_indices_kernel(const int *__restrict__ forced, int M, int r, int ld_forced,
+                                    int *__restrict__ idx, int *__restrict__ inv, unsigned *status) {
+  const int b = blockIdx.x;
+  const int *f = forced + static_cast<long long>(b) * ld_forced;
+  int *idx_b = idx + static_cast<long long>(b) * r;
+  int *inv_b = inv + static_cast<long long>(b) * M;
+  for (int i = threadIdx.x; i < M; i += blockDim.x) inv_b[i] = -1;
+  __syncthreads();
+  for (int j = threadIdx.x; j < r; j += blockDim.x) {
+    int v = f[j];
+    const bool bad = v < 0 || v >= M || (j > 0 && f[j - 1] >= v);
+    if (bad) atomicOr(status, kStatusBadIndex);
+    v = min(max(v, 0), M - 1);
+    idx_b[j] = v;
+    inv_b[v] = j;
+  }
+}
+
+cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_forced, int *idx, int *inv,
+                                unsigned *status, cudaStream_t st) {
+  copy_indices_kernel<<<B, 256, 0, st>>>(forced, M, r, ld_forced, idx, inv, status);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// y = LN(x) * (1 + scale) + shift  (or LN(x) * gamma): one CTA of 128 threads per row, the row
+// held in registers (two-pass mean / variance), bf16 output, 16-byte accesses.
+constexpr int kLnThreads = 128;
+constexpr int kLnMaxVec = 8;                    // 8 x (8 elements) x 128 threads = 8192 columns
+
+__global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__restrict__ x, RowMap xmap, int rows,
+                                                                 int C, const float *__restrict__ shift,
+                                                                 const float *__restrict__ scale,
+                                                                 long long vec_stride, int bmul, int boff,
+                                                                 const bf16 *__restrict__ gamma, float eps,
+                                                                 bf16 *__restrict__ y) {
+  __shared__ float red[kLnThreads / 32];
+  const int e = blockIdx.x / rows, j = blockIdx.x - e * rows;
+  const float *xr = x + (static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb + j) * C;
+  bf16 *yr = y + static_cast<long long>(blockIdx.x) * C;
+  const int nvec = C / 8;                       // 8-element groups in the row
+  float v[kLnMaxVec][8];
+  float sum = 0.f;
+#pragma unroll
+  for (int t = 0; t < kLnMaxVec; ++t) {
+    const int g = threadIdx.x + t * kLnThreads;
+    if (g < nvec) {
+      const float4 a = reinterpret_cast<const float4 *>(xr)[2 * g], c = reinterpret_cast<const float4 *>(xr)[2 * g + 1];
+      v[t][0] = a.x; v[t][1] = a.y; v[t][2] = a.z; v[t][3] = a.w;
+      v[t][4] = c.x; v[t][5] = c.y; v[t][6] = c.z; v[t][7] = c.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sum += v[t][i];
+    }
+  }
+  auto block_sum = [&](float val) {
+    val = warp_sum(val);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = val;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kLnThreads / 32; ++w) tot += red[w];
+    return tot;
+  };
+  const float mean = block_sum(sum) / C;
+  float sq = 0.f;
+#pragma unroll
+  for (int t = 0; t < kLnMaxVec; ++t) {
+    const int g = threadIdx.x + t * kLnThreads;
+    if (g < nvec) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float d = v[t][i] - mean;
+        sq = fmaf(d, d, sq);
+      }
+    }
+  }
+  const float rstd = rsqrtf(block_sum(sq) / C + eps);
+  const long long voff = static_cast<long long>(e * bmul + boff) * vec_stride;
+#pragma unroll
+  for (int t = 0; t < kLnMaxVec; ++t) {
+    const int g = threadIdx.x + t * kLnThreads;
+    if (g < nvec) {
+      float o[8];
+      if (gamma != nullptr) {
+        const uint4 gu = __ldg(reinterpret_cast<const uint4 *>(gamma) + g);
+        const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&gu);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 gf = __bfloat1622float2(gh[i]);
+          o[2 * i] = (v[t][2 * i] - mean) * rstd * gf.x;
+          o[2 * i + 1] = (v[t][2 * i + 1] - mean) * rstd * gf.y;
+        }
+      } else {
+        const float4 *sc = reinterpret_cast<const float4 *>(scale + voff) + 2 * g;
+        const float4 *sh = reinterpret_cast<const float4 *>(shift + voff) + 2 * g;
+        const float4 s0 = __ldg(sc), s1 = __ldg(sc + 1), h0 = __ldg(sh), h1 = __ldg(sh + 1);
+        const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        const float shv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = fmaf((v[t][i] - mean) * rstd, 1.0f + scv[i], shv[i]);
+      }
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&h2);
+      }
+      reinterpret_cast<uint4 *>(yr)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int C, const float *shift,
+                               const float *scale, long long vec_stride, int bmul, int boff, const bf16 *gamma,
+                               float eps, bf16 *y, cudaStream_t st) {
+  if (E * rows <= 0) return cudaSuccess;
+  if (C % 8 != 0 || C > 8 * kLnThreads * kLnMaxVec) return cudaErrorInvalidValue;
+  ln_modulate_kernel<<<E * rows, kLnThreads, 0, st>>>(x, xmap, rows, C, shift, scale, vec_stride, bmul, boff, gamma,
+                                                      eps, y);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Restoration fill: rows outside the index set take the bilinearly upsampled cached row
+// (half-pixel centres, source coordinate clamped at 0, neighbours clamped at the edge).
+// One warp per output row; rows inside the index set are skipped.
+__global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__ prev, float *__restrict__ out, int E,
+                                                       int bmul, int boff, int h0, int w0, int h1, int w1, int C,
+                                                       const int *__restrict__ inv) {
+  const int M1 = h1 * w1;
+  const long long gw = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (gw >= static_cast<long long>(E) * M1) return;
+  const int e = static_cast<int>(gw / M1), i = static_cast<int>(gw - static_cast<long long>(e) * M1);
+  if (inv != nullptr && inv[static_cast<long long>(e) * M1 + i] >= 0) return;
+  const int b = e * bmul + boff;
+  const int y = i / w1, xq = i - y * w1;
+  const float sy = fmaxf((y + 0.5f) * (static_cast<float>(h0) / h1) - 0.5f, 0.f);
+  const float sx = fmaxf((xq + 0.5f) * (static_cast<float>(w0) / w1) - 0.5f, 0.f);
+  const int y0 = min(static_cast<int>(sy), h0 - 1), x0 = min(static_cast<int>(sx), w0 - 1);
+  const int y1 = min(y0 + 1, h0 - 1), x1 = min(x0 + 1, w0 - 1);
+  const float fy = sy - y0, fx = sx - x0;
+  const float *src = prev + static_cast<long long>(b) * h0 * w0 * C;
+  const float4 *p00 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y0) * w0 + x0) * C);
+  const float4 *p01 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y0) * w0 + x1) * C);
+  const float4 *p10 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y1) * w0 + x0) * C);
+  const float4 *p11 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y1) * w0 + x1) * C);
+  float4 *dst = reinterpret_cast<float4 *>(out + (static_cast<long long>(b) * M1 + i) * C);
+  const float w00 = (1.f - fy) * (1.f - fx), w01 = (1.f - fy) * fx, w10 = fy * (1.f - fx), w11 = fy * fx;
+  for (int c = threadIdx.x & 31; c < C / 4; c += 32) {
+    const float4 a = __ldg(p00 + c), bq = __ldg(p01 + c), cq = __ldg(p10 + c), d = __ldg(p11 + c);
+    float4 o;
+    o.x = w00 * a.x + w01 * bq.x + w10 * cq.x + w11 * d.x;
+    o.y = w00 * a.y + w01 * bq.y + w10 * cq.y + w11 * d.y;
+    o.z = w00 * a.z + w01 * bq.z + w10 * cq.z + w11 * d.z;
+    o.w = w00 * a.w + w01 * bq.w + w10 * cq.w + w11 * d.w;
+    dst[c] = o;
+  }
+}
+
+cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1, int w1,
+                            int C, const int *inv, cudaStream_t st) {
+  const long long warps = static_cast<long long>(E) * h1 * w1;
+  if (warps <= 0) return cudaSuccess;
+  rtr_fill_kernel<<<static_cast<unsigned>((warps + 7) / 8), 256, 0, st>>>(prev, out, E, bmul, boff, h0, w0, h1, w1, C,
+                                                                         inv);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// xt[e][c][m] (bf16, row stride Mp) = x[row(e, m)][c] (fp32): 32 x 32 tiles through shared memory.
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
+                                                             int Mp, bf16 *__restrict__ xt) {
+  __shared__ float tile[32][33];
+  const int e = blockIdx.z, m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const float *src = x + static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb * C;
+  for (int k = ty; k < 32; k += 8) {
+    const int m = m0 + k, c = c0 + tx;
+    tile[k][tx] = (m < M && c < C) ? src[static_cast<long long>(m) * C + c] : 0.f;
+  }
+  __syncthreads();
+  bf16 *dst = xt + static_cast<long long>(e) * C * Mp;
+  for (int k = ty; k < 32; k += 8) {
+    const int c = c0 + k, m = m0 + tx;
+    if (c < C && m < Mp) dst[static_cast<long long>(c) * Mp + m] = __float2bfloat16_rn(m < M ? tile[tx][k] : 0.f);
+  }
+}
+
+cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mp, bf16 *xt,
+                                  cudaStream_t st) {
+  dim3 grid((Mp + 31) / 32, (C + 31) / 32, E);
+  transpose_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, Mp, xt);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+__global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__restrict__ x, long long n8) {
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n8) return;
+  const uint4 u = __ldg(reinterpret_cast<const uint4 *>(tok) + i);
+  const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+  const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]), c = __bfloat1622float2(h[2]),
+               d = __bfloat1622float2(h[3]);
+  reinterpret_cast<float4 *>(x)[2 * i] = make_float4(a.x, a.y, b.x, b.y);
+  reinterpret_cast<float4 *>(x)[2 * i + 1] = make_float4(c.x, c.y, d.x, d.y);
+}
+
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st) {
+  const long long n8 = static_cast<long long>(B) * per_elem / 8;
+  if (n8 <= 0) return cudaSuccess;
+  tokens_to_f32_kernel<<<static_cast<unsigned>((n8 + 255) / 256), 256, 0, st>>>(tok, x, n8);
+  return cudaGetLastError();
+}
+
+__global__ void out_to_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C, bf16 *__restrict__ out) {
+  const int e = blockIdx.y;
+  const long long per = static_cast<long long>(M) * C / 8;
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= per) return;
+  const float4 *src = reinterpret_cast<const float4 *>(x + static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb * C);
+  const float4 a = src[2 * i], b = src[2 * i + 1];
+  __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w),
+                 h2 = __floats2bfloat162_rn(b.x, b.y), h3 = __floats2bfloat162_rn(b.z, b.w);
+  uint4 u = make_uint4(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1),
+                       *reinterpret_cast<uint32_t *>(&h2), *reinterpret_cast<uint32_t *>(&h3));
+  reinterpret_cast<uint4 *>(out + static_cast<long long>(e) * M * C)[i] = u;
+}
+
+cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st) {
+  const long long per = static_cast<long long>(M) * C / 8;
+  dim3 grid(static_cast<unsigned>((per + 255) / 256), E);
+  out_to_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, out);
+  return cudaGetLastError();
+}
+
+__global__ void silu_bf16_kernel(const bf16 *__restrict__ in, bf16 *__restrict__ out, long long n) {
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float v = __bfloat162float(in[i]);
+  out[i] = __float2bfloat16_rn(v / (1.0f + __expf(-v)));
+}
+
+cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  silu_bf16_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(in, out, n);
+  return cudaGetLastError();
+}
+
+// K, V [B][L][H*D] -> cache layout K [B][H][L_cap][D], V^T [B][H][D][L_cap] (one block's worth).
+__global__ void load_kv_kernel(const bf16 *__restrict__ K, const bf16 *__restrict__ V, int L, int H, int D, int L_cap,
+                               bf16 *__restrict__ kc, bf16 *__restrict__ vt) {
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int C = H * D;
+  for (long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; t < static_cast<long long>(L) * D;
+       t += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int l = static_cast<int>(t / D), d = static_cast<int>(t - static_cast<long long>(l) * D);
+    const long long src = (static_cast<long long>(b) * L + l) * C + h * D + d;
+    kc[((static_cast<long long>(b) * H + h) * L_cap + l) * D + d] = K[src];
+    vt[((static_cast<long long>(b) * H + h) * D + d) * L_cap + l] = V[src];
+  }
+}
+
+cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,
+                           cudaStream_t st) {
+  if (L <= 0) return cudaSuccess;
+  dim3 grid(static_cast<unsigned>((static_cast<long long>(L) * D + 255) / 256), H, B);
+  load_kv_kernel<<<grid, 256, 0, st>>>(K, V, L, H, D, L_cap, kc, vt);
+  return cudaGetLastError();
+}
+
+}  // namespace fvar

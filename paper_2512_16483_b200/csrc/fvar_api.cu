@@ -1,0 +1,806 @@
+// Host side of libfvar: the C ABI, workspace layout, TMA descriptors and the sequencing of one
+// scale step over block groups.  See include/fvar.h for the contract of every entry point.
+#include <stdio.h>
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include <string>
+#include <vector>
+
+#include "../../include/fvar.h"
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace fvar {
+
+// ------------------------------------------------------------------------------------------------
+// Tensor maps (the driver entry point is fetched through the runtime: no link against libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+bool tmap_init_driver() {
+  if (g_encode) return true;
+  void *fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess) return false;
+  if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return false;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return true;
+}
+
+bool tmap_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t ld_elems, uint32_t box_rows) {
+  if (!tmap_init_driver()) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld_elems * 2) % 16 || box_rows == 0 || box_rows > 256) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld_elems * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1_elems,
+             uint64_t ld2_elems, uint32_t box0, uint32_t box1) {
+  if (!tmap_init_driver()) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld1_elems * 2) % 16 || (ld2_elems * 2) % 16 || box1 == 0 ||
+      box1 > 256)
+    return false;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {ld1_elems * 2, ld2_elems * 2};
+  cuuint32_t box[3] = {box0, box1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Status word used by the kernel-level entry points (contexts carry their own in the workspace).
+__device__ unsigned g_kernel_status;
+
+static std::string g_init_error;
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
+static const int kBNs[3] = {64, 128, 256};
+
+enum WeightId { W_QKV = 0, W_O, W_FC1, W_FC2, W_ADA, W_CQ, W_CKV, W_CO, W_COUNT };
+
+}  // namespace fvar
+
+using namespace fvar;
+
+struct fvar_ctx {
+  fvar_cfg cfg;
+  std::vector<int> hw;                 // 2 * n_scales
+  std::vector<int> Mk;                 // tokens per scale
+  int G, C, F, H, D, Bmax, Mmax, L_cap, ctx_cap, num_sms;
+  cudaStream_t st;
+  std::string err;
+  long long launches;
+  // weights (device pointers per block)
+  std::vector<const bf16 *> w[W_COUNT];
+  std::vector<const bf16 *> b_qkv, b_o, b_fc1, b_fc2, b_ada, ln_c_gamma;
+  std::vector<CUtensorMap> wmap;       // [blk][W_COUNT][3]
+  // workspace regions
+  uint8_t *ws;
+  size_t ws_bytes;
+  unsigned *status;
+  bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *xt, *qt_pool;
+  float *ada, *gcache, *x0, *xs, *scores;
+  int *idx, *inv;
+  std::vector<size_t> qt_off;          // [scale][group] offset (elements) into qt_pool
+  std::vector<int> qt_r;               // [scale][group] rank of the stored projection (0: none)
+  std::vector<CUtensorMap> qt_map;     // [scale][group]
+  std::vector<CUtensorMap> xt_map;     // [scale][3]
+  std::vector<CUtensorMap> kmap, vmap, ckmap, cvmap;   // per block
+  CUtensorMap y_map, a_map, q_map, h_map, silu_map;
+  // state
+  int B;                               // batch of the current generation (0: no cond set)
+  std::vector<int> len;                // committed cache rows per block
+  std::vector<int> staged;             // rows staged by the last step per block
+  int staged_scale;                    // scale whose rows are staged (-1: none)
+  int last_scale;                      // last stepped scale (-1: none)
+  int cache_scale;                     // scale of the valid group cache (-1: none)
+  int cache_slot;                      // slot holding it
+  int null_only_seen;
+  std::vector<int> last_rank;          // r per group of the last step
+  int last_E, last_M;
+
+  size_t kv_block_elems() const { return static_cast<size_t>(Bmax) * H * L_cap * D; }
+  size_t ckv_block_elems() const { return static_cast<size_t>(Bmax) * H * ctx_cap * D; }
+  float *gslot(int slot, int g) const {
+    return gcache + (static_cast<size_t>(slot) * G + g) * Bmax * Mmax * C;
+  }
+  const CUtensorMap &wm(int blk, int wid, int bn) const { return wmap[(blk * W_COUNT + wid) * 3 + bn_index(bn)]; }
+};
+
+namespace {
+
+struct Layout {
+  size_t status, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
+  std::vector<size_t> qt_off;
+};
+
+bool shape_ok(const fvar_cfg *c, std::string *why) {
+  auto bad = [&](const char *m) { if (why) *why = m; return false; };
+  if (!c || !c->scale_hw) return bad("null cfg");
+  if (c->n_blocks <= 0 || c->blocks_per_group <= 0 || c->n_blocks % c->blocks_per_group) return bad("block grouping");
+  if (c->width <= 0 || c->width % 64 || c->width > 8192) return bad("width must be a multiple of 64, <= 8192");
+  if (c->head_dim != 64 && c->head_dim != 128) return bad("head_dim must be 64 or 128");
+  if (c->n_heads * c->head_dim != c->width) return bad("n_heads * head_dim != width");
+  if (c->ffn_dim <= 0 || c->ffn_dim % 64) return bad("ffn_dim must be a multiple of 64");
+  if (c->n_scales <= 0 || c->max_batch <= 0) return bad("n_scales / max_batch");
+  for (int k = 0; k < c->n_scales; ++k)
+    if (c->scale_hw[2 * k] <= 0 || c->scale_hw[2 * k + 1] <= 0) return bad("scale_hw");
+  if (c->has_cross_attn && (c->ctx_len <= 0 || c->ctx_width <= 0 || c->ctx_width % 64)) return bad("context shape");
+  if (!(c->ln_eps > 0.f)) return bad("ln_eps");
+  return true;
+}
+
+Layout make_layout(const fvar_cfg *c) {
+  Layout L;
+  const size_t B = c->max_batch, C = c->width, F = c->ffn_dim, nb = c->n_blocks, G = nb / c->blocks_per_group;
+  size_t Mmax = 0, Ltot = 0;
+  for (int k = 0; k < c->n_scales; ++k) {
+    const size_t m = static_cast<size_t>(c->scale_hw[2 * k]) * c->scale_hw[2 * k + 1];
+    Mmax = m > Mmax ? m : Mmax;
+    Ltot += m;
+  }
+  const size_t L_cap = align_up(Ltot, 128), ctx_cap = c->has_cross_attn ? align_up(c->ctx_len, 128) : 0;
+  const size_t Mp = align_up(Mmax, 8);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
+  L.status = take(256);
+  L.kc = take(nb * B * L_cap * C * 2);
+  L.vt = take(nb * B * L_cap * C * 2);
+  L.ckc = take(nb * B * ctx_cap * C * 2);
+  L.cvt = take(nb * B * ctx_cap * C * 2);
+  L.ada = take(nb * B * 6 * C * 4);
+  L.silu_c = take(align_up(B, 128) * C * 2);
+  L.gcache = take(2 * G * B * Mmax * C * 4);
+  L.x0 = take(B * Mmax * C * 4);
+  L.xs = take(B * Mmax * C * 4);
+  L.y = take(B * Mmax * C * 2);
+  L.q = take(B * Mmax * C * 2);
+  L.a = take(B * Mmax * C * 2);
+  L.hbuf = take(B * Mmax * F * 2);
+  L.xt = take(B * C * Mp * 2);
+  L.scores = take(B * Mmax * 4);
+  L.idx = take(G * B * Mmax * 4);
+  L.inv = take(G * B * Mmax * 4);
+  L.qt_pool = off;
+  size_t pool = 0;
+  L.qt_off.resize(static_cast<size_t>(c->n_scales) * G);
+  for (int k = 0; k < c->n_scales; ++k) {
+    const size_t m = static_cast<size_t>(c->scale_hw[2 * k]) * c->scale_hw[2 * k + 1];
+    for (size_t g = 0; g < G; ++g) {
+      L.qt_off[k * G + g] = pool;
+      pool += align_up(m * align_up(m, 8), 512);       // elements; r <= M rows of padded length
+    }
+  }
+  take(pool * 2);
+  L.total = off;
+  return L;
+}
+
+fvar_status fail(fvar_ctx *ctx, fvar_status s, const std::string &msg) {
+  if (ctx) ctx->err = msg; else g_init_error = msg;
+  return s;
+}
+
+fvar_status cuda_fail(fvar_ctx *ctx, cudaError_t e, const char *what) {
+  return fail(ctx, FVAR_ECUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+#define FV_CUDA(ctx, call, what)                                \
+  do {                                                          \
+    cudaError_t e__ = (call);                                   \
+    if (e__ != cudaSuccess) return cuda_fail(ctx, e__, what);   \
+  } while (0)
+
+// out = A W^T (+ epilogue) on the context's stream; picks the tile width from the problem size.
+fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
+  const int tiles_m = (g.R + 127) / 128 * g.nbatch;
+  const int bn = gemm_pick_block_n(tiles_m, g.N, ctx->num_sms);
+  g.status = ctx->status;
+  FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->st), what);
+  ctx->launches++;
+  return FVAR_OK;
+}
+
+GemmArgs gemm_args(int R, int N, int K) {
+  GemmArgs g;
+  memset(&g, 0, sizeof(g));
+  g.R = R; g.N = N; g.K = K;
+  g.nbatch = 1;
+  g.rows_per_batch = R > 0 ? R : 1;
+  g.bmul = 1;
+  g.rmap = RowMap{1, 0, R};
+  g.omap = RowMap{1, 0, R};
+  return g;
+}
+
+}  // namespace
+
+// ================================================================================================
+extern "C" {
+
+size_t fvar_workspace_bytes(const fvar_cfg *cfg) {
+  if (!shape_ok(cfg, nullptr)) return 0;
+  return make_layout(cfg).total;
+}
+
+fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *workspace, size_t bytes,
+                      void *cuda_stream, fvar_ctx **out) {
+  if (!out) return fail(nullptr, FVAR_EINVAL, "out is NULL");
+  *out = nullptr;
+  std::string why;
+  if (!shape_ok(cfg, &why)) return fail(nullptr, FVAR_EINVAL, "bad shape: " + why);
+  if (!weights || !workspace) return fail(nullptr, FVAR_EINVAL, "weights / workspace is NULL");
+  if (reinterpret_cast<uintptr_t>(workspace) & 1023) return fail(nullptr, FVAR_EINVAL, "workspace must be 1024-byte aligned");
+  const Layout L = make_layout(cfg);
+  if (bytes < L.total) return fail(nullptr, FVAR_ENOMEM, "workspace too small");
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
+    return fail(nullptr, FVAR_ECUDA, "no CUDA device");
+  if (prop.major != 10) return fail(nullptr, FVAR_ECUDA, "libfvar needs an sm_100 device (B200)");
+  if (!tmap_init_driver()) return fail(nullptr, FVAR_ECUDA, "cuTensorMapEncodeTiled is not available");
+
+  fvar_ctx *c = new fvar_ctx();
+  c->cfg = *cfg;
+  c->hw.assign(cfg->scale_hw, cfg->scale_hw + 2 * cfg->n_scales);
+  c->cfg.scale_hw = c->hw.data();
+  c->G = cfg->n_blocks / cfg->blocks_per_group;
+  c->C = cfg->width; c->F = cfg->ffn_dim; c->H = cfg->n_heads; c->D = cfg->head_dim; c->Bmax = cfg->max_batch;
+  c->Mmax = 0;
+  size_t Ltot = 0;
+  for (int k = 0; k < cfg->n_scales; ++k) {
+    const int m = c->hw[2 * k] * c->hw[2 * k + 1];
+    c->Mk.push_back(m);
+    c->Mmax = m > c->Mmax ? m : c->Mmax;
+    Ltot += m;
+  }
+  c->L_cap = static_cast<int>(align_up(Ltot, 128));
+  c->ctx_cap = cfg->has_cross_attn ? static_cast<int>(align_up(cfg->ctx_len, 128)) : 0;
+  c->num_sms = prop.multiProcessorCount;
+  c->st = static_cast<cudaStream_t>(cuda_stream);
+  c->launches = 0;
+  c->ws = static_cast<uint8_t *>(workspace);
+  c->ws_bytes = bytes;
+  auto at = [&](size_t off) { return c->ws + off; };
+  c->status = reinterpret_cast<unsigned *>(at(L.status));
+  c->kc = reinterpret_cast<bf16 *>(at(L.kc)); c->vt = reinterpret_cast<bf16 *>(at(L.vt));
+  c->ckc = reinterpret_cast<bf16 *>(at(L.ckc)); c->cvt = reinterpret_cast<bf16 *>(at(L.cvt));
+  c->ada = reinterpret_cast<float *>(at(L.ada)); c->silu_c = reinterpret_cast<bf16 *>(at(L.silu_c));
+  c->gcache = reinterpret_cast<float *>(at(L.gcache));
+  c->x0 = reinterpret_cast<float *>(at(L.x0)); c->xs = reinterpret_cast<float *>(at(L.xs));
+  c->y = reinterpret_cast<bf16 *>(at(L.y)); c->q = reinterpret_cast<bf16 *>(at(L.q));
+  c->a = reinterpret_cast<bf16 *>(at(L.a)); c->hbuf = reinterpret_cast<bf16 *>(at(L.hbuf));
+  c->xt = reinterpret_cast<bf16 *>(at(L.xt)); c->scores = reinterpret_cast<float *>(at(L.scores));
+  c->idx = reinterpret_cast<int *>(at(L.idx)); c->inv = reinterpret_cast<int *>(at(L.inv));
+  c->qt_pool = reinterpret_cast<bf16 *>(at(L.qt_pool));
+  c->qt_off = L.qt_off;
+  c->qt_r.assign(L.qt_off.size(), 0);
+  c->qt_map.resize(L.qt_off.size());
+
+  auto destroy_fail = [&](fvar_status s, const std::string &m) { delete c; return fail(nullptr, s, m); };
+
+  const int nb = cfg->n_blocks;
+  const void *const *srcs[W_COUNT] = {weights->w_qkv, weights->w_o, weights->w_fc1, weights->w_fc2,
+                                      weights->w_ada, weights->w_cq, weights->w_ckv, weights->w_co};
+  const int n_w = cfg->has_cross_attn ? W_COUNT : W_CQ;
+  for (int i = 0; i < n_w; ++i) {
+    if (!srcs[i]) return destroy_fail(FVAR_EINVAL, "a weight array is NULL");
+    for (int b = 0; b < nb; ++b) {
+      if (!srcs[i][b]) return destroy_fail(FVAR_EINVAL, "a weight pointer is NULL");
+      c->w[i].push_back(static_cast<const bf16 *>(srcs[i][b]));
+    }
+  }
+  const void *const *bsrc[6] = {weights->b_qkv, weights->b_o, weights->b_fc1, weights->b_fc2, weights->b_ada,
+                                weights->ln_c_gamma};
+  std::vector<const bf16 *> *bdst[6] = {&c->b_qkv, &c->b_o, &c->b_fc1, &c->b_fc2, &c->b_ada, &c->ln_c_gamma};
+  for (int i = 0; i < (cfg->has_cross_attn ? 6 : 5); ++i) {
+    if (!bsrc[i]) return destroy_fail(FVAR_EINVAL, "a bias array is NULL");
+    for (int b = 0; b < nb; ++b) {
+      if (!bsrc[i][b]) return destroy_fail(FVAR_EINVAL, "a bias pointer is NULL");
+      bdst[i]->push_back(static_cast<const bf16 *>(bsrc[i][b]));
+    }
+  }
+
+  // Tensor maps.  Weights: [out][in], one map per tile width.  Activations: full-capacity buffers.
+  const int C = c->C, F = c->F;
+  const int w_rows[W_COUNT] = {3 * C, C, F, C, 6 * C, C, 2 * C, C};
+  const int w_cols[W_COUNT] = {C, C, C, F, C, C, cfg->ctx_width, C};
+  c->wmap.resize(static_cast<size_t>(nb) * W_COUNT * 3);
+  bool ok = true;
+  for (int b = 0; b < nb && ok; ++b)
+    for (int i = 0; i < n_w && ok; ++i)
+      for (int t = 0; t < 3 && ok; ++t)
+        ok = tmap_2d(&c->wmap[(b * W_COUNT + i) * 3 + t], c->w[i][b], w_cols[i], w_rows[i], w_cols[i], kBNs[t]);
+  const size_t act_rows = static_cast<size_t>(c->Bmax) * c->Mmax;
+  ok = ok && tmap_2d(&c->y_map, c->y, C, act_rows, C, 128) && tmap_2d(&c->a_map, c->a, C, act_rows, C, 128) &&
+       tmap_2d(&c->q_map, c->q, C, act_rows, C, 128) && tmap_2d(&c->h_map, c->hbuf, F, act_rows, F, 128) &&
+       tmap_2d(&c->silu_map, c->silu_c, C, c->Bmax, C, 128);
+  c->xt_map.resize(static_cast<size_t>(cfg->n_scales) * 3);
+  for (int k = 0; k < cfg->n_scales && ok; ++k)
+    for (int t = 0; t < 3 && ok; ++t)
+      ok = tmap_2d(&c->xt_map[k * 3 + t], c->xt, c->Mk[k], static_cast<size_t>(c->Bmax) * C, align_up(c->Mk[k], 8),
+                   kBNs[t]);
+  c->kmap.resize(nb); c->vmap.resize(nb); c->ckmap.resize(nb); c->cvmap.resize(nb);
+  const int BH = c->Bmax * c->H, D = c->D;
+  for (int b = 0; b < nb && ok; ++b) {
+    ok = tmap_3d(&c->kmap[b], c->kc + b * c->kv_block_elems(), D, c->L_cap, BH, D, static_cast<uint64_t>(c->L_cap) * D, 64, 128) &&
+         tmap_3d(&c->vmap[b], c->vt + b * c->kv_block_elems(), c->L_cap, D, BH, c->L_cap, static_cast<uint64_t>(c->L_cap) * D, 64, D);
+    if (ok && cfg->has_cross_attn)
+      ok = tmap_3d(&c->ckmap[b], c->ckc + b * c->ckv_block_elems(), D, c->ctx_cap, BH, D, static_cast<uint64_t>(c->ctx_cap) * D, 64, 128) &&
+           tmap_3d(&c->cvmap[b], c->cvt + b * c->ckv_block_elems(), c->ctx_cap, D, BH, c->ctx_cap, static_cast<uint64_t>(c->ctx_cap) * D, 64, D);
+  }
+  if (!ok) return destroy_fail(FVAR_ECUDA, "tensor map encoding failed");
+
+  cudaError_t e = cudaMemsetAsync(c->ws, 0, L.total, c->st);
+  if (e != cudaSuccess) return destroy_fail(FVAR_ECUDA, std::string("workspace memset: ") + cudaGetErrorString(e));
+
+  c->B = 0;
+  c->len.assign(nb, 0);
+  c->staged.assign(nb, 0);
+  c->staged_scale = -1; c->last_scale = -1; c->cache_scale = -1; c->cache_slot = 0; c->null_only_seen = 0;
+  c->last_rank.assign(c->G, 0);
+  c->last_E = 0; c->last_M = 0;
+  *out = c;
+  return FVAR_OK;
+}
+
+fvar_status fvar_reset(fvar_ctx *ctx) {
+  if (!ctx) return FVAR_EINVAL;
+  std::fill(ctx->len.begin(), ctx->len.end(), 0);
+  std::fill(ctx->staged.begin(), ctx->staged.end(), 0);
+  ctx->staged_scale = -1; ctx->last_scale = -1; ctx->cache_scale = -1; ctx->null_only_seen = 0;
+  return FVAR_OK;
+}
+
+void fvar_destroy(fvar_ctx *ctx) { delete ctx; }
+
+const char *fvar_last_error(const fvar_ctx *ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+int fvar_cache_len(const fvar_ctx *ctx, int block) {
+  if (!ctx || block < 0 || block >= ctx->cfg.n_blocks) return -1;
+  return ctx->len[block];
+}
+
+long long fvar_launch_count(const fvar_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+fvar_status fvar_poll_status(fvar_ctx *ctx) {
+  unsigned word = 0;
+  if (ctx) {
+    FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+    FV_CUDA(ctx, cudaMemcpy(&word, ctx->status, sizeof(word), cudaMemcpyDeviceToHost), "status read");
+    if (word) FV_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof(word)), "status clear");
+  } else {
+    FV_CUDA(ctx, cudaDeviceSynchronize(), "device synchronize");
+    FV_CUDA(ctx, cudaMemcpyFromSymbol(&word, g_kernel_status, sizeof(word)), "status read");
+    if (word) {
+      const unsigned zero = 0;
+      FV_CUDA(ctx, cudaMemcpyToSymbol(g_kernel_status, &zero, sizeof(zero)), "status clear");
+    }
+  }
+  if (word & kStatusTimeout) return fail(ctx, FVAR_ETIMEOUT, "a device-side wait ran out");
+  if (word & kStatusBadIndex) return fail(ctx, FVAR_EINVAL, "forced_indices out of range or not ascending");
+  return FVAR_OK;
+}
+
+fvar_status fvar_set_cond(fvar_ctx *ctx, int B, const void *cond, const void *context) {
+  if (!ctx) return FVAR_EINVAL;
+  if (B <= 0 || B > ctx->Bmax || !cond) return fail(ctx, FVAR_EINVAL, "set_cond: bad batch or NULL cond");
+  if (ctx->cfg.has_cross_attn && !context) return fail(ctx, FVAR_EINVAL, "set_cond: context is NULL");
+  const int C = ctx->C, nb = ctx->cfg.n_blocks;
+  FV_CUDA(ctx, launch_silu_bf16(static_cast<const bf16 *>(cond), ctx->silu_c, static_cast<long long>(B) * C, ctx->st), "silu");
+  ctx->launches++;
+  for (int blk = 0; blk < nb; ++blk) {
+    GemmArgs g = gemm_args(B, 6 * C, C);
+    g.bias = ctx->b_ada[blk];
+    g.out_f32 = ctx->ada + static_cast<size_t>(blk) * ctx->Bmax * 6 * C;
+    g.ld_out = 6 * C;
+    fvar_status s = run_gemm(ctx, EPI_F32, ctx->silu_map, blk, W_ADA, g, "ada gemm");
+    if (s != FVAR_OK) return s;
+  }
+  if (ctx->cfg.has_cross_attn) {
+    CUtensorMap ctx_map;
+    const int T = ctx->cfg.ctx_len, Wc = ctx->cfg.ctx_width;
+    if (!tmap_2d(&ctx_map, context, Wc, static_cast<uint64_t>(B) * T, Wc, 128))
+      return fail(ctx, FVAR_EINVAL, "set_cond: context must be 16-byte aligned");
+    for (int blk = 0; blk < nb; ++blk) {
+      GemmArgs g = gemm_args(B * T, 2 * C, Wc);
+      g.rows_per_batch = T;
+      g.kc = ctx->ckc + blk * ctx->ckv_block_elems();
+      g.vt = ctx->cvt + blk * ctx->ckv_block_elems();
+      g.C = C; g.H = ctx->H; g.D = ctx->D; g.L_cap = ctx->ctx_cap; g.L_prev = 0; g.col_base = C;
+      g.out_bf16 = ctx->q; g.ld_out = C;           // unused: no column maps to the q part
+      fvar_status s = run_gemm(ctx, EPI_QKV, ctx_map, blk, W_CKV, g, "context kv gemm");
+      if (s != FVAR_OK) return s;
+    }
+  }
+  ctx->B = B;
+  return fvar_reset(ctx);
+}
+
+fvar_status fvar_set_projection(fvar_ctx *ctx, int scale_idx, int group, const void *Qt, int r) {
+  if (!ctx) return FVAR_EINVAL;
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || group < 0 || group >= ctx->G || !Qt)
+    return fail(ctx, FVAR_EINVAL, "set_projection: bad scale / group / pointer");
+  const int M = ctx->Mk[scale_idx];
+  if (r <= 0 || r > M) return fail(ctx, FVAR_EINVAL, "set_projection: need 0 < r <= M");
+  const size_t Mp = align_up(M, 8), slot = static_cast<size_t>(scale_idx) * ctx->G + group;
+  bf16 *dst = ctx->qt_pool + ctx->qt_off[slot];
+  FV_CUDA(ctx, cudaMemcpy2DAsync(dst, Mp * 2, Qt, static_cast<size_t>(M) * 2, static_cast<size_t>(M) * 2, r,
+                                 cudaMemcpyDeviceToDevice, ctx->st), "projection copy");
+  if (!tmap_2d(&ctx->qt_map[slot], dst, M, r, Mp, 128)) return fail(ctx, FVAR_ECUDA, "projection tensor map");
+  ctx->qt_r[slot] = r;
+  return FVAR_OK;
+}
+
+fvar_status fvar_load_kv(fvar_ctx *ctx, const void *K, const void *V, int L) {
+  if (!ctx) return FVAR_EINVAL;
+  if (ctx->B <= 0) return fail(ctx, FVAR_ESTATE, "load_kv before set_cond");
+  if (!K || !V || L < 0 || L > ctx->L_cap) return fail(ctx, FVAR_EINVAL, "load_kv: bad arguments");
+  const size_t per_blk = static_cast<size_t>(ctx->B) * L * ctx->C;
+  for (int blk = 0; blk < ctx->cfg.n_blocks; ++blk) {
+    FV_CUDA(ctx, launch_load_kv(static_cast<const bf16 *>(K) + blk * per_blk, static_cast<const bf16 *>(V) + blk * per_blk,
+                                ctx->B, L, ctx->H, ctx->D, ctx->L_cap, ctx->kc + blk * ctx->kv_block_elems(),
+                                ctx->vt + blk * ctx->kv_block_elems(), ctx->st), "load_kv");
+    ctx->launches++;
+    ctx->len[blk] = L;
+  }
+  ctx->staged_scale = -1;
+  return FVAR_OK;
+}
+
+fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cache) {
+  if (!ctx) return FVAR_EINVAL;
+  if (ctx->B <= 0) return fail(ctx, FVAR_ESTATE, "load_group_cache before set_cond");
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || !cache) return fail(ctx, FVAR_EINVAL, "load_group_cache: bad arguments");
+  const int M = ctx->Mk[scale_idx];
+  const size_t per = static_cast<size_t>(ctx->B) * M * ctx->C;
+  for (int g = 0; g < ctx->G; ++g)
+    FV_CUDA(ctx, cudaMemcpyAsync(ctx->gslot(0, g), cache + g * per, per * 4, cudaMemcpyDeviceToDevice, ctx->st), "group cache copy");
+  ctx->cache_scale = scale_idx;
+  ctx->cache_slot = 0;
+  if (ctx->last_scale < scale_idx) ctx->last_scale = scale_idx;
+  return FVAR_OK;
+}
+
+fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, const fvar_keep_policy *pol, void *out) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!pol) return fail(ctx, FVAR_EINVAL, "scale_step: policy is NULL");
+  if (pol->mode == FVAR_SKIP) return FVAR_OK;
+  if (pol->mode != FVAR_DENSE && pol->mode != FVAR_LOWRANK_RTR) return fail(ctx, FVAR_EINVAL, "scale_step: bad mode");
+  if (pol->cfg_mode != FVAR_CFG_PAIR && pol->cfg_mode != FVAR_CFG_NULL_ONLY) return fail(ctx, FVAR_EINVAL, "scale_step: bad cfg_mode");
+  if (!tokens || !out) return fail(ctx, FVAR_EINVAL, "scale_step: NULL tokens / out");
+  if (ctx->B <= 0) return fail(ctx, FVAR_ESTATE, "scale_step before set_cond");
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales) return fail(ctx, FVAR_EINVAL, "scale_step: bad scale_idx");
+  if (scale_idx < ctx->last_scale) return fail(ctx, FVAR_ESTATE, "scale_step: scale_idx decreased");
+  const bool null_only = pol->cfg_mode == FVAR_CFG_NULL_ONLY;
+  if (null_only && (ctx->B % 2)) return fail(ctx, FVAR_EINVAL, "scale_step: null-only needs an even batch");
+  if (!null_only && ctx->null_only_seen) return fail(ctx, FVAR_ESTATE, "scale_step: pair step after a null-only step");
+
+  const int C = ctx->C, F = ctx->F, H = ctx->H, D = ctx->D, G = ctx->G, bpg = ctx->cfg.blocks_per_group;
+  const int M = ctx->Mk[scale_idx], B = ctx->B;
+  const int E = null_only ? B / 2 : B, bmul = null_only ? 2 : 1, boff = null_only ? 1 : 0;
+  std::vector<int> rank(G, M);
+  if (pol->mode == FVAR_LOWRANK_RTR) {
+    for (int g = 0; g < G; ++g) {
+      int r = pol->rank_per_group ? pol->rank_per_group[g] : static_cast<int>(floorf(pol->keep_ratio * M + 0.5f));
+      if (!pol->rank_per_group) r = r < 1 ? 1 : (r > M ? M : r);
+      if (r < 1 || r > M) return fail(ctx, FVAR_EINVAL, "scale_step: need 1 <= r <= M");
+      rank[g] = r;
+    }
+  }
+  int r_max = 0;
+  bool any_late = false;
+  for (int g = 0; g < G; ++g) {
+    if (rank[g] < M) {
+      any_late = true;
+      r_max = rank[g] > r_max ? rank[g] : r_max;
+      if (ctx->qt_r[static_cast<size_t>(scale_idx) * G + g] != rank[g])
+        return fail(ctx, FVAR_ESTATE, "scale_step: no projection of this rank set for a group");
+    }
+    for (int blk = g * bpg; blk < (g + 1) * bpg; ++blk)
+      if (ctx->len[blk] + rank[g] > ctx->L_cap) return fail(ctx, FVAR_ESTATE, "scale_step: KV cache is full");
+  }
+  if (any_late && (ctx->cache_scale < 0 || ctx->cache_scale > scale_idx))
+    return fail(ctx, FVAR_ESTATE, "scale_step: low-rank step without the previous scale's group outputs");
+
+  const int prev_slot = ctx->cache_slot, cur_slot = ctx->cache_scale < 0 ? 0 : (ctx->cache_slot ^ 1);
+  const int h0 = ctx->cache_scale >= 0 ? ctx->hw[2 * ctx->cache_scale] : 0;
+  const int w0 = ctx->cache_scale >= 0 ? ctx->hw[2 * ctx->cache_scale + 1] : 0;
+  const int h1 = ctx->hw[2 * scale_idx], w1 = ctx->hw[2 * scale_idx + 1];
+  const float scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(D));
+  const size_t ada_blk = static_cast<size_t>(ctx->Bmax) * 6 * C;
+  cudaStream_t st = ctx->st;
+
+  FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, B, static_cast<long long>(M) * C, st), "tokens_to_f32");
+  ctx->launches++;
+  const float *X_in = ctx->x0;
+  const RowMap bmap{bmul, boff, M};              // buffers indexed by the caller's batch element
+  fvar_status s;
+
+  for (int g = 0; g < G; ++g) {
+    const int r = rank[g];
+    const bool late = r < M;
+    const int R = E * r;
+    float *gout = ctx->gslot(cur_slot, g);
+    int *idx_g = ctx->idx + static_cast<size_t>(g) * ctx->Bmax * ctx->Mmax;
+    int *inv_g = ctx->inv + static_cast<size_t>(g) * ctx->Bmax * ctx->Mmax;
+    const RowMap smap{1, 0, r};                  // the compact work stream of this group
+
+    if (late) {
+      if (pol->forced_indices) {
+        FV_CUDA(ctx, launch_copy_indices(pol->forced_indices + static_cast<size_t>(g) * E * r_max, E, M, r, r_max, idx_g,
+                                         inv_g, ctx->status, st), "copy_indices");
+        ctx->launches++;
+      } else {
+        if (null_only) {
+          for (int e = 0; e < E; ++e) {
+            FV_CUDA(ctx, launch_row_scores(X_in + static_cast<size_t>(e * bmul + boff) * M * C, M, C,
+                                           ctx->scores + static_cast<size_t>(e) * M, st), "row_scores");
+            ctx->launches++;
+          }
+        } else {
+          FV_CUDA(ctx, launch_row_scores(X_in, static_cast<long long>(E) * M, C, ctx->scores, st), "row_scores");
+          ctx->launches++;
+        }
+        FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, st), "select_topr");
+        ctx->launches++;
+      }
+      const int Mp = static_cast<int>(align_up(M, 8));
+      FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mp, ctx->xt, st), "transpose");
+      ctx->launches++;
+      // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e
+      GemmArgs ga = gemm_args(r, C, M);
+      ga.nbatch = E;
+      ga.a_batch_rows = 0;
+      ga.b_batch_rows = C;
+      ga.out_f32 = ctx->xs;
+      ga.ld_out = C;
+      ga.status = ctx->status;
+      const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, ctx->num_sms);
+      FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
+                               ctx->xt_map[scale_idx * 3 + bn_index(bn)], ga, ctx->num_sms, st), "projection gemm");
+      ctx->launches++;
+    }
+
+    for (int t = 0; t < bpg; ++t) {
+      const int blk = g * bpg + t;
+      const bool first_dense = (t == 0) && !late, last = (t == bpg - 1);
+      const float *in_ptr = first_dense ? X_in : ctx->xs;
+      const RowMap in_map = first_dense ? bmap : smap;
+      const float *ada = ctx->ada + blk * ada_blk;
+      const int L_prev = ctx->len[blk];
+
+      FV_CUDA(ctx, launch_ln_modulate(in_ptr, in_map, E, r, C, ada, ada + C, 6 * C, bmul, boff, nullptr,
+                                      ctx->cfg.ln_eps, ctx->y, st), "ln_modulate 1");
+      ctx->launches++;
+      {
+        GemmArgs ga = gemm_args(R, 3 * C, C);
+        ga.bias = ctx->b_qkv[blk];
+        ga.rows_per_batch = r; ga.bmul = bmul; ga.boff = boff;
+        ga.out_bf16 = ctx->q; ga.ld_out = C;
+        ga.kc = ctx->kc + blk * ctx->kv_block_elems();
+        ga.vt = ctx->vt + blk * ctx->kv_block_elems();
+        ga.C = C; ga.H = H; ga.D = D; ga.L_cap = ctx->L_cap; ga.L_prev = L_prev; ga.col_base = 0;
+        if ((s = run_gemm(ctx, EPI_QKV, ctx->y_map, blk, W_QKV, ga, "qkv gemm")) != FVAR_OK) return s;
+      }
+      {
+        AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
+        ctx->launches++;
+      }
+      {
+        GemmArgs ga = gemm_args(R, C, C);
+        ga.bias = ctx->b_o[blk];
+        ga.rows_per_batch = r; ga.bmul = bmul; ga.boff = boff;
+        ga.resid = in_ptr; ga.rmap = in_map;
+        ga.out_f32 = ctx->xs; ga.omap = smap; ga.ld_out = C;
+        ga.gate = ada + 2 * C; ga.gate_stride = 6 * C;
+        if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_O, ga, "out-proj gemm")) != FVAR_OK) return s;
+      }
+      if (ctx->cfg.has_cross_attn) {
+        FV_CUDA(ctx, launch_ln_modulate(ctx->xs, smap, E, r, C, nullptr, nullptr, 0, bmul, boff, ctx->ln_c_gamma[blk],
+                                        ctx->cfg.ln_eps, ctx->y, st), "ln cross");
+        ctx->launches++;
+        GemmArgs gq = gemm_args(R, C, C);
+        gq.out_bf16 = ctx->q; gq.ld_out = C;
+        if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
+        AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
+        ctx->launches++;
+        GemmArgs go = gemm_args(R, C, C);
+        go.rows_per_batch = r; go.bmul = bmul; go.boff = boff;
+        go.resid = ctx->xs; go.rmap = smap; go.out_f32 = ctx->xs; go.omap = smap; go.ld_out = C;
+        if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_CO, go, "cross out gemm")) != FVAR_OK) return s;
+      }
+      FV_CUDA(ctx, launch_ln_modulate(ctx->xs, smap, E, r, C, ada + 3 * C, ada + 4 * C, 6 * C, bmul, boff, nullptr,
+                                      ctx->cfg.ln_eps, ctx->y, st), "ln_modulate 2");
+      ctx->launches++;
+      {
+        GemmArgs ga = gemm_args(R, F, C);
+        ga.bias = ctx->b_fc1[blk];
+        ga.out_bf16 = ctx->hbuf; ga.ld_out = F;
+        if ((s = run_gemm(ctx, EPI_GELU_BF16, ctx->y_map, blk, W_FC1, ga, "fc1 gemm")) != FVAR_OK) return s;
+      }
+      {
+        GemmArgs ga = gemm_args(R, C, F);
+        ga.bias = ctx->b_fc2[blk];
+        ga.rows_per_batch = r; ga.bmul = bmul; ga.boff = boff;
+        ga.resid = ctx->xs; ga.rmap = smap; ga.ld_out = C;
+        ga.gate = ada + 5 * C; ga.gate_stride = 6 * C;
+        if (last) {
+          ga.out_f32 = gout; ga.omap = bmap;
+          ga.scatter = late ? idx_g : nullptr;
+        } else {
+          ga.out_f32 = ctx->xs; ga.omap = smap;
+        }
+        if ((s = run_gemm(ctx, EPI_RESID, ctx->h_map, blk, W_FC2, ga, "fc2 gemm")) != FVAR_OK) return s;
+      }
+      ctx->staged[blk] = r;
+    }
+    if (late) {
+      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, st), "rtr_fill");
+      ctx->launches++;
+    }
+    X_in = gout;
+    ctx->last_rank[g] = r;
+  }
+  FV_CUDA(ctx, launch_out_to_bf16(X_in, bmap, E, M, C, static_cast<bf16 *>(out), st), "out_to_bf16");
+  ctx->launches++;
+
+  ctx->cache_scale = scale_idx;
+  ctx->cache_slot = cur_slot;
+  ctx->staged_scale = scale_idx;
+  ctx->last_scale = scale_idx;
+  ctx->last_E = E; ctx->last_M = M;
+  if (null_only) ctx->null_only_seen = 1;
+  return FVAR_OK;
+}
+
+fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int scale_idx, const fvar_keep_policy *pol,
+                                 void *out_host) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!pol) return fail(ctx, FVAR_EINVAL, "scale_step_host: policy is NULL");
+  if (pol->mode == FVAR_SKIP) return FVAR_OK;
+  if (!tokens_host || !out_host) return fail(ctx, FVAR_EINVAL, "scale_step_host: NULL tokens / out");
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || ctx->B <= 0) return fail(ctx, FVAR_EINVAL, "scale_step_host: bad scale_idx or no cond");
+  // Staging: the bf16 tokens land in the hidden-activation buffer (free until the first fc1) and
+  // the bf16 output in the attention-output buffer (free after the last out-proj).
+  const size_t M = ctx->Mk[scale_idx], in_bytes = static_cast<size_t>(ctx->B) * M * ctx->C * 2;
+  const int E = pol->cfg_mode == FVAR_CFG_NULL_ONLY ? ctx->B / 2 : ctx->B;
+  FV_CUDA(ctx, cudaMemcpyAsync(ctx->hbuf, tokens_host, in_bytes, cudaMemcpyHostToDevice, ctx->st), "tokens H2D");
+  fvar_status s = fvar_scale_step(ctx, ctx->hbuf, scale_idx, pol, ctx->a);
+  if (s != FVAR_OK) return s;
+  FV_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->a, static_cast<size_t>(E) * M * ctx->C * 2, cudaMemcpyDeviceToHost, ctx->st), "out D2H");
+  FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  return FVAR_OK;
+}
+
+fvar_status fvar_kv_append(fvar_ctx *ctx, int scale_idx) {
+  if (!ctx) return FVAR_EINVAL;
+  if (ctx->staged_scale < 0 || ctx->staged_scale != scale_idx) return fail(ctx, FVAR_ESTATE, "kv_append: nothing staged for this scale");
+  for (int blk = 0; blk < ctx->cfg.n_blocks; ++blk) {
+    ctx->len[blk] += ctx->staged[blk];
+    ctx->staged[blk] = 0;
+  }
+  ctx->staged_scale = -1;
+  return FVAR_OK;
+}
+
+fvar_status fvar_get_indices(fvar_ctx *ctx, int group, int *idx_dev, int *count_host) {
+  if (!ctx) return FVAR_EINVAL;
+  if (group < 0 || group >= ctx->G || !idx_dev || !count_host) return fail(ctx, FVAR_EINVAL, "get_indices: bad arguments");
+  if (ctx->last_scale < 0 || ctx->last_rank[group] <= 0 || ctx->last_rank[group] >= ctx->last_M)
+    return fail(ctx, FVAR_ESTATE, "get_indices: the last step did not select rows for this group");
+  const int r = ctx->last_rank[group];
+  FV_CUDA(ctx, cudaMemcpyAsync(idx_dev, ctx->idx + static_cast<size_t>(group) * ctx->Bmax * ctx->Mmax,
+                               static_cast<size_t>(ctx->last_E) * r * 4, cudaMemcpyDeviceToDevice, ctx->st), "indices copy");
+  *count_host = r;
+  return FVAR_OK;
+}
+
+fvar_status fvar_get_group_output(fvar_ctx *ctx, int group, float *out_dev) {
+  if (!ctx) return FVAR_EINVAL;
+  if (group < 0 || group >= ctx->G || !out_dev) return fail(ctx, FVAR_EINVAL, "get_group_output: bad arguments");
+  if (ctx->cache_scale < 0) return fail(ctx, FVAR_ESTATE, "get_group_output: no scale stepped yet");
+  const size_t n = static_cast<size_t>(ctx->B) * ctx->Mk[ctx->cache_scale] * ctx->C;
+  FV_CUDA(ctx, cudaMemcpyAsync(out_dev, ctx->gslot(ctx->cache_slot, group), n * 4, cudaMemcpyDeviceToDevice, ctx->st), "group output copy");
+  return FVAR_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ kernel-level
+static unsigned *kernel_status_ptr() {
+  static unsigned *p = nullptr;
+  if (!p) {
+    void *addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_kernel_status) != cudaSuccess) return nullptr;
+    p = static_cast<unsigned *>(addr);
+  }
+  return p;
+}
+
+static fvar_status kfail(fvar_status s, const char *m) { g_init_error = m; return s; }
+#define FK_CUDA(call, what)                                                                          \
+  do {                                                                                               \
+    cudaError_t e__ = (call);                                                                        \
+    if (e__ != cudaSuccess) return kfail(FVAR_ECUDA, (std::string(what) + ": " + cudaGetErrorString(e__)).c_str()); \
+  } while (0)
+
+fvar_status fvar_row_scores(const float *x, int B, int M, int C, float *scores, void *stream) {
+  if (!x || !scores || B <= 0 || M <= 0 || C <= 0 || C % 4) return kfail(FVAR_EINVAL, "row_scores: bad arguments");
+  FK_CUDA(launch_row_scores(x, static_cast<long long>(B) * M, C, scores, static_cast<cudaStream_t>(stream)), "row_scores");
+  return FVAR_OK;
+}
+
+fvar_status fvar_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, void *stream) {
+  if (!scores || !idx || !inv || B <= 0 || M <= 0 || r <= 0 || r > M) return kfail(FVAR_EINVAL, "select_topr: bad arguments");
+  FK_CUDA(launch_select_topr(scores, B, M, r, idx, inv, static_cast<cudaStream_t>(stream)), "select_topr");
+  return FVAR_OK;
+}
+
+fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, const float *shift, const float *scale,
+                             long long vec_stride, float eps, void *y, void *stream) {
+  if (!x || !y || !shift || !scale || R <= 0 || C <= 0 || C % 8 || C > 8192 || rows_per_batch <= 0 || R % rows_per_batch)
+    return kfail(FVAR_EINVAL, "ln_modulate: bad arguments");
+  FK_CUDA(launch_ln_modulate(x, RowMap{1, 0, rows_per_batch}, R / rows_per_batch, rows_per_batch, C, shift, scale,
+                             vec_stride, 1, 0, nullptr, eps, static_cast<bf16 *>(y), static_cast<cudaStream_t>(stream)),
+          "ln_modulate");
+  return FVAR_OK;
+}
+
+fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out, void *stream) {
+  if (!A || !W || !out || R <= 0 || N <= 0 || K <= 0 || K % 8) return kfail(FVAR_EINVAL, "gemm: bad arguments");
+  int dev = 0, sms = 0;
+  FK_CUDA(cudaGetDevice(&dev), "get device");
+  FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
+  const int bn = gemm_pick_block_n((R + 127) / 128, N, sms);
+  CUtensorMap ta, tw;
+  if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, W, K, N, K, bn)) return kfail(FVAR_EINVAL, "gemm: operands must be 16-byte aligned");
+  GemmArgs g = gemm_args(R, N, K);
+  g.bias = static_cast<const bf16 *>(bias);
+  g.out_f32 = out;
+  g.ld_out = N;
+  g.status = kernel_status_ptr();
+  if (!g.status) return kfail(FVAR_ECUDA, "gemm: status word");
+  FK_CUDA(launch_gemm(EPI_F32, bn, ta, tw, g, sms, static_cast<cudaStream_t>(stream)), "gemm");
+  return FVAR_OK;
+}
+
+fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B, int H, int r, int D, int L, int L_cap,
+                           void *out, void *stream) {
+  if (!q || !Kc || !Vt || !out || B <= 0 || H <= 0 || r <= 0 || (D != 64 && D != 128) || L <= 0 || L > L_cap || L_cap % 8)
+    return kfail(FVAR_EINVAL, "attention: bad arguments");
+  CUtensorMap tq, tk, tv;
+  const uint64_t BH = static_cast<uint64_t>(B) * H;
+  if (!tmap_2d(&tq, q, static_cast<uint64_t>(H) * D, static_cast<uint64_t>(B) * r, static_cast<uint64_t>(H) * D, 128) ||
+      !tmap_3d(&tk, Kc, D, L_cap, BH, D, static_cast<uint64_t>(L_cap) * D, 64, 128) ||
+      !tmap_3d(&tv, Vt, L_cap, D, BH, L_cap, static_cast<uint64_t>(L_cap) * D, 64, D))
+    return kfail(FVAR_EINVAL, "attention: operands must be 16-byte aligned");
+  AttnArgs a{B, H, r, D, L, L_cap, 1, 0, static_cast<bf16 *>(out), 1.4426950408889634f / sqrtf(static_cast<float>(D)),
+             kernel_status_ptr()};
+  if (!a.status) return kfail(FVAR_ECUDA, "attention: status word");
+  FK_CUDA(launch_attention(tq, tk, tv, a, static_cast<cudaStream_t>(stream)), "attention");
+  return FVAR_OK;
+}
+
+fvar_status fvar_rtr_fill(const float *prev, int B, int h0, int w0, int h1, int w1, int C, const int *inv, float *out,
+                          void *stream) {
+  if (!prev || !out || B <= 0 || h0 <= 0 || w0 <= 0 || h1 <= 0 || w1 <= 0 || C <= 0 || C % 4)
+    return kfail(FVAR_EINVAL, "rtr_fill: bad arguments");
+  FK_CUDA(launch_rtr_fill(prev, out, B, 1, 0, h0, w0, h1, w1, C, inv, static_cast<cudaStream_t>(stream)), "rtr_fill");
+  return FVAR_OK;
+}
+
+}  // extern "C"

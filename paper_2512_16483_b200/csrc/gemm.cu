@@ -1,0 +1,339 @@
+// Tensor-core GEMM for sm_100a: out[R][N] = A[R][K] * W[N][K]^T with fused epilogues.
+//
+// One persistent CTA per SM walks the tile list.  Warp 0 feeds a ring of shared-memory stages
+// with TMA (128-byte swizzle), warp 1 issues tcgen05.mma into one of two TMEM accumulators,
+// warps 2-5 drain the other accumulator (tcgen05.ld) and apply the epilogue, so the epilogue of
+// tile i overlaps the main loop of tile i+1.  Every wait is bounded; on expiry the CTA flags the
+// status word, lets its outstanding copies land, frees its TMEM and returns.
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace fvar {
+
+constexpr int kBlockM = 128;
+constexpr int kBlockK = 64;             // 64 bf16 = one 128-byte swizzle row
+constexpr int kGemmThreads = 192;
+constexpr int kSmemBudget = 196608;     // bytes of operand stages per CTA (192 KiB)
+
+template <int BN>
+struct GemmCfg {
+  static constexpr int kStageBytesA = kBlockM * kBlockK * 2;
+  static constexpr int kStageBytesB = BN * kBlockK * 2;
+  static constexpr int kStageBytes = kStageBytesA + kStageBytesB;
+  static constexpr int kStages = kSmemBudget / kStageBytes;
+  static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;     // two accumulators
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+  static_assert(kStages >= 3 && kStages <= 12, "stage count");
+  static_assert((kTmemCols & (kTmemCols - 1)) == 0 && kTmemCols <= 512, "TMEM columns");
+  // More than half of an SM's shared memory per CTA: at most one CTA per SM, so the TMEM
+  // allocation (up to all 512 columns) can never wait on a co-resident CTA.
+  static_assert(kSmemBytes > 116 * 1024, "one CTA per SM");
+};
+
+__device__ __forceinline__ float gelu_tanh_f(float x) {
+  const float k0 = 0.7978845608028654f, k1 = 0.044715f;
+  float u = k0 * (x + k1 * x * x * x);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return 0.5f * x * (1.0f + t);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Epilogue for one thread: one output row, 32 consecutive columns starting at col0 (col0 % 32 == 0).
+template <int EPI>
+__device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t (&acc)[32], int batch, int row,
+                                               int col0) {
+  float v[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
+  const bool full = (col0 + 32 <= p.N);
+  if (p.bias != nullptr) {
+    if (full) {
+      const uint4 *bp = reinterpret_cast<const uint4 *>(p.bias + col0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 u = __ldg(bp + q);
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          float2 f = __bfloat1622float2(h[t]);
+          v[q * 8 + t * 2] += f.x;
+          v[q * 8 + t * 2 + 1] += f.y;
+        }
+      }
+    } else {
+      for (int i = 0; i < 32; ++i)
+        if (col0 + i < p.N) v[i] += __bfloat162float(p.bias[col0 + i]);
+    }
+  }
+  const long long grow = static_cast<long long>(batch) * p.R + row;   // row in the flattened output
+
+  if constexpr (EPI == EPI_F32) {
+    float *dst = p.out_f32 + grow * p.ld_out + col0;
+    if (full && (p.ld_out & 3) == 0) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        reinterpret_cast<float4 *>(dst)[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+    } else {
+      for (int i = 0; i < 32; ++i)
+        if (col0 + i < p.N) dst[i] = v[i];
+    }
+  } else if constexpr (EPI == EPI_BF16 || EPI == EPI_GELU_BF16) {
+    if constexpr (EPI == EPI_GELU_BF16) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_f(v[i]);
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(p.out_bf16 + grow * p.ld_out + col0);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      dst[q] = make_uint4(pack_bf16(v[q * 8], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+                          pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+  } else if constexpr (EPI == EPI_QKV) {
+    const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
+    const int b = e * p.bmul + p.boff;
+    const int vc = col0 + p.col_base;
+    if (vc < p.C) {
+      uint4 *dst = reinterpret_cast<uint4 *>(p.out_bf16 + static_cast<long long>(row) * p.ld_out + vc);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        dst[q] = make_uint4(pack_bf16(v[q * 8], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+                            pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+    } else if (vc < 2 * p.C) {
+      const int c = vc - p.C, h = c / p.D, d0 = c - h * p.D;
+      bf16 *base = p.kc + ((static_cast<long long>(b) * p.H + h) * p.L_cap + p.L_prev + j) * p.D + d0;
+      uint4 *dst = reinterpret_cast<uint4 *>(base);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        dst[q] = make_uint4(pack_bf16(v[q * 8], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+                            pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+    } else {
+      const int c = vc - 2 * p.C, h = c / p.D, d0 = c - h * p.D;
+      bf16 *base = p.vt + ((static_cast<long long>(b) * p.H + h) * p.D + d0) * p.L_cap + p.L_prev + j;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) base[static_cast<long long>(i) * p.L_cap] = __float2bfloat16_rn(v[i]);
+    }
+  } else {  // EPI_RESID
+    const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
+    const int b = e * p.bmul + p.boff;
+    const float *res = p.resid + (static_cast<long long>(e * p.rmap.bmul + p.rmap.boff) * p.rmap.rpb + j) * p.ld_out + col0;
+    const int jo = p.scatter ? __ldg(p.scatter + static_cast<long long>(e) * p.rows_per_batch + j) : j;
+    float *dst = p.out_f32 + (static_cast<long long>(e * p.omap.bmul + p.omap.boff) * p.omap.rpb + jo) * p.ld_out + col0;
+    const float *g = p.gate ? p.gate + static_cast<long long>(b) * p.gate_stride + col0 : nullptr;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      float4 r4 = reinterpret_cast<const float4 *>(res)[q];
+      float4 g4 = g ? __ldg(reinterpret_cast<const float4 *>(g) + q) : make_float4(1.f, 1.f, 1.f, 1.f);
+      float4 o;
+      o.x = fmaf(g4.x, v[q * 4], r4.x);
+      o.y = fmaf(g4.y, v[q * 4 + 1], r4.y);
+      o.z = fmaf(g4.z, v[q * 4 + 2], r4.z);
+      o.w = fmaf(g4.w, v[q * 4 + 3], r4.w);
+      reinterpret_cast<float4 *>(dst)[q] = o;
+    }
+  }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+            const __grid_constant__ GemmArgs p) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int S = Cfg::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ volatile int abort_flag;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + S * Cfg::kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * S + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (p.R + kBlockM - 1) / kBlockM;
+  const int tiles_n = (p.N + BN - 1) / BN;
+  const int tiles_per_batch = tiles_m * tiles_n;
+  const int total_tiles = tiles_per_batch * p.nbatch;
+  const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 128);
+    }
+    mbar_fence_init();
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmW);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_holder), Cfg::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0;                      // bit s set: stage s has been armed at least once
+      uint32_t last_parity = 0;                // bit s: parity of the phase last armed on stage s
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+        const int e = tile / tiles_per_batch, rem = tile - e * tiles_per_batch;
+        const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
+        const int row_a = e * p.a_batch_rows + m_idx * kBlockM;
+        const int row_w = e * p.b_batch_rows + n_idx * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(stage), Cfg::kStageBytes);
+          const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+          tma_load_2d(sa, &tmA, full_bar(stage), kb * kBlockK, row_a);
+          tma_load_2d(sa + Cfg::kStageBytesA, &tmW, full_bar(stage), kb * kBlockK, row_w);
+          armed |= 1u << stage;
+          last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Let every copy that was issued land before the CTA's shared memory is released.
+        for (int s = 0; s < S; ++s)
+          if (armed & (1u << s)) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(full_bar(s), (last_parity >> s) & 1u) && clock64() - t0 < kWaitCycles) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      constexpr uint32_t idesc = umma_idesc_bf16(kBlockM, BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+        const int a = it & 1;
+        const uint32_t aphase = (it >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + a * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, p.status, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + Cfg::kStageBytesA);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)
+            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+          umma_commit(empty_bar(stage));
+          if (++stage == S) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(a));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quad = warp & 3;                 // TMEM lanes [32 * quad, 32 * quad + 32)
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+      const int e = tile / tiles_per_batch, rem = tile - e * tiles_per_batch;
+      const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
+      const int a = it & 1;
+      const uint32_t aphase = (it >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m_idx * kBlockM + quad * 32 + lane;
+      const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = n_idx * BN + c * 32;
+        if (col0 >= p.N) break;                // uniform across the warp
+        uint32_t acc[32];
+        tmem_ld32(taddr + c * 32, acc);
+        tmem_ld_wait();
+        if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0);
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(a));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  }
+}
+
+int gemm_pick_block_n(int tiles_m_total, int N, int num_sms) {
+  // Largest tile whose tile count still fills the machine; small problems take narrow tiles so
+  // that more SMs stream the weight matrix.
+  const int cand[3] = {256, 128, 64};
+  for (int i = 0; i < 3; ++i) {
+    const int bn = cand[i];
+    if (N % bn != 0 && i < 2) continue;
+    const long long tiles = static_cast<long long>(tiles_m_total) * ((N + bn - 1) / bn);
+    if (tiles >= 2ll * num_sms || i == 2) return bn;
+  }
+  return 64;
+}
+
+template <int BN, int EPI>
+static cudaError_t launch_one(const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, int num_sms,
+                              cudaStream_t st) {
+  using Cfg = GemmCfg<BN>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t err = cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           Cfg::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    attr_set = true;
+  }
+  const long long tiles = static_cast<long long>((a.R + kBlockM - 1) / kBlockM) * ((a.N + BN - 1) / BN) * a.nbatch;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
+  gemm_kernel<BN, EPI><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, a);
+  return cudaGetLastError();
+}
+
+template <int BN>
+static cudaError_t launch_bn(int epi, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, int num_sms,
+                             cudaStream_t st) {
+  switch (epi) {
+    case EPI_F32: return launch_one<BN, EPI_F32>(tmA, tmW, a, num_sms, st);
+    case EPI_BF16: return launch_one<BN, EPI_BF16>(tmA, tmW, a, num_sms, st);
+    case EPI_GELU_BF16: return launch_one<BN, EPI_GELU_BF16>(tmA, tmW, a, num_sms, st);
+    case EPI_QKV: return launch_one<BN, EPI_QKV>(tmA, tmW, a, num_sms, st);
+    case EPI_RESID: return launch_one<BN, EPI_RESID>(tmA, tmW, a, num_sms, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_gemm(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
+                        int num_sms, cudaStream_t st) {
+  switch (block_n) {
+    case 64: return launch_bn<64>(epi, tmA, tmW, a, num_sms, st);
+    case 128: return launch_bn<128>(epi, tmA, tmW, a, num_sms, st);
+    case 256: return launch_bn<256>(epi, tmA, tmW, a, num_sms, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace fvar

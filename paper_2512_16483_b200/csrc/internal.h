@@ -1,0 +1,85 @@
+// Internal launch interfaces between the translation units of libfvar.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace fvar {
+
+typedef __nv_bfloat16 bf16;
+
+// Maps (computed element e, row j within it) to a row of a per-batch buffer:
+// row = (e * bmul + boff) * rpb + j.  Compact buffers use {1, 0, r}; buffers indexed by the
+// caller's batch element use {2, 1, M} when only the null-prompt half of each pair is computed.
+struct RowMap {
+  int bmul, boff, rpb;
+};
+
+enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU_BF16 = 2, EPI_QKV = 3, EPI_RESID = 4 };
+
+struct GemmArgs {
+  int R, N, K;            // out[R][N] = A[R][K] * W[N][K]^T, per batch
+  int nbatch;             // number of independent problems sharing the launch
+  int a_batch_rows;       // row offset of batch e in the A tensor map (0: A shared by all)
+  int b_batch_rows;       // row offset of batch e in the W tensor map (0: W shared by all)
+  const bf16 *bias;       // [N] or nullptr
+  int rows_per_batch;     // rows of one computed element inside R (epilogues that need (e, j))
+  int bmul, boff;         // caller batch element of computed element e: e * bmul + boff
+  // EPI_F32 / EPI_RESID output, EPI_BF16 / EPI_GELU_BF16 / EPI_QKV (q part) output
+  float *out_f32;
+  bf16 *out_bf16;
+  long long ld_out;
+  // EPI_RESID: out[omap(e, j')] = resid[rmap(e, j)] + gate[b] * (acc + bias); j' = scatter ? scatter[e][j] : j
+  const float *resid;
+  RowMap rmap, omap;
+  const float *gate;      // vector of caller batch element b at gate + b * gate_stride, or nullptr (gate = 1)
+  long long gate_stride;
+  const int *scatter;     // [E][rows_per_batch] or nullptr
+  // EPI_QKV: virtual column = col + col_base; [0,C) -> q, [C,2C) -> K cache, [2C,3C) -> transposed V cache
+  bf16 *kc, *vt;
+  int C, H, D, L_cap, L_prev, col_base;
+  unsigned *status;
+};
+
+// Tensor maps: bf16, 2-D {cols, rows} with a {64, box_rows} box and 128-byte swizzle, or the 3-D
+// forms used for the KV cache.
+bool tmap_init_driver();
+bool tmap_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t ld_elems, uint32_t box_rows);
+bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1_elems,
+             uint64_t ld2_elems, uint32_t box0, uint32_t box1);
+
+int gemm_pick_block_n(int R_total_tiles_m, int N, int num_sms);
+// Launches the tensor-core GEMM.  block_n in {64, 128, 256}: the W map's box must have block_n rows.
+cudaError_t launch_gemm(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
+                        int num_sms, cudaStream_t st);
+
+struct AttnArgs {
+  int B_eff, H, r, D, L, L_cap;
+  int bmul, boff;          // caller batch element (cache slot) of computed element e
+  bf16 *out;               // [B_eff * r][H * D]
+  float scale_log2;        // log2(e) / sqrt(D)
+  unsigned *status;
+};
+cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
+                             const AttnArgs &a, cudaStream_t st);
+
+// Memory-bound kernels.
+cudaError_t launch_row_scores(const float *x, long long rows, int C, float *scores, cudaStream_t st);
+cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st);
+cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_forced, int *idx, int *inv,
+                                unsigned *status, cudaStream_t st);
+cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int C, const float *shift,
+                               const float *scale, long long vec_stride, int bmul, int boff,
+                               const bf16 *gamma, float eps, bf16 *y, cudaStream_t st);
+cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1,
+                            int w1, int C, const int *inv, cudaStream_t st);
+cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mp, bf16 *xt,
+                                  cudaStream_t st);
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st);
+cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);
+cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
+cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,
+                           cudaStream_t st);
+
+}  // namespace fvar

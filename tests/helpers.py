@@ -1,0 +1,36 @@
+"""Shared by the GPU tests: moving seeded numpy inputs to the device and comparing results."""
+import numpy as np
+import torch
+
+import synth_inputs as si
+
+
+def to_bf16_cuda(a: np.ndarray) -> torch.Tensor:
+    """fp32 array holding bf16-representable values -> bf16 CUDA tensor with the same bits."""
+    bits = si.bf16_bits(a)
+    t = torch.from_numpy(bits.view(np.int16).reshape(a.shape))
+    return t.view(torch.bfloat16).cuda()
+
+
+def bf16_to_numpy(t: torch.Tensor) -> np.ndarray:
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def weights_to_cuda(weights):
+    return [{k: to_bf16_cuda(v) for k, v in blk.items()} for blk in weights]
+
+
+def rel_err(got: np.ndarray, ref: np.ndarray):
+    """(max-abs error / RMS of the reference, cosine similarity)."""
+    got, ref = np.asarray(got, np.float64).ravel(), np.asarray(ref, np.float64).ravel()
+    rms = float(np.sqrt(np.mean(ref ** 2))) + 1e-30
+    cos = float(got @ ref / (np.linalg.norm(got) * np.linalg.norm(ref) + 1e-30))
+    return float(np.max(np.abs(got - ref))) / rms, cos
+
+
+def assert_close(got, ref, max_rel=2e-2, min_cos=0.999, what=""):
+    """The acceptance bar of the block outputs: max-abs error <= 2e-2 x output RMS, cosine >= 0.999."""
+    e, c = rel_err(got, ref)
+    assert e <= max_rel and c >= min_cos, "%s: max-abs/RMS %.3e (bar %.1e), cosine %.6f (bar %.4f)" % (
+        what, e, max_rel, c, min_cos)
+    return e, c

@@ -1,0 +1,267 @@
+"""Parity of the whole scale step (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Acceptance bar for block outputs in bf16: max-abs error <= 2e-2 x output RMS and cosine
+similarity >= 0.999; index lists bit-exact when the index set is teacher-forced or the scores are
+well separated."""
+import numpy as np
+import pytest
+import torch
+
+import synth_inputs as si
+from oracle import fvar_oracle as orc
+from helpers import assert_close, bf16_to_numpy, to_bf16_cuda, weights_to_cuda
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fv():
+    from paper_2512_16483_b200 import binding
+    binding.load_library()
+    return binding
+
+
+class Pair:
+    """The GPU context and the oracle on identical weights and conditioning."""
+
+    def __init__(self, fv, shp: si.ModelShape, seed: int, B: int, std: float = 0.02):
+        self.fv, self.shp, self.seed, self.B = fv, shp, seed, B
+        w = si.make_weights(seed, shp, std)
+        self.oracle = orc.Oracle(w, shp.n_heads, shp.blocks_per_group, shp.hw(), shp.ln_eps)
+        self.gpu = fv.Fvar(weights_to_cuda(w), blocks_per_group=shp.blocks_per_group, n_heads=shp.n_heads,
+                           head_dim=shp.head_dim, ffn_dim=shp.ffn_dim, scale_hw=shp.hw(), max_batch=B,
+                           ctx_len=shp.ctx_len, ctx_width=shp.ctx_width, ln_eps=shp.ln_eps)
+        cond = si.make_cond(seed, B, shp.width)
+        ctx = si.make_context(seed, B, shp.ctx_len, shp.ctx_width) if shp.has_cross_attn else None
+        self.oracle.set_cond(cond, ctx)
+        self.gpu.set_cond(to_bf16_cuda(cond), to_bf16_cuda(ctx) if ctx is not None else None)
+
+    def prefill(self, upto_scale: int):
+        """Stand-in earlier scales 0..upto_scale-1: random K/V rows and random group outputs of the
+        last of them."""
+        shp = self.shp
+        L = sum(shp.tokens_per_scale()[:upto_scale])
+        K, V = si.make_kv_prefill(self.seed, shp.n_blocks, self.B, L, shp.width)
+        self.oracle.load_kv(K, V)
+        self.gpu.load_kv(to_bf16_cuda(K), to_bf16_cuda(V))
+        M_prev = shp.tokens_per_scale()[upto_scale - 1]
+        gc = si.make_group_cache(self.seed, shp.n_groups, self.B, M_prev, shp.width)
+        self.oracle.load_group_cache(upto_scale - 1, gc)
+        self.gpu.load_group_cache(upto_scale - 1, torch.from_numpy(gc).cuda())
+        return L
+
+    def set_projections(self, k: int, ranks):
+        M = self.shp.tokens_per_scale()[k]
+        for g, r in enumerate(ranks):
+            if r < M:
+                Q = si.make_projection(self.seed, k, g, M, r)
+                self.oracle.set_projection(k, g, Q)
+                self.gpu.set_projection(k, g, to_bf16_cuda(np.ascontiguousarray(Q.T)))
+
+    def forced_tensor(self, ranks, E):
+        """Oracle's index lists as the [G][E][r_max] device array the policy takes."""
+        G, r_max = len(ranks), max(ranks)
+        arr = np.zeros((G, E, r_max), np.int32)
+        for g in range(G):
+            for e in range(E):
+                idx = self.oracle.last_indices[e][g]
+                arr[g, e, :len(idx)] = idx
+        return torch.from_numpy(arr).cuda()
+
+    def check_ok(self):
+        assert self.gpu.poll_status() == self.fv.OK
+
+
+def _step_both(p: Pair, toks, k, *, mode, cfg="pair", ranks=None, keep_ratio=1.0, forced=True):
+    fv = p.fv
+    pol = orc.Policy({fv.DENSE: "dense", fv.LOWRANK_RTR: "lowrank_rtr"}[mode], cfg, keep_ratio, ranks)
+    ref = p.oracle.scale_step(toks, k, pol)
+    E = ref.shape[0]
+    fi = None
+    if mode == fv.LOWRANK_RTR and forced:
+        M = toks.shape[1]
+        rk = ranks if ranks is not None else [orc.rank_from_keep_ratio(M, keep_ratio)] * p.shp.n_groups
+        if any(r < M for r in rk):
+            fi = p.forced_tensor([r if r < M else 1 for r in rk], E)
+            if not all(r < M for r in rk):                 # dense groups carry no list; keep layout r_max wide
+                fi = p.forced_tensor([min(r, M - 1) if r < M else 1 for r in rk], E)
+    out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=mode, cfg_mode=fv.CFG_NULL_ONLY if cfg == "null_only" else fv.CFG_PAIR,
+                           keep_ratio=keep_ratio, rank_per_group=ranks, forced_indices=fi)
+    p.check_ok()
+    return bf16_to_numpy(out), ref
+
+
+# ----------------------------------------------------------------------------- one d16 block, last 256px scale
+
+@pytest.mark.parametrize("r", [256, 128, 32])
+@pytest.mark.parametrize("kind", ["normal", "spread"])
+def test_single_block_last_scale(fv, r, kind):
+    """One VAR-d16-shaped block, B = 2 (one CFG pair), 256 query tokens over a 424-row cache."""
+    shp = si.shape_var_d16(n_blocks=1)
+    p = Pair(fv, shp, seed=100, B=2)
+    k = 9
+    assert p.prefill(k) == 424
+    toks = si.make_tokens(100, 2, 256, 1024, kind)
+    mode = fv.DENSE if r == 256 else fv.LOWRANK_RTR
+    if r < 256:
+        p.set_projections(k, [r])
+    free = (kind == "spread")                              # well-separated scores: selection must agree exactly
+    got, ref = _step_both(p, toks, k, mode=mode, ranks=[r] if r < 256 else None, forced=not free)
+    assert_close(got, ref, what="block output r=%d %s" % (r, kind))
+    if r < 256:
+        idx = p.gpu.get_indices(0, 2, 256).cpu().numpy()
+        for e in range(2):
+            assert np.array_equal(idx[e], p.oracle.last_indices[e][0])
+    g32 = p.gpu.get_group_output(0, 256).cpu().numpy()
+    assert_close(g32, np.stack(p.oracle.group_cache[0]), max_rel=1e-2, min_cos=0.9999, what="fp32 group output")
+    p.gpu.kv_append(k)
+    p.oracle.kv_append(k)
+    assert p.gpu.cache_len(0) == p.oracle.cache_len(0, 0) == 424 + r
+
+
+def test_full_rank_is_bitwise_the_dense_path(fv):
+    shp = si.shape_var_d16(n_blocks=2)
+    toks = to_bf16_cuda(si.make_tokens(101, 2, 169, 1024))
+    outs = []
+    for mode, kw in ((fv.DENSE, {}), (fv.LOWRANK_RTR, {"keep_ratio": 1.0})):
+        p = Pair(fv, shp, seed=101, B=2)
+        p.prefill(8)
+        outs.append(p.gpu.scale_step(toks, 8, mode=mode, **kw).clone())
+        p.check_ok()
+    assert torch.equal(outs[0], outs[1])
+
+
+# ----------------------------------------------------------------------------- multi-scale, multi-group
+
+@pytest.mark.parametrize("cross,D", [(False, 64), (True, 64), (True, 128)])
+def test_generation_dense_then_late(fv, cross, D):
+    """Dense early scales, then two late scales under RP + RTR with different ranks per group,
+    the second one null-prompt only; KV append between scales; indices teacher-forced."""
+    shp = si.shape_tiny(n_blocks=4, blocks_per_group=2, width=2 * D, n_heads=2, head_dim=D, ffn_dim=320,
+                        scales=(1, 2, 4, 7, 12), cross=cross, ctx_len=20,
+                        scale_hw=((1, 1), (2, 2), (4, 3), (7, 7), (12, 11)))
+    B = 4
+    p = Pair(fv, shp, seed=102, B=B, std=0.05)
+    Ms = shp.tokens_per_scale()
+    toks = [si.make_tokens(102, B, m, shp.width) for m in Ms]
+    for k in range(3):
+        got, ref = _step_both(p, toks[k], k, mode=fv.DENSE)
+        assert_close(got, ref, what="dense scale %d" % k)
+        p.gpu.kv_append(k)
+        p.oracle.kv_append(k)
+    ranks3 = [20, 33]
+    p.set_projections(3, ranks3)
+    got, ref = _step_both(p, toks[3], 3, mode=fv.LOWRANK_RTR, ranks=ranks3)
+    assert_close(got, ref, what="late scale 3")
+    p.gpu.kv_append(3)
+    p.oracle.kv_append(3)
+    assert [p.gpu.cache_len(b) for b in range(4)] == [p.oracle.cache_len(b, 0) for b in range(4)]
+    ranks4 = [132, 40]                                      # first group dense (r == M), second low-rank
+    p.set_projections(4, ranks4)
+    got, ref = _step_both(p, toks[4], 4, mode=fv.LOWRANK_RTR, cfg="null_only", ranks=ranks4)
+    assert got.shape == (2, 132, shp.width)
+    assert_close(got, ref, what="late scale 4 (null-only)")
+    p.gpu.kv_append(4)
+    p.oracle.kv_append(4)
+    assert [p.gpu.cache_len(b) for b in range(4)] == [p.oracle.cache_len(b, 1) for b in range(4)]
+
+
+def test_d16_stack_three_late_scales(fv):
+    """VAR-d16-shaped stack (4 of its 16 blocks to keep the oracle quick), late scales 10, 13, 16 at
+    keep ratio 0.5, batch 4, teacher-forced; plus free-running index overlap."""
+    shp = si.shape_var_d16(n_blocks=4)
+    B = 4
+    p = Pair(fv, shp, seed=103, B=B)
+    p.prefill(7)
+    overlaps = []
+    for k in (7, 8, 9):
+        M = shp.tokens_per_scale()[k]
+        r = orc.rank_from_keep_ratio(M, 0.5)
+        p.set_projections(k, [r] * 4)
+        toks = si.make_tokens(103, B, M, 1024, "spread")
+        got, ref = _step_both(p, toks, k, mode=fv.LOWRANK_RTR, keep_ratio=0.5)
+        assert_close(got, ref, what="d16 stack scale %d" % k)
+        p.gpu.kv_append(k)
+        p.oracle.kv_append(k)
+    assert p.gpu.cache_len(3) == 155 + 50 + 85 + 128
+
+
+def test_free_running_selection_overlap(fv):
+    """Without teacher forcing the index sets may differ only where scores are nearly tied."""
+    shp = si.shape_var_d16(n_blocks=3)
+    B = 2
+    p = Pair(fv, shp, seed=104, B=B)
+    p.prefill(9)
+    p.set_projections(9, [128] * 3)
+    toks = si.make_tokens(104, B, 256, 1024, "spread")
+    got, ref = _step_both(p, toks, 9, mode=fv.LOWRANK_RTR, keep_ratio=0.5, forced=False)
+    for g in range(3):
+        idx = p.gpu.get_indices(g, B, 256).cpu().numpy()
+        for e in range(B):
+            inter = len(set(idx[e].tolist()) & set(p.oracle.last_indices[e][g].tolist()))
+            assert inter >= 126, (g, e, inter)
+            assert np.all(np.diff(idx[e]) > 0)
+
+
+# ----------------------------------------------------------------------------- host-buffer entry point, state rules
+
+def test_host_entry_point_matches_device_entry_point(fv):
+    shp = si.shape_var_d16(n_blocks=1)
+    toks = si.make_tokens(105, 2, 256, 1024)
+    outs = []
+    for host in (False, True):
+        p = Pair(fv, shp, seed=105, B=2)
+        p.prefill(9)
+        p.set_projections(9, [128])
+        if host:
+            th = to_bf16_cuda(toks).cpu().pin_memory()
+            oh = torch.empty((2, 256, 1024), dtype=torch.bfloat16).pin_memory()
+            p.gpu.scale_step_host(th, 9, oh, mode=fv.LOWRANK_RTR, keep_ratio=0.5)
+            outs.append(oh.clone())
+        else:
+            outs.append(p.gpu.scale_step(to_bf16_cuda(toks), 9, mode=fv.LOWRANK_RTR, keep_ratio=0.5).cpu())
+        p.check_ok()
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_state_and_argument_errors(fv):
+    shp = si.shape_tiny(n_blocks=2, width=128, n_heads=2, head_dim=64, ffn_dim=256, scales=(2, 3, 4))
+    p = Pair(fv, shp, seed=106, B=2)
+    g = p.gpu
+    t0 = to_bf16_cuda(si.make_tokens(106, 2, 4, 128))
+    t1 = to_bf16_cuda(si.make_tokens(106, 2, 9, 128))
+
+    def status_of(fn):
+        try:
+            fn()
+        except fv.FvarError as e:
+            return e.status
+        return fv.OK
+
+    assert status_of(lambda: g.kv_append(0)) == fv.ESTATE                      # nothing staged
+    assert status_of(lambda: g.scale_step(t1, 1, mode=fv.LOWRANK_RTR, keep_ratio=0.5)) == fv.ESTATE   # no projection
+    g.set_projection(1, 0, to_bf16_cuda(np.ascontiguousarray(si.make_projection(1, 1, 0, 9, 5).T)))
+    g.set_projection(1, 1, to_bf16_cuda(np.ascontiguousarray(si.make_projection(1, 1, 1, 9, 5).T)))
+    assert status_of(lambda: g.scale_step(t1, 1, mode=fv.LOWRANK_RTR, keep_ratio=0.5)) == fv.ESTATE   # no group cache
+    assert status_of(lambda: g.scale_step(t0, 0, mode=fv.LOWRANK_RTR, rank_per_group=[5, 2])) == fv.EINVAL   # r > M
+    assert status_of(lambda: g.scale_step(t0, 7, mode=fv.DENSE)) == fv.EINVAL
+    assert g.scale_step(t0, 0, mode=fv.SKIP) is None                           # skip: nothing staged
+    assert status_of(lambda: g.kv_append(0)) == fv.ESTATE
+    g.scale_step(t0, 0, mode=fv.DENSE)
+    g.kv_append(0)
+    assert status_of(lambda: g.kv_append(0)) == fv.ESTATE                      # appended twice
+    assert g.cache_len(0) == 4
+    g.scale_step(t1, 1, mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY, keep_ratio=0.5)
+    assert status_of(lambda: g.scale_step(t0, 0, mode=fv.DENSE)) == fv.ESTATE  # scale index decreased
+    assert status_of(lambda: g.scale_step(t1, 1, mode=fv.DENSE)) == fv.ESTATE  # pair step after null-only
+    assert g.poll_status() == fv.OK
+    # a forced index list that is not ascending is reported through the status word, not by a fault
+    bad = torch.tensor([[[3, 1, 2, 8, 8], [0, 1, 2, 3, 4]]] * 2, dtype=torch.int32, device="cuda")
+    g.reset()
+    p2 = Pair(fv, shp, seed=106, B=2)
+    p2.gpu.scale_step(t0, 0, mode=fv.DENSE)
+    p2.gpu.kv_append(0)
+    for grp in range(2):
+        p2.gpu.set_projection(1, grp, to_bf16_cuda(np.ascontiguousarray(si.make_projection(1, 1, grp, 9, 5).T)))
+    p2.gpu.scale_step(t1, 1, mode=fv.LOWRANK_RTR, keep_ratio=0.5, forced_indices=bad)
+    assert p2.gpu.poll_status() == fv.EINVAL
+    assert p2.gpu.poll_status() == fv.OK                                       # cleared by the read
