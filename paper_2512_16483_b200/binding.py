@@ -264,6 +264,8 @@ class Fvar:
         return pol, keep
 
     def out_shape(self, scale_idx: int, cfg_mode: int):
+        if not 0 <= scale_idx < len(self.scale_hw):
+            return (1,)                                  # the library rejects the index
         h, w = self.scale_hw[scale_idx]
         return (self.B // 2 if cfg_mode == CFG_NULL_ONLY else self.B, h * w, self.width)
 

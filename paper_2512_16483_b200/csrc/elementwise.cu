@@ -320,9 +320,13 @@ cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int 
 }
 
 // ------------------------------------------------------------------------------------------------
-// xt[e][c][m] (bf16, row stride Mp) = x[row(e, m)][c] (fp32): 32 x 32 tiles through shared memory.
+// Transposed two-term bf16 split of the fp32 rows for the projection GEMM:
+// xt[e][c][m] = hi(x[row(e, m)][c]) and xt[e][c][Mk + m] = lo(...), hi = bf16(x), lo = bf16(x - hi),
+// so that the tensor-core product Q^T (hi + lo) carries ~16 mantissa bits of x.  Mk = M rounded up
+// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  32 x 32 tiles
+// through shared memory.
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
-                                                             int Mp, bf16 *__restrict__ xt) {
+                                                             int Mk, bf16 *__restrict__ xt) {
   __shared__ float tile[32][33];
   const int e = blockIdx.z, m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -332,17 +336,23 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__rest
     tile[k][tx] = (m < M && c < C) ? src[static_cast<long long>(m) * C + c] : 0.f;
   }
   __syncthreads();
-  bf16 *dst = xt + static_cast<long long>(e) * C * Mp;
+  bf16 *dst = xt + static_cast<long long>(e) * C * 2 * Mk;
   for (int k = ty; k < 32; k += 8) {
     const int c = c0 + k, m = m0 + tx;
-    if (c < C && m < Mp) dst[static_cast<long long>(c) * Mp + m] = __float2bfloat16_rn(m < M ? tile[tx][k] : 0.f);
+    if (c < C && m < Mk) {
+      const float v = tile[tx][k];
+      const bf16 hi = __float2bfloat16_rn(v);
+      const bf16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+      dst[static_cast<long long>(c) * 2 * Mk + m] = hi;
+      dst[static_cast<long long>(c) * 2 * Mk + Mk + m] = lo;
+    }
   }
 }
 
-cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mp, bf16 *xt,
+cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
                                   cudaStream_t st) {
-  dim3 grid((Mp + 31) / 32, (C + 31) / 32, E);
-  transpose_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, Mp, xt);
+  dim3 grid((Mk + 31) / 32, (C + 31) / 32, E);
+  transpose_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, Mk, xt);
   return cudaGetLastError();
 }
 

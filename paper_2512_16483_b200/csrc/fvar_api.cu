@@ -152,7 +152,7 @@ Layout make_layout(const fvar_cfg *c) {
     Ltot += m;
   }
   const size_t L_cap = align_up(Ltot, 128), ctx_cap = c->has_cross_attn ? align_up(c->ctx_len, 128) : 0;
-  const size_t Mp = align_up(Mmax, 8);
+  const size_t Mk = align_up(Mmax, 64);          // projection operands: [hi | lo] halves of Mk columns
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
   L.status = take(256);
@@ -169,7 +169,7 @@ Layout make_layout(const fvar_cfg *c) {
   L.q = take(B * Mmax * C * 2);
   L.a = take(B * Mmax * C * 2);
   L.hbuf = take(B * Mmax * F * 2);
-  L.xt = take(B * C * Mp * 2);
+  L.xt = take(B * C * 2 * Mk * 2);
   L.scores = take(B * Mmax * 4);
   L.idx = take(G * B * Mmax * 4);
   L.inv = take(G * B * Mmax * 4);
@@ -180,7 +180,7 @@ Layout make_layout(const fvar_cfg *c) {
     const size_t m = static_cast<size_t>(c->scale_hw[2 * k]) * c->scale_hw[2 * k + 1];
     for (size_t g = 0; g < G; ++g) {
       L.qt_off[k * G + g] = pool;
-      pool += align_up(m * align_up(m, 8), 512);       // elements; r <= M rows of padded length
+      pool += align_up(m * 2 * align_up(m, 64), 512);  // elements; r <= M rows of [Q^T | Q^T]
     }
   }
   take(pool * 2);
@@ -331,8 +331,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->xt_map.resize(static_cast<size_t>(cfg->n_scales) * 3);
   for (int k = 0; k < cfg->n_scales && ok; ++k)
     for (int t = 0; t < 3 && ok; ++t)
-      ok = tmap_2d(&c->xt_map[k * 3 + t], c->xt, c->Mk[k], static_cast<size_t>(c->Bmax) * C, align_up(c->Mk[k], 8),
-                   kBNs[t]);
+      ok = tmap_2d(&c->xt_map[k * 3 + t], c->xt, align_up(c->Mk[k], 64) + c->Mk[k], static_cast<size_t>(c->Bmax) * C,
+                   2 * align_up(c->Mk[k], 64), kBNs[t]);
   c->kmap.resize(nb); c->vmap.resize(nb); c->ckmap.resize(nb); c->cvmap.resize(nb);
   const int BH = c->Bmax * c->H, D = c->D;
   for (int b = 0; b < nb && ok; ++b) {
@@ -436,11 +436,14 @@ fvar_status fvar_set_projection(fvar_ctx *ctx, int scale_idx, int group, const v
     return fail(ctx, FVAR_EINVAL, "set_projection: bad scale / group / pointer");
   const int M = ctx->Mk[scale_idx];
   if (r <= 0 || r > M) return fail(ctx, FVAR_EINVAL, "set_projection: need 0 < r <= M");
-  const size_t Mp = align_up(M, 8), slot = static_cast<size_t>(scale_idx) * ctx->G + group;
+  // Stored as [Q^T | Q^T] with each half padded to Mk columns: the projection GEMM multiplies it
+  // with the [hi | lo] split of the token rows (the padding stays zero from fvar_init).
+  const size_t Mk = align_up(M, 64), slot = static_cast<size_t>(scale_idx) * ctx->G + group;
   bf16 *dst = ctx->qt_pool + ctx->qt_off[slot];
-  FV_CUDA(ctx, cudaMemcpy2DAsync(dst, Mp * 2, Qt, static_cast<size_t>(M) * 2, static_cast<size_t>(M) * 2, r,
-                                 cudaMemcpyDeviceToDevice, ctx->st), "projection copy");
-  if (!tmap_2d(&ctx->qt_map[slot], dst, M, r, Mp, 128)) return fail(ctx, FVAR_ECUDA, "projection tensor map");
+  for (int half = 0; half < 2; ++half)
+    FV_CUDA(ctx, cudaMemcpy2DAsync(dst + half * Mk, 2 * Mk * 2, Qt, static_cast<size_t>(M) * 2, static_cast<size_t>(M) * 2, r,
+                                   cudaMemcpyDeviceToDevice, ctx->st), "projection copy");
+  if (!tmap_2d(&ctx->qt_map[slot], dst, Mk + M, r, 2 * Mk, 128)) return fail(ctx, FVAR_ECUDA, "projection tensor map");
   ctx->qt_r[slot] = r;
   return FVAR_OK;
 }
@@ -558,11 +561,12 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, st), "select_topr");
         ctx->launches++;
       }
-      const int Mp = static_cast<int>(align_up(M, 8));
-      FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mp, ctx->xt, st), "transpose");
+      const int Mk = static_cast<int>(align_up(M, 64));
+      FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mk, ctx->xt, st), "transpose");
       ctx->launches++;
-      // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e
-      GemmArgs ga = gemm_args(r, C, M);
+      // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e; the reduction
+      // runs over the hi and lo halves of X
+      GemmArgs ga = gemm_args(r, C, Mk + M);
       ga.nbatch = E;
       ga.a_batch_rows = 0;
       ga.b_batch_rows = C;

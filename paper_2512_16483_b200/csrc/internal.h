@@ -74,7 +74,7 @@ cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int
                                const bf16 *gamma, float eps, bf16 *y, cudaStream_t st);
 cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1,
                             int w1, int C, const int *inv, cudaStream_t st);
-cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mp, bf16 *xt,
+cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
                                   cudaStream_t st);
 cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st);
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);

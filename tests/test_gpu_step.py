@@ -8,7 +8,7 @@ import torch
 
 import synth_inputs as si
 from oracle import fvar_oracle as orc
-from helpers import assert_close, bf16_to_numpy, to_bf16_cuda, weights_to_cuda
+from helpers import assert_close, assert_out_close, bf16_to_numpy, to_bf16_cuda, weights_to_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -64,7 +64,8 @@ class Pair:
         for g in range(G):
             for e in range(E):
                 idx = self.oracle.last_indices[e][g]
-                arr[g, e, :len(idx)] = idx
+                if len(idx) <= r_max:                        # dense groups (r == M) carry no list
+                    arr[g, e, :len(idx)] = idx
         return torch.from_numpy(arr).cuda()
 
     def check_ok(self):
@@ -82,8 +83,6 @@ def _step_both(p: Pair, toks, k, *, mode, cfg="pair", ranks=None, keep_ratio=1.0
         rk = ranks if ranks is not None else [orc.rank_from_keep_ratio(M, keep_ratio)] * p.shp.n_groups
         if any(r < M for r in rk):
             fi = p.forced_tensor([r if r < M else 1 for r in rk], E)
-            if not all(r < M for r in rk):                 # dense groups carry no list; keep layout r_max wide
-                fi = p.forced_tensor([min(r, M - 1) if r < M else 1 for r in rk], E)
     out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=mode, cfg_mode=fv.CFG_NULL_ONLY if cfg == "null_only" else fv.CFG_PAIR,
                            keep_ratio=keep_ratio, rank_per_group=ranks, forced_indices=fi)
     p.check_ok()
@@ -106,13 +105,13 @@ def test_single_block_last_scale(fv, r, kind):
         p.set_projections(k, [r])
     free = (kind == "spread")                              # well-separated scores: selection must agree exactly
     got, ref = _step_both(p, toks, k, mode=mode, ranks=[r] if r < 256 else None, forced=not free)
-    assert_close(got, ref, what="block output r=%d %s" % (r, kind))
+    assert_out_close(got, ref, what="block output r=%d %s" % (r, kind))
     if r < 256:
         idx = p.gpu.get_indices(0, 2, 256).cpu().numpy()
         for e in range(2):
             assert np.array_equal(idx[e], p.oracle.last_indices[e][0])
     g32 = p.gpu.get_group_output(0, 256).cpu().numpy()
-    assert_close(g32, np.stack(p.oracle.group_cache[0]), max_rel=1e-2, min_cos=0.9999, what="fp32 group output")
+    assert_close(g32, np.stack(p.oracle.group_cache[0]), what="fp32 group output")
     p.gpu.kv_append(k)
     p.oracle.kv_append(k)
     assert p.gpu.cache_len(0) == p.oracle.cache_len(0, 0) == 424 + r
@@ -145,13 +144,13 @@ def test_generation_dense_then_late(fv, cross, D):
     toks = [si.make_tokens(102, B, m, shp.width) for m in Ms]
     for k in range(3):
         got, ref = _step_both(p, toks[k], k, mode=fv.DENSE)
-        assert_close(got, ref, what="dense scale %d" % k)
+        assert_out_close(got, ref, what="dense scale %d" % k)
         p.gpu.kv_append(k)
         p.oracle.kv_append(k)
     ranks3 = [20, 33]
     p.set_projections(3, ranks3)
     got, ref = _step_both(p, toks[3], 3, mode=fv.LOWRANK_RTR, ranks=ranks3)
-    assert_close(got, ref, what="late scale 3")
+    assert_out_close(got, ref, what="late scale 3")
     p.gpu.kv_append(3)
     p.oracle.kv_append(3)
     assert [p.gpu.cache_len(b) for b in range(4)] == [p.oracle.cache_len(b, 0) for b in range(4)]
@@ -159,7 +158,7 @@ def test_generation_dense_then_late(fv, cross, D):
     p.set_projections(4, ranks4)
     got, ref = _step_both(p, toks[4], 4, mode=fv.LOWRANK_RTR, cfg="null_only", ranks=ranks4)
     assert got.shape == (2, 132, shp.width)
-    assert_close(got, ref, what="late scale 4 (null-only)")
+    assert_out_close(got, ref, what="late scale 4 (null-only)")
     p.gpu.kv_append(4)
     p.oracle.kv_append(4)
     assert [p.gpu.cache_len(b) for b in range(4)] == [p.oracle.cache_len(b, 1) for b in range(4)]
@@ -179,7 +178,7 @@ def test_d16_stack_three_late_scales(fv):
         p.set_projections(k, [r] * 4)
         toks = si.make_tokens(103, B, M, 1024, "spread")
         got, ref = _step_both(p, toks, k, mode=fv.LOWRANK_RTR, keep_ratio=0.5)
-        assert_close(got, ref, what="d16 stack scale %d" % k)
+        assert_out_close(got, ref, what="d16 stack scale %d" % k)
         p.gpu.kv_append(k)
         p.oracle.kv_append(k)
     assert p.gpu.cache_len(3) == 155 + 50 + 85 + 128
