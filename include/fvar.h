@@ -140,6 +140,23 @@ fvar_status fvar_get_group_output(fvar_ctx *ctx, int group, float *out_dev);
 fvar_status fvar_load_kv(fvar_ctx *ctx, const void *K, const void *V, int L);
 fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cache);
 
+/* Returns to the state the last fvar_load_kv and fvar_load_group_cache established (cache lengths,
+ * group outputs, last stepped scale), so that the late scales can be run again, e.g. under another
+ * policy.  O(1), host only; the loaded group outputs are kept in a slot of their own that steps never
+ * overwrite.  FVAR_ESTATE if nothing was loaded. */
+fvar_status fvar_restore_loaded(fvar_ctx *ctx);
+
+/* Measurement aid: while enabled, every kernel launch of this context is bracketed by CUDA events on
+ * the context's stream.  fvar_profile_read synchronises and sums, for one kernel class, the event
+ * time, the number of launches and the algorithmic flops and bytes (minimum traffic: operands read
+ * once, results written once) of the launches recorded since fvar_profile_enable(ctx, 1). */
+enum { FVAR_KCLASS_GEMM = 0, FVAR_KCLASS_ATTENTION = 1, FVAR_KCLASS_LN = 2, FVAR_KCLASS_SCORE = 3,
+       FVAR_KCLASS_SELECT = 4, FVAR_KCLASS_TRANSPOSE = 5, FVAR_KCLASS_RTR_FILL = 6, FVAR_KCLASS_CONVERT = 7,
+       FVAR_KCLASS_COUNT = 8 };
+fvar_status fvar_profile_enable(fvar_ctx *ctx, int on);
+fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long long *launches, double *flops,
+                              double *bytes);
+
 /* Committed cache rows of `block` (host value). */
 int fvar_cache_len(const fvar_ctx *ctx, int block);
 

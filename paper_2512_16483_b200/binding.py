@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libfvar.so")
 OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
+KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")
 
@@ -78,6 +79,9 @@ def load_library() -> ct.CDLL:
         "fvar_launch_count": (ll, [vp]),
         "fvar_poll_status": (i, [vp]),
         "fvar_reset": (i, [vp]),
+        "fvar_restore_loaded": (i, [vp]),
+        "fvar_profile_enable": (i, [vp, i]),
+        "fvar_profile_read": (i, [vp, i, P(ct.c_double), P(ll), P(ct.c_double), P(ct.c_double)]),
         "fvar_destroy": (None, [vp]),
         "fvar_last_error": (ct.c_char_p, [vp]),
         "fvar_row_scores": (i, [vp, i, i, i, vp, vp]),
@@ -97,7 +101,8 @@ def load_library() -> ct.CDLL:
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
-            "fvar_destroy", "fvar_last_error", "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
+            "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_profile_enable", "fvar_profile_read",
+            "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
             "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill")
 
 
@@ -325,3 +330,15 @@ class Fvar:
 
     def reset(self):
         self._check(self.lib.fvar_reset(self.ctx))
+
+    def restore_loaded(self):
+        self._check(self.lib.fvar_restore_loaded(self.ctx))
+
+    def profile_enable(self, on: bool):
+        self._check(self.lib.fvar_profile_enable(self.ctx, int(on)))
+
+    def profile_read(self, kclass: int):
+        """(total ms, launches, algorithmic flops, algorithmic bytes) of one kernel class."""
+        ms, n, fl, by = ct.c_double(0), ct.c_longlong(0), ct.c_double(0), ct.c_double(0)
+        self._check(self.lib.fvar_profile_read(self.ctx, kclass, ct.byref(ms), ct.byref(n), ct.byref(fl), ct.byref(by)))
+        return ms.value, n.value, fl.value, by.value

@@ -110,11 +110,37 @@ struct fvar_ctx {
   int null_only_seen;
   std::vector<int> last_rank;          // r per group of the last step
   int last_E, last_M;
+  int loaded_len, loaded_cache_scale;  // state set by fvar_load_kv / fvar_load_group_cache (-1: none)
+  // per-launch event timing (fvar_profile_*)
+  struct ProfRec { int kclass; double flops, bytes; cudaEvent_t e0, e1; };
+  bool prof_on;
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used;
 
   size_t kv_block_elems() const { return static_cast<size_t>(Bmax) * H * L_cap * D; }
   size_t ckv_block_elems() const { return static_cast<size_t>(Bmax) * H * ctx_cap * D; }
+  // slots 0 and 1 alternate between scale steps; slot 2 holds what fvar_load_group_cache loaded
   float *gslot(int slot, int g) const {
     return gcache + (static_cast<size_t>(slot) * G + g) * Bmax * Mmax * C;
+  }
+  cudaEvent_t event() {
+    if (ev_used == ev_pool.size()) {
+      cudaEvent_t e = nullptr;
+      cudaEventCreate(&e);
+      ev_pool.push_back(e);
+    }
+    return ev_pool[ev_used++];
+  }
+  void prof_begin(int kclass, double flops, double bytes) {
+    if (!prof_on) return;
+    ProfRec r{kclass, flops, bytes, event(), event()};
+    cudaEventRecord(r.e0, st);
+    prof.push_back(r);
+  }
+  void launched() {
+    launches++;
+    if (prof_on && !prof.empty()) cudaEventRecord(prof.back().e1, st);
   }
   const CUtensorMap &wm(int blk, int wid, int bn) const { return wmap[(blk * W_COUNT + wid) * 3 + bn_index(bn)]; }
 };
@@ -162,7 +188,7 @@ Layout make_layout(const fvar_cfg *c) {
   L.cvt = take(nb * B * ctx_cap * C * 2);
   L.ada = take(nb * B * 6 * C * 4);
   L.silu_c = take(align_up(B, 128) * C * 2);
-  L.gcache = take(2 * G * B * Mmax * C * 4);
+  L.gcache = take(3 * G * B * Mmax * C * 4);
   L.x0 = take(B * Mmax * C * 4);
   L.xs = take(B * Mmax * C * 4);
   L.y = take(B * Mmax * C * 2);
@@ -208,8 +234,11 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, in
   const int tiles_m = (g.R + 127) / 128 * g.nbatch;
   const int bn = gemm_pick_block_n(tiles_m, g.N, ctx->num_sms);
   g.status = ctx->status;
+  ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
+                  2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
+                      (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N * g.nbatch);
   FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->st), what);
-  ctx->launches++;
+  ctx->launched();
   return FVAR_OK;
 }
 
@@ -353,6 +382,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->staged_scale = -1; c->last_scale = -1; c->cache_scale = -1; c->cache_slot = 0; c->null_only_seen = 0;
   c->last_rank.assign(c->G, 0);
   c->last_E = 0; c->last_M = 0;
+  c->loaded_len = -1; c->loaded_cache_scale = -1;
+  c->prof_on = false; c->ev_used = 0;
   *out = c;
   return FVAR_OK;
 }
@@ -362,10 +393,52 @@ fvar_status fvar_reset(fvar_ctx *ctx) {
   std::fill(ctx->len.begin(), ctx->len.end(), 0);
   std::fill(ctx->staged.begin(), ctx->staged.end(), 0);
   ctx->staged_scale = -1; ctx->last_scale = -1; ctx->cache_scale = -1; ctx->null_only_seen = 0;
+  ctx->loaded_len = -1; ctx->loaded_cache_scale = -1;
   return FVAR_OK;
 }
 
-void fvar_destroy(fvar_ctx *ctx) { delete ctx; }
+fvar_status fvar_restore_loaded(fvar_ctx *ctx) {
+  if (!ctx) return FVAR_EINVAL;
+  if (ctx->loaded_len < 0 || ctx->loaded_cache_scale < 0)
+    return fail(ctx, FVAR_ESTATE, "restore_loaded: needs fvar_load_kv and fvar_load_group_cache first");
+  std::fill(ctx->len.begin(), ctx->len.end(), ctx->loaded_len);
+  std::fill(ctx->staged.begin(), ctx->staged.end(), 0);
+  ctx->staged_scale = -1;
+  ctx->last_scale = ctx->loaded_cache_scale;
+  ctx->cache_scale = ctx->loaded_cache_scale;
+  ctx->cache_slot = 2;
+  ctx->null_only_seen = 0;
+  return FVAR_OK;
+}
+
+fvar_status fvar_profile_enable(fvar_ctx *ctx, int on) {
+  if (!ctx) return FVAR_EINVAL;
+  FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  ctx->prof.clear();
+  ctx->ev_used = 0;
+  ctx->prof_on = on != 0;
+  return FVAR_OK;
+}
+
+fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long long *launches, double *flops,
+                              double *bytes) {
+  if (!ctx || !total_ms || !launches || !flops || !bytes) return FVAR_EINVAL;
+  FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  *total_ms = 0; *launches = 0; *flops = 0; *bytes = 0;
+  for (const auto &r : ctx->prof) {
+    if (r.kclass != kclass) continue;
+    float ms = 0.f;
+    FV_CUDA(ctx, cudaEventElapsedTime(&ms, r.e0, r.e1), "event elapsed");
+    *total_ms += ms; *launches += 1; *flops += r.flops; *bytes += r.bytes;
+  }
+  return FVAR_OK;
+}
+
+void fvar_destroy(fvar_ctx *ctx) {
+  if (!ctx) return;
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  delete ctx;
+}
 
 const char *fvar_last_error(const fvar_ctx *ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
 
@@ -401,7 +474,7 @@ fvar_status fvar_set_cond(fvar_ctx *ctx, int B, const void *cond, const void *co
   if (ctx->cfg.has_cross_attn && !context) return fail(ctx, FVAR_EINVAL, "set_cond: context is NULL");
   const int C = ctx->C, nb = ctx->cfg.n_blocks;
   FV_CUDA(ctx, launch_silu_bf16(static_cast<const bf16 *>(cond), ctx->silu_c, static_cast<long long>(B) * C, ctx->st), "silu");
-  ctx->launches++;
+  ctx->launched();
   for (int blk = 0; blk < nb; ++blk) {
     GemmArgs g = gemm_args(B, 6 * C, C);
     g.bias = ctx->b_ada[blk];
@@ -457,10 +530,11 @@ fvar_status fvar_load_kv(fvar_ctx *ctx, const void *K, const void *V, int L) {
     FV_CUDA(ctx, launch_load_kv(static_cast<const bf16 *>(K) + blk * per_blk, static_cast<const bf16 *>(V) + blk * per_blk,
                                 ctx->B, L, ctx->H, ctx->D, ctx->L_cap, ctx->kc + blk * ctx->kv_block_elems(),
                                 ctx->vt + blk * ctx->kv_block_elems(), ctx->st), "load_kv");
-    ctx->launches++;
+    ctx->launched();
     ctx->len[blk] = L;
   }
   ctx->staged_scale = -1;
+  ctx->loaded_len = L;
   return FVAR_OK;
 }
 
@@ -471,10 +545,11 @@ fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cac
   const int M = ctx->Mk[scale_idx];
   const size_t per = static_cast<size_t>(ctx->B) * M * ctx->C;
   for (int g = 0; g < ctx->G; ++g)
-    FV_CUDA(ctx, cudaMemcpyAsync(ctx->gslot(0, g), cache + g * per, per * 4, cudaMemcpyDeviceToDevice, ctx->st), "group cache copy");
+    FV_CUDA(ctx, cudaMemcpyAsync(ctx->gslot(2, g), cache + g * per, per * 4, cudaMemcpyDeviceToDevice, ctx->st), "group cache copy");
   ctx->cache_scale = scale_idx;
-  ctx->cache_slot = 0;
-  if (ctx->last_scale < scale_idx) ctx->last_scale = scale_idx;
+  ctx->cache_slot = 2;
+  ctx->last_scale = scale_idx;
+  ctx->loaded_cache_scale = scale_idx;
   return FVAR_OK;
 }
 
@@ -519,7 +594,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   if (any_late && (ctx->cache_scale < 0 || ctx->cache_scale > scale_idx))
     return fail(ctx, FVAR_ESTATE, "scale_step: low-rank step without the previous scale's group outputs");
 
-  const int prev_slot = ctx->cache_slot, cur_slot = ctx->cache_scale < 0 ? 0 : (ctx->cache_slot ^ 1);
+  const int prev_slot = ctx->cache_slot, cur_slot = (ctx->cache_scale < 0 || ctx->cache_slot == 2) ? 0 : (ctx->cache_slot ^ 1);
   const int h0 = ctx->cache_scale >= 0 ? ctx->hw[2 * ctx->cache_scale] : 0;
   const int w0 = ctx->cache_scale >= 0 ? ctx->hw[2 * ctx->cache_scale + 1] : 0;
   const int h1 = ctx->hw[2 * scale_idx], w1 = ctx->hw[2 * scale_idx + 1];
@@ -527,8 +602,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   const size_t ada_blk = static_cast<size_t>(ctx->Bmax) * 6 * C;
   cudaStream_t st = ctx->st;
 
+  ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * B * M * C);
   FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, B, static_cast<long long>(M) * C, st), "tokens_to_f32");
-  ctx->launches++;
+  ctx->launched();
   const float *X_in = ctx->x0;
   const RowMap bmap{bmul, boff, M};              // buffers indexed by the caller's batch element
   fvar_status s;
@@ -544,26 +620,31 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
 
     if (late) {
       if (pol->forced_indices) {
+        ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * E * (M + 2.0 * r));
         FV_CUDA(ctx, launch_copy_indices(pol->forced_indices + static_cast<size_t>(g) * E * r_max, E, M, r, r_max, idx_g,
                                          inv_g, ctx->status, st), "copy_indices");
-        ctx->launches++;
+        ctx->launched();
       } else {
         if (null_only) {
           for (int e = 0; e < E; ++e) {
+            ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * M * C, 4.0 * M * C + 4.0 * M);
             FV_CUDA(ctx, launch_row_scores(X_in + static_cast<size_t>(e * bmul + boff) * M * C, M, C,
                                            ctx->scores + static_cast<size_t>(e) * M, st), "row_scores");
-            ctx->launches++;
+            ctx->launched();
           }
         } else {
+          ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
           FV_CUDA(ctx, launch_row_scores(X_in, static_cast<long long>(E) * M, C, ctx->scores, st), "row_scores");
-          ctx->launches++;
+          ctx->launched();
         }
+        ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r));
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, st), "select_topr");
-        ctx->launches++;
+        ctx->launched();
       }
       const int Mk = static_cast<int>(align_up(M, 64));
+      ctx->prof_begin(FVAR_KCLASS_TRANSPOSE, 0.0, 4.0 * E * M * C + 4.0 * E * C * Mk);
       FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mk, ctx->xt, st), "transpose");
-      ctx->launches++;
+      ctx->launched();
       // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e; the reduction
       // runs over the hi and lo halves of X
       GemmArgs ga = gemm_args(r, C, Mk + M);
@@ -574,9 +655,10 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       ga.ld_out = C;
       ga.status = ctx->status;
       const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, ctx->num_sms);
+      ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + static_cast<double>(E) * M * C) + 4.0 * E * r * C);
       FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
                                ctx->xt_map[scale_idx * 3 + bn_index(bn)], ga, ctx->num_sms, st), "projection gemm");
-      ctx->launches++;
+      ctx->launched();
     }
 
     for (int t = 0; t < bpg; ++t) {
@@ -587,9 +669,10 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       const float *ada = ctx->ada + blk * ada_blk;
       const int L_prev = ctx->len[blk];
 
+      ctx->prof_begin(FVAR_KCLASS_LN, 0.0, 6.0 * R * C);
       FV_CUDA(ctx, launch_ln_modulate(in_ptr, in_map, E, r, C, ada, ada + C, 6 * C, bmul, boff, nullptr,
                                       ctx->cfg.ln_eps, ctx->y, st), "ln_modulate 1");
-      ctx->launches++;
+      ctx->launched();
       {
         GemmArgs ga = gemm_args(R, 3 * C, C);
         ga.bias = ctx->b_qkv[blk];
@@ -602,8 +685,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       }
       {
         AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * (L_prev + r) * C, 4.0 * E * (L_prev + r) * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
-        ctx->launches++;
+        ctx->launched();
       }
       {
         GemmArgs ga = gemm_args(R, C, C);
@@ -615,23 +699,26 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_O, ga, "out-proj gemm")) != FVAR_OK) return s;
       }
       if (ctx->cfg.has_cross_attn) {
+        ctx->prof_begin(FVAR_KCLASS_LN, 0.0, 6.0 * R * C);
         FV_CUDA(ctx, launch_ln_modulate(ctx->xs, smap, E, r, C, nullptr, nullptr, 0, bmul, boff, ctx->ln_c_gamma[blk],
                                         ctx->cfg.ln_eps, ctx->y, st), "ln cross");
-        ctx->launches++;
+        ctx->launched();
         GemmArgs gq = gemm_args(R, C, C);
         gq.out_bf16 = ctx->q; gq.ld_out = C;
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
         AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
-        ctx->launches++;
+        ctx->launched();
         GemmArgs go = gemm_args(R, C, C);
         go.rows_per_batch = r; go.bmul = bmul; go.boff = boff;
         go.resid = ctx->xs; go.rmap = smap; go.out_f32 = ctx->xs; go.omap = smap; go.ld_out = C;
         if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_CO, go, "cross out gemm")) != FVAR_OK) return s;
       }
+      ctx->prof_begin(FVAR_KCLASS_LN, 0.0, 6.0 * R * C);
       FV_CUDA(ctx, launch_ln_modulate(ctx->xs, smap, E, r, C, ada + 3 * C, ada + 4 * C, 6 * C, bmul, boff, nullptr,
                                       ctx->cfg.ln_eps, ctx->y, st), "ln_modulate 2");
-      ctx->launches++;
+      ctx->launched();
       {
         GemmArgs ga = gemm_args(R, F, C);
         ga.bias = ctx->b_fc1[blk];
@@ -655,14 +742,16 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       ctx->staged[blk] = r;
     }
     if (late) {
+      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M);
       FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, st), "rtr_fill");
-      ctx->launches++;
+      ctx->launched();
     }
     X_in = gout;
     ctx->last_rank[g] = r;
   }
+  ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * E * M * C);
   FV_CUDA(ctx, launch_out_to_bf16(X_in, bmap, E, M, C, static_cast<bf16 *>(out), st), "out_to_bf16");
-  ctx->launches++;
+  ctx->launched();
 
   ctx->cache_scale = scale_idx;
   ctx->cache_slot = cur_slot;
