@@ -211,6 +211,24 @@ fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B,
 fvar_status fvar_rtr_fill(const float *prev, int B, int h0, int w0, int h1, int w1, int C, const int *inv,
                           float *out, void *stream);
 
+/* Row selection for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a packaging variant of fvar_row_scores followed by fvar_select_topr, same results bit for bit).
+ * Who needs it: code that runs inside someone else's memory plan -- an inference server that
+ * reserves all of HBM at start-up, a plugin under another framework's allocator, a real-time loop
+ * where cudaMalloc's implicit synchronisation is not acceptable -- and so has nowhere to put the
+ * [B][M] scores that sit between the two kernels.  Here they live in a fixed fp32 array inside the
+ * library image: FVAR_STATIC_SELECT_MAX_ROWS entries (256 KiB), resident on every GPU that loads
+ * the library until the process exits.  The call allocates and frees nothing.
+ *   x dev fp32 [B][M][C] (C % 4 == 0); idx dev int32 [B][r]; inv dev int32 [B][M]; both written in full.
+ *   B * M > FVAR_STATIC_SELECT_MAX_ROWS -> FVAR_EUNSUPPORTED with a message (use the two-call form).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before starting any stream capture.  All calls on a
+ * device share the one array, which simply keeps the previous call's scores: every entry a call
+ * reads it has just written, so nothing needs clearing -- but two calls whose kernels can overlap
+ * on the GPU (different streams without an ordering between them) race on it; serialise them. */
+#define FVAR_STATIC_SELECT_MAX_ROWS 65536
+fvar_status fvar_select_rows_static(const float *x, int B, int M, int C, int r, int *idx, int *inv, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -90,6 +90,7 @@ def load_library() -> ct.CDLL:
         "fvar_gemm_bf16": (i, [vp, vp, vp, i, i, i, vp, vp]),
         "fvar_attention": (i, [vp, vp, vp, i, i, i, i, i, i, vp, vp]),
         "fvar_rtr_fill": (i, [vp, i, i, i, i, i, i, vp, vp, vp]),
+        "fvar_select_rows_static": (i, [vp, i, i, i, i, vp, vp, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -103,7 +104,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_profile_enable", "fvar_profile_read",
             "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill")
+            "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
 
 def _stream() -> int:
@@ -183,6 +184,16 @@ def fvar_rtr_fill(prev: torch.Tensor, hw_in, hw_out, inv: Optional[torch.Tensor]
     _check_kernel(load_library().fvar_rtr_fill(prev.data_ptr(), B, hw_in[0], hw_in[1], hw_out[0], hw_out[1], C,
                                                _ptr(inv), out.data_ptr(), _stream()))
     return out
+
+
+def fvar_select_rows_static(x: torch.Tensor, r: int, idx: torch.Tensor, inv: torch.Tensor):
+    """Top-r row selection of x fp32 [B][M][C] into caller-provided idx int32 [B][r] and inv int32 [B][M],
+    with the intermediate scores kept in the library's built-in array: nothing is allocated, here or in
+    the library.  For callers whose device memory is fully planned by someone else."""
+    _dev(x, torch.float32), _dev(idx, torch.int32), _dev(inv, torch.int32)
+    B, M, C = x.shape
+    assert idx.shape == (B, r) and inv.shape == (B, M)
+    _check_kernel(load_library().fvar_select_rows_static(x.data_ptr(), B, M, C, r, idx.data_ptr(), inv.data_ptr(), _stream()))
 
 
 def kernel_poll_status() -> int:

@@ -64,6 +64,8 @@ __device__ unsigned g_kernel_status;
 
 static std::string g_init_error;
 
+void set_global_error(const char *msg) { g_init_error = msg ? msg : ""; }
+
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
 static const int kBNs[3] = {64, 128, 256};

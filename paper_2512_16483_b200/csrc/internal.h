@@ -64,6 +64,9 @@ struct AttnArgs {
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                              const AttnArgs &a, cudaStream_t st);
 
+// Records the message fvar_last_error(NULL) returns.
+void set_global_error(const char *msg);
+
 // Memory-bound kernels.
 cudaError_t launch_row_scores(const float *x, long long rows, int C, float *scores, cudaStream_t st);
 cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st);
