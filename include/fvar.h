@@ -146,6 +146,14 @@ fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cac
  * overwrite.  FVAR_ESTATE if nothing was loaded. */
 fvar_status fvar_restore_loaded(fvar_ctx *ctx);
 
+/* Options.  FVAR_OPT_CUDA_GRAPHS (default 1): fvar_scale_step captures the chain of launches between
+ * its input and output conversions into a CUDA graph the first time it sees a combination of scale,
+ * ranks, cache lengths and batch, and replays the graph afterwards (the launches only touch the
+ * workspace).  Instantiating a graph is the one place where the CUDA driver may allocate memory on the
+ * library's behalf.  Steps with forced_indices or with profiling enabled are launched directly. */
+enum { FVAR_OPT_CUDA_GRAPHS = 0 };
+fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value);
+
 /* Measurement aid: while enabled, every kernel launch of this context is bracketed by CUDA events on
  * the context's stream.  fvar_profile_read synchronises and sums, for one kernel class, the event
  * time, the number of launches and the algorithmic flops and bytes (minimum traffic: operands read

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libfvar.so")
 OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
+OPT_CUDA_GRAPHS = 0
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")
@@ -80,6 +81,7 @@ def load_library() -> ct.CDLL:
         "fvar_poll_status": (i, [vp]),
         "fvar_reset": (i, [vp]),
         "fvar_restore_loaded": (i, [vp]),
+        "fvar_set_option": (i, [vp, i, i]),
         "fvar_profile_enable": (i, [vp, i]),
         "fvar_profile_read": (i, [vp, i, P(ct.c_double), P(ll), P(ct.c_double), P(ct.c_double)]),
         "fvar_destroy": (None, [vp]),
@@ -102,7 +104,7 @@ def load_library() -> ct.CDLL:
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
-            "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_profile_enable", "fvar_profile_read",
+            "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read",
             "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
             "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
@@ -341,6 +343,9 @@ class Fvar:
 
     def reset(self):
         self._check(self.lib.fvar_reset(self.ctx))
+
+    def set_option(self, option: int, value: int):
+        self._check(self.lib.fvar_set_option(self.ctx, option, value))
 
     def restore_loaded(self):
         self._check(self.lib.fvar_restore_loaded(self.ctx))

@@ -277,16 +277,27 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 }
 
 template <int D>
+static cudaError_t set_attr() {
+  static bool attr_set = false;
+  if (attr_set) return cudaSuccess;
+  cudaError_t err = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         AttnCfg<D>::kSmemBytes);
+  if (err == cudaSuccess) attr_set = true;
+  return err;
+}
+
+cudaError_t attention_prepare() {
+  cudaError_t e = set_attr<64>();
+  if (e == cudaSuccess) e = set_attr<128>();
+  return e;
+}
+
+template <int D>
 static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const AttnArgs &a,
                             cudaStream_t st) {
   using Cfg = AttnCfg<D>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t err = cudaFuncSetAttribute(attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           Cfg::kSmemBytes);
-    if (err != cudaSuccess) return err;
-    attr_set = true;
-  }
+  cudaError_t err = set_attr<D>();
+  if (err != cudaSuccess) return err;
   dim3 grid((a.r + kQRows - 1) / kQRows, a.H, a.B_eff);
   attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(tmQ, tmK, tmV, a);
   return cudaGetLastError();

@@ -13,16 +13,18 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Row score s_i = sum_c x[i][c]^2: one warp per row, float4 loads.
-__global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict__ x, long long rows, int C,
-                                                         float *__restrict__ scores) {
+// Row score s_i = sum_c x[i][c]^2: one warp per row, float4 loads.  Row (e, i) of the compact
+// score array reads row xmap(e, i) of x.
+__global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict__ x, RowMap xmap, int M,
+                                                         long long rows, int C, float *__restrict__ scores) {
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;
   const int lane = threadIdx.x & 31;
-  const float4 *p = reinterpret_cast<const float4 *>(x + row * C);
+  const int e = static_cast<int>(row / M), i = static_cast<int>(row - static_cast<long long>(e) * M);
+  const float4 *p = reinterpret_cast<const float4 *>(x + (static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb + i) * C);
   float acc = 0.f;
-  for (int i = lane; i < C / 4; i += 32) {
-    float4 v = __ldg(p + i);
+  for (int c = lane; c < C / 4; c += 32) {
+    float4 v = __ldg(p + c);
     acc = fmaf(v.x, v.x, acc);
     acc = fmaf(v.y, v.y, acc);
     acc = fmaf(v.z, v.z, acc);
@@ -32,9 +34,10 @@ __global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict
   if (lane == 0) scores[row] = acc;
 }
 
-cudaError_t launch_row_scores(const float *x, long long rows, int C, float *scores, cudaStream_t st) {
+cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, float *scores, cudaStream_t st) {
+  const long long rows = static_cast<long long>(E) * M;
   if (rows <= 0) return cudaSuccess;
-  row_scores_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(x, rows, C, scores);
+  row_scores_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(x, xmap, M, rows, C, scores);
   return cudaGetLastError();
 }
 
@@ -75,15 +78,33 @@ __global__ void __launch_bounds__(kSelThreads) select_topr_kernel(const float *_
       if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      unsigned acc = 0;
-      int d = 255;
-      for (; d > 0; --d) {
-        if (acc + hist[d] >= need) break;
-        acc += hist[d];
+    if (warp == 0) {
+      // Find the digit d at which the count of keys with a larger digit first reaches `need`:
+      // lane l owns the 8 bins 255 - 8l ... 248 - 8l; a warp scan gives the count above its range.
+      unsigned cnt[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        cnt[j] = hist[255 - 8 * lane - j];
+        tot += cnt[j];
       }
-      s_prefix = prefix | (static_cast<unsigned>(d) << shift);
-      s_need = need - acc;
+      unsigned incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      unsigned acc = incl - tot;
+      if (acc < need && need <= incl) {          // exactly one lane: the matching set holds >= need keys
+        int d = 255 - 8 * lane;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (acc + cnt[j] >= need) break;
+          acc += cnt[j];
+          --d;
+        }
+        s_prefix = prefix | (static_cast<unsigned>(d) << shift);
+        s_need = need - acc;
+      }
     }
     __syncthreads();
     prefix = s_prefix;

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <map>
 
 #include <string>
 #include <vector>
@@ -115,6 +116,14 @@ struct fvar_ctx {
   int loaded_len, loaded_cache_scale;  // state set by fvar_load_kv / fvar_load_group_cache (-1: none)
   // per-launch event timing (fvar_profile_*)
   struct ProfRec { int kclass; double flops, bytes; cudaEvent_t e0, e1; };
+  // CUDA graphs of the step body, keyed by everything that is baked into the launches
+  struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
+  std::map<std::string, GraphEntry> graphs;
+  bool use_graphs;
+  void drop_graphs() {
+    for (auto &kv : graphs) cudaGraphExecDestroy(kv.second.exec);
+    graphs.clear();
+  }
   bool prof_on;
   std::vector<ProfRec> prof;
   std::vector<cudaEvent_t> ev_pool;
@@ -234,7 +243,7 @@ fvar_status cuda_fail(fvar_ctx *ctx, cudaError_t e, const char *what) {
 // out = A W^T (+ epilogue) on the context's stream; picks the tile width from the problem size.
 fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
   const int tiles_m = (g.R + 127) / 128 * g.nbatch;
-  const int bn = gemm_pick_block_n(tiles_m, g.N, ctx->num_sms);
+  const int bn = gemm_pick_block_n(tiles_m, g.N, g.K, ctx->num_sms);
   g.status = ctx->status;
   ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
                   2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
@@ -386,6 +395,9 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->last_E = 0; c->last_M = 0;
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
+  c->use_graphs = true;
+  if (gemm_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
+    return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   *out = c;
   return FVAR_OK;
 }
@@ -411,6 +423,19 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx) {
   ctx->cache_slot = 2;
   ctx->null_only_seen = 0;
   return FVAR_OK;
+}
+
+fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value) {
+  if (!ctx) return FVAR_EINVAL;
+  if (option == FVAR_OPT_CUDA_GRAPHS) {
+    ctx->use_graphs = value != 0;
+    if (!value) {
+      FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+      ctx->drop_graphs();
+    }
+    return FVAR_OK;
+  }
+  return fail(ctx, FVAR_EINVAL, "set_option: unknown option");
 }
 
 fvar_status fvar_profile_enable(fvar_ctx *ctx, int on) {
@@ -439,6 +464,7 @@ fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long 
 void fvar_destroy(fvar_ctx *ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  ctx->drop_graphs();
   delete ctx;
 }
 
@@ -611,6 +637,10 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   const RowMap bmap{bmul, boff, M};              // buffers indexed by the caller's batch element
   fvar_status s;
 
+  // Everything between the input and output conversions touches workspace memory only, so for a
+  // given (scale, ranks, cache lengths, slots) it is the same chain of launches every time: it is
+  // captured into a CUDA graph on first use and replayed afterwards.
+  auto body = [&]() -> fvar_status {
   for (int g = 0; g < G; ++g) {
     const int r = rank[g];
     const bool late = r < M;
@@ -627,18 +657,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
                                          inv_g, ctx->status, st), "copy_indices");
         ctx->launched();
       } else {
-        if (null_only) {
-          for (int e = 0; e < E; ++e) {
-            ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * M * C, 4.0 * M * C + 4.0 * M);
-            FV_CUDA(ctx, launch_row_scores(X_in + static_cast<size_t>(e * bmul + boff) * M * C, M, C,
-                                           ctx->scores + static_cast<size_t>(e) * M, st), "row_scores");
-            ctx->launched();
-          }
-        } else {
-          ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
-          FV_CUDA(ctx, launch_row_scores(X_in, static_cast<long long>(E) * M, C, ctx->scores, st), "row_scores");
-          ctx->launched();
-        }
+        ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
+        FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C, ctx->scores, st), "row_scores");
+        ctx->launched();
         ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r));
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, st), "select_topr");
         ctx->launched();
@@ -656,7 +677,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       ga.out_f32 = ctx->xs;
       ga.ld_out = C;
       ga.status = ctx->status;
-      const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, ctx->num_sms);
+      const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, Mk + M, ctx->num_sms);
       ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + static_cast<double>(E) * M * C) + 4.0 * E * r * C);
       FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
                                ctx->xt_map[scale_idx * 3 + bn_index(bn)], ga, ctx->num_sms, st), "projection gemm");
@@ -751,6 +772,48 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
     X_in = gout;
     ctx->last_rank[g] = r;
   }
+  return FVAR_OK;
+  };
+
+  if (ctx->use_graphs && !ctx->prof_on && !pol->forced_indices) {
+    std::string key;
+    auto put = [&](long long v) { key.append(reinterpret_cast<const char *>(&v), sizeof(v)); };
+    put(scale_idx); put(B); put(E); put(prev_slot); put(cur_slot); put(ctx->cache_scale);
+    for (int g = 0; g < G; ++g) put(rank[g]);
+    for (int blk = 0; blk < ctx->cfg.n_blocks; ++blk) put(ctx->len[blk]);
+    auto it = ctx->graphs.find(key);
+    if (it == ctx->graphs.end()) {
+      if (ctx->graphs.size() >= 256) ctx->drop_graphs();
+      const long long l0 = ctx->launches;
+      FV_CUDA(ctx, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal), "begin capture");
+      s = body();
+      cudaGraph_t graph = nullptr;
+      cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      if (s != FVAR_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return s;
+      }
+      if (ce != cudaSuccess) return cuda_fail(ctx, ce, "end capture");
+      fvar_ctx::GraphEntry ge;
+      ge.kernels = ctx->launches - l0;
+      ctx->launches = l0;
+      ce = cudaGraphInstantiate(&ge.exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (ce != cudaSuccess) return cuda_fail(ctx, ce, "graph instantiate");
+      it = ctx->graphs.emplace(key, ge).first;
+    } else {
+      // host-side bookkeeping the body would have done
+      for (int g = 0; g < G; ++g) {
+        ctx->last_rank[g] = rank[g];
+        for (int blk = g * bpg; blk < (g + 1) * bpg; ++blk) ctx->staged[blk] = rank[g];
+      }
+      X_in = ctx->gslot(cur_slot, G - 1);
+    }
+    FV_CUDA(ctx, cudaGraphLaunch(it->second.exec, st), "graph launch");
+    ctx->launches += it->second.kernels;
+  } else {
+    if ((s = body()) != FVAR_OK) return s;
+  }
   ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * E * M * C);
   FV_CUDA(ctx, launch_out_to_bf16(X_in, bmap, E, M, C, static_cast<bf16 *>(out), st), "out_to_bf16");
   ctx->launched();
@@ -835,7 +898,7 @@ static fvar_status kfail(fvar_status s, const char *m) { g_init_error = m; retur
 
 fvar_status fvar_row_scores(const float *x, int B, int M, int C, float *scores, void *stream) {
   if (!x || !scores || B <= 0 || M <= 0 || C <= 0 || C % 4) return kfail(FVAR_EINVAL, "row_scores: bad arguments");
-  FK_CUDA(launch_row_scores(x, static_cast<long long>(B) * M, C, scores, static_cast<cudaStream_t>(stream)), "row_scores");
+  FK_CUDA(launch_row_scores(x, RowMap{1, 0, M}, B, M, C, scores, static_cast<cudaStream_t>(stream)), "row_scores");
   return FVAR_OK;
 }
 
@@ -860,7 +923,7 @@ fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R
   int dev = 0, sms = 0;
   FK_CUDA(cudaGetDevice(&dev), "get device");
   FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
-  const int bn = gemm_pick_block_n((R + 127) / 128, N, sms);
+  const int bn = gemm_pick_block_n((R + 127) / 128, N, K, sms);
   CUtensorMap ta, tw;
   if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, W, K, N, K, bn)) return kfail(FVAR_EINVAL, "gemm: operands must be 16-byte aligned");
   GemmArgs g = gemm_args(R, N, K);

@@ -5,6 +5,8 @@
 // warps 2-5 drain the other accumulator (tcgen05.ld) and apply the epilogue, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  Every wait is bounded; on expiry the CTA flags the
 // status word, lets its outstanding copies land, frees its TMEM and returns.
+#include <stdlib.h>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -282,30 +284,72 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
-int gemm_pick_block_n(int tiles_m_total, int N, int num_sms) {
-  // Largest tile whose tile count still fills the machine; small problems take narrow tiles so
-  // that more SMs stream the weight matrix.
-  const int cand[3] = {256, 128, 64};
-  for (int i = 0; i < 3; ++i) {
-    const int bn = cand[i];
-    if (N % bn != 0 && i < 2) continue;
-    const long long tiles = static_cast<long long>(tiles_m_total) * ((N + bn - 1) / bn);
-    if (tiles >= 2ll * num_sms || i == 2) return bn;
+// Tuning override: FVAR_GEMM_BLOCK_N=64|128|256 forces the tile width (when it divides the problem).
+static int forced_block_n() {
+  static int v = -1;
+  if (v < 0) {
+    const char *e = getenv("FVAR_GEMM_BLOCK_N");
+    v = e ? atoi(e) : 0;
+    if (v != 64 && v != 128 && v != 256) v = 0;
   }
-  return 64;
+  return v;
+}
+
+int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms) {
+  if (forced_block_n()) return forced_block_n();
+  // Cost model fitted to measurements on B200: an SM takes in about 100 GB/s from L2, so one K step
+  // of a 128 x BN tile (16 KiB of A + BN * 128 B of W) costs t_k microseconds; a wave of tiles costs
+  // num_kb * t_k plus an epilogue that is only hidden behind the next tile of the same CTA.
+  const int cand[3] = {64, 128, 256};
+  const float t_k[3] = {0.31f, 0.36f, 0.47f}, t_epi[3] = {1.0f, 1.5f, 2.5f};
+  const int num_kb = (K + kBlockK - 1) / kBlockK;
+  int best = 64;
+  float best_cost = 1e30f;
+  for (int i = 0; i < 3; ++i) {
+    const long long tiles = static_cast<long long>(tiles_m_total) * ((N + cand[i] - 1) / cand[i]);
+    const long long waves = (tiles + num_sms - 1) / num_sms;
+    const float cost = waves * (num_kb * t_k[i] + t_epi[i]);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = cand[i];
+    }
+  }
+  return best;
+}
+
+template <int BN, int EPI>
+static cudaError_t set_attr() {
+  static bool attr_set = false;
+  if (attr_set) return cudaSuccess;
+  cudaError_t err = cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         GemmCfg<BN>::kSmemBytes);
+  if (err == cudaSuccess) attr_set = true;
+  return err;
+}
+
+template <int BN>
+static cudaError_t set_attr_bn() {
+  cudaError_t e = set_attr<BN, EPI_F32>();
+  if (e == cudaSuccess) e = set_attr<BN, EPI_BF16>();
+  if (e == cudaSuccess) e = set_attr<BN, EPI_GELU_BF16>();
+  if (e == cudaSuccess) e = set_attr<BN, EPI_QKV>();
+  if (e == cudaSuccess) e = set_attr<BN, EPI_RESID>();
+  return e;
+}
+
+cudaError_t gemm_prepare() {
+  cudaError_t e = set_attr_bn<64>();
+  if (e == cudaSuccess) e = set_attr_bn<128>();
+  if (e == cudaSuccess) e = set_attr_bn<256>();
+  return e;
 }
 
 template <int BN, int EPI>
 static cudaError_t launch_one(const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, int num_sms,
                               cudaStream_t st) {
   using Cfg = GemmCfg<BN>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t err = cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           Cfg::kSmemBytes);
-    if (err != cudaSuccess) return err;
-    attr_set = true;
-  }
+  cudaError_t err = set_attr<BN, EPI>();
+  if (err != cudaSuccess) return err;
   const long long tiles = static_cast<long long>((a.R + kBlockM - 1) / kBlockM) * ((a.N + BN - 1) / BN) * a.nbatch;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);

@@ -49,10 +49,14 @@ bool tmap_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uin
 bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1_elems,
              uint64_t ld2_elems, uint32_t box0, uint32_t box1);
 
-int gemm_pick_block_n(int R_total_tiles_m, int N, int num_sms);
+int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms);
 // Launches the tensor-core GEMM.  block_n in {64, 128, 256}: the W map's box must have block_n rows.
 cudaError_t launch_gemm(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
                         int num_sms, cudaStream_t st);
+
+// Set the dynamic shared-memory attribute of every instantiation (once, outside any stream capture).
+cudaError_t gemm_prepare();
+cudaError_t attention_prepare();
 
 struct AttnArgs {
   int B_eff, H, r, D, L, L_cap;
@@ -68,7 +72,7 @@ cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, con
 void set_global_error(const char *msg);
 
 // Memory-bound kernels.
-cudaError_t launch_row_scores(const float *x, long long rows, int C, float *scores, cudaStream_t st);
+cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, float *scores, cudaStream_t st);
 cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st);
 cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_forced, int *idx, int *inv,
                                 unsigned *status, cudaStream_t st);

@@ -264,3 +264,38 @@ def test_state_and_argument_errors(fv):
     p2.gpu.scale_step(t1, 1, mode=fv.LOWRANK_RTR, keep_ratio=0.5, forced_indices=bad)
     assert p2.gpu.poll_status() == fv.EINVAL
     assert p2.gpu.poll_status() == fv.OK                                       # cleared by the read
+
+
+def test_graph_replay_matches_direct_launch(fv):
+    """The step body is captured into a CUDA graph on first use and replayed afterwards; capture,
+    replay and direct launches must give the same bits, and the cache bookkeeping must not differ."""
+    shp = si.shape_var_d16(n_blocks=2)
+    B = 4
+    p = Pair(fv, shp, seed=107, B=B)
+    p.prefill(8)
+    toks = {k: to_bf16_cuda(si.make_tokens(107, B, shp.tokens_per_scale()[k], 1024, "spread")) for k in (8, 9)}
+    for k in (8, 9):
+        p.set_projections(k, [orc.rank_from_keep_ratio(shp.tokens_per_scale()[k], 0.5)] * 2)
+
+    def run():
+        p.gpu.restore_loaded()
+        outs = []
+        for k in (8, 9):
+            outs.append(p.gpu.scale_step(toks[k], k, mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY, keep_ratio=0.5).clone())
+            p.gpu.kv_append(k)
+        p.check_ok()
+        return outs, [p.gpu.cache_len(b) for b in range(2)], p.gpu.get_indices(1, B // 2, 256).clone()
+
+    n0 = p.gpu.launch_count()
+    captured = run()
+    n1 = p.gpu.launch_count()
+    replayed = run()
+    n2 = p.gpu.launch_count()
+    p.gpu.set_option(fv.OPT_CUDA_GRAPHS, 0)
+    direct = run()
+    n3 = p.gpu.launch_count()
+    assert n1 - n0 == n2 - n1 == n3 - n2 > 0
+    for other in (replayed, direct):
+        assert all(torch.equal(a, b) for a, b in zip(captured[0], other[0]))
+        assert captured[1] == other[1] == [255 + 85 + 128] * 2
+        assert torch.equal(captured[2], other[2])
