@@ -86,6 +86,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
   const uint32_t tmem_o = tmem_base + 256;
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -299,8 +301,7 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   cudaError_t err = set_attr<D>();
   if (err != cudaSuccess) return err;
   dim3 grid((a.r + kQRows - 1) / kQRows, a.H, a.B_eff);
-  attention_kernel<D><<<grid, kAttnThreads, Cfg::kSmemBytes, st>>>(tmQ, tmK, tmV, a);
-  return cudaGetLastError();
+  return launch_pdl(attention_kernel<D>, grid, dim3(kAttnThreads), Cfg::kSmemBytes, st, tmQ, tmK, tmV, a);
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,

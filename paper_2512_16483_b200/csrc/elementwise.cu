@@ -17,6 +17,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 // score array reads row xmap(e, i) of x.
 __global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict__ x, RowMap xmap, int M,
                                                          long long rows, int C, float *__restrict__ scores) {
+  pdl_wait();
+  pdl_launch_dependents();
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;
   const int lane = threadIdx.x & 31;
@@ -37,8 +39,7 @@ __global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict
 cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, float *scores, cudaStream_t st) {
   const long long rows = static_cast<long long>(E) * M;
   if (rows <= 0) return cudaSuccess;
-  row_scores_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, st>>>(x, xmap, M, rows, C, scores);
-  return cudaGetLastError();
+  return launch_pdl(row_scores_kernel, dim3(static_cast<unsigned>((rows + 7) / 8)), dim3(256), 0, st, x, xmap, M, rows, C, scores);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -57,6 +58,8 @@ __device__ __forceinline__ unsigned score_key(float s) {
 
 __global__ void __launch_bounds__(kSelThreads) select_topr_kernel(const float *__restrict__ scores, int M, int r,
                                                                   int *__restrict__ idx, int *__restrict__ inv) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ unsigned hist[256];
   __shared__ unsigned s_prefix, s_need;
   __shared__ int warp_gt[32], warp_eq[32];
@@ -165,14 +168,15 @@ __global__ void __launch_bounds__(kSelThreads) select_topr_kernel(const float *_
 
 cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st) {
   if (B <= 0) return cudaSuccess;
-  select_topr_kernel<<<B, kSelThreads, 0, st>>>(scores, M, r, idx, inv);
-  return cudaGetLastError();
+  return launch_pdl(select_topr_kernel, dim3(B), dim3(kSelThreads), 0, st, scores, M, r, idx, inv);
 }
 
 // Test hook: take the caller's index lists instead of selecting.  Checks range and strict ascent;
 // a bad list sets a status bit and the offending entry is clamped into range.
 __global__ void copy_indices_kernel(const int *__restrict__ forced, int M, int r, int ld_forced,
                                     int *__restrict__ idx, int *__restrict__ inv, unsigned *status) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.x;
   const int *f = forced + static_cast<long long>(b) * ld_forced;
   int *idx_b = idx + static_cast<long long>(b) * r;
@@ -191,8 +195,7 @@ __global__ void copy_indices_kernel(const int *__restrict__ forced, int M, int r
 
 cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_forced, int *idx, int *inv,
                                 unsigned *status, cudaStream_t st) {
-  copy_indices_kernel<<<B, 256, 0, st>>>(forced, M, r, ld_forced, idx, inv, status);
-  return cudaGetLastError();
+  return launch_pdl(copy_indices_kernel, dim3(B), dim3(256), 0, st, forced, M, r, ld_forced, idx, inv, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -207,6 +210,8 @@ __global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__
                                                                  long long vec_stride, int bmul, int boff,
                                                                  const bf16 *__restrict__ gamma, float eps,
                                                                  bf16 *__restrict__ y) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float red[kLnThreads / 32];
   const int e = blockIdx.x / rows, j = blockIdx.x - e * rows;
   const float *xr = x + (static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb + j) * C;
@@ -289,9 +294,8 @@ cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int
                                float eps, bf16 *y, cudaStream_t st) {
   if (E * rows <= 0) return cudaSuccess;
   if (C % 8 != 0 || C > 8 * kLnThreads * kLnMaxVec) return cudaErrorInvalidValue;
-  ln_modulate_kernel<<<E * rows, kLnThreads, 0, st>>>(x, xmap, rows, C, shift, scale, vec_stride, bmul, boff, gamma,
+  return launch_pdl(ln_modulate_kernel, dim3(E * rows), dim3(kLnThreads), 0, st, x, xmap, rows, C, shift, scale, vec_stride, bmul, boff, gamma,
                                                       eps, y);
-  return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -301,6 +305,8 @@ cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int
 __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__ prev, float *__restrict__ out, int E,
                                                        int bmul, int boff, int h0, int w0, int h1, int w1, int C,
                                                        const int *__restrict__ inv) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int M1 = h1 * w1;
   const long long gw = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
   if (gw >= static_cast<long long>(E) * M1) return;
@@ -335,9 +341,8 @@ cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int 
                             int C, const int *inv, cudaStream_t st) {
   const long long warps = static_cast<long long>(E) * h1 * w1;
   if (warps <= 0) return cudaSuccess;
-  rtr_fill_kernel<<<static_cast<unsigned>((warps + 7) / 8), 256, 0, st>>>(prev, out, E, bmul, boff, h0, w0, h1, w1, C,
+  return launch_pdl(rtr_fill_kernel, dim3(static_cast<unsigned>((warps + 7) / 8)), dim3(256), 0, st, prev, out, E, bmul, boff, h0, w0, h1, w1, C,
                                                                          inv);
-  return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -348,6 +353,8 @@ cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int 
 // through shared memory.
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
                                                              int Mk, bf16 *__restrict__ xt) {
+  pdl_wait();
+  pdl_launch_dependents();
   __shared__ float tile[32][33];
   const int e = blockIdx.z, m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
@@ -373,12 +380,13 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__rest
 cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
                                   cudaStream_t st) {
   dim3 grid((Mk + 31) / 32, (C + 31) / 32, E);
-  transpose_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, Mk, xt);
-  return cudaGetLastError();
+  return launch_pdl(transpose_bf16_kernel, dim3(grid), dim3(256), 0, st, x, xmap, M, C, Mk, xt);
 }
 
 // ------------------------------------------------------------------------------------------------
 __global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__restrict__ x, long long n8) {
+  pdl_wait();
+  pdl_launch_dependents();
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n8) return;
   const uint4 u = __ldg(reinterpret_cast<const uint4 *>(tok) + i);
@@ -392,11 +400,12 @@ __global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__rest
 cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st) {
   const long long n8 = static_cast<long long>(B) * per_elem / 8;
   if (n8 <= 0) return cudaSuccess;
-  tokens_to_f32_kernel<<<static_cast<unsigned>((n8 + 255) / 256), 256, 0, st>>>(tok, x, n8);
-  return cudaGetLastError();
+  return launch_pdl(tokens_to_f32_kernel, dim3(static_cast<unsigned>((n8 + 255) / 256)), dim3(256), 0, st, tok, x, n8);
 }
 
 __global__ void out_to_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C, bf16 *__restrict__ out) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int e = blockIdx.y;
   const long long per = static_cast<long long>(M) * C / 8;
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -413,11 +422,12 @@ __global__ void out_to_bf16_kernel(const float *__restrict__ x, RowMap xmap, int
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st) {
   const long long per = static_cast<long long>(M) * C / 8;
   dim3 grid(static_cast<unsigned>((per + 255) / 256), E);
-  out_to_bf16_kernel<<<grid, 256, 0, st>>>(x, xmap, M, C, out);
-  return cudaGetLastError();
+  return launch_pdl(out_to_bf16_kernel, dim3(grid), dim3(256), 0, st, x, xmap, M, C, out);
 }
 
 __global__ void silu_bf16_kernel(const bf16 *__restrict__ in, bf16 *__restrict__ out, long long n) {
+  pdl_wait();
+  pdl_launch_dependents();
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const float v = __bfloat162float(in[i]);
@@ -426,13 +436,14 @@ __global__ void silu_bf16_kernel(const bf16 *__restrict__ in, bf16 *__restrict__
 
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
-  silu_bf16_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(in, out, n);
-  return cudaGetLastError();
+  return launch_pdl(silu_bf16_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, in, out, n);
 }
 
 // K, V [B][L][H*D] -> cache layout K [B][H][L_cap][D], V^T [B][H][D][L_cap] (one block's worth).
 __global__ void load_kv_kernel(const bf16 *__restrict__ K, const bf16 *__restrict__ V, int L, int H, int D, int L_cap,
                                bf16 *__restrict__ kc, bf16 *__restrict__ vt) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int b = blockIdx.z, h = blockIdx.y;
   const int C = H * D;
   for (long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; t < static_cast<long long>(L) * D;
@@ -448,8 +459,7 @@ cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, in
                            cudaStream_t st) {
   if (L <= 0) return cudaSuccess;
   dim3 grid(static_cast<unsigned>((static_cast<long long>(L) * D + 255) / 256), H, B);
-  load_kv_kernel<<<grid, 256, 0, st>>>(K, V, L, H, D, L_cap, kc, vt);
-  return cudaGetLastError();
+  return launch_pdl(load_kv_kernel, dim3(grid), dim3(256), 0, st, K, V, L, H, D, L_cap, kc, vt);
 }
 
 }  // namespace fvar

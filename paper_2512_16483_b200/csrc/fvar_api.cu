@@ -2,6 +2,7 @@
 // scale step over block groups.  See include/fvar.h for the contract of every entry point.
 #include <stdio.h>
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -65,6 +66,15 @@ __device__ unsigned g_kernel_status;
 
 static std::string g_init_error;
 
+bool pdl_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char *e = getenv("FVAR_NO_PDL");
+    v = (e && e[0] == '1') ? 0 : 1;
+  }
+  return v != 0;
+}
+
 void set_global_error(const char *msg) { g_init_error = msg ? msg : ""; }
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -82,7 +92,9 @@ struct fvar_ctx {
   std::vector<int> hw;                 // 2 * n_scales
   std::vector<int> Mk;                 // tokens per scale
   int G, C, F, H, D, Bmax, Mmax, L_cap, ctx_cap, num_sms;
-  cudaStream_t st;
+  cudaStream_t st;         // the caller's stream
+  cudaStream_t launch_st;  // where launches go: st, or cap_st while a graph is being captured
+  cudaStream_t cap_st;     // private stream used only for capture (the legacy default stream cannot be captured)
   std::string err;
   long long launches;
   // weights (device pointers per block)
@@ -248,7 +260,7 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, in
   ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
                   2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
                       (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N * g.nbatch);
-  FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->st), what);
+  FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->launch_st), what);
   ctx->launched();
   return FVAR_OK;
 }
@@ -311,6 +323,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->ctx_cap = cfg->has_cross_attn ? static_cast<int>(align_up(cfg->ctx_len, 128)) : 0;
   c->num_sms = prop.multiProcessorCount;
   c->st = static_cast<cudaStream_t>(cuda_stream);
+  c->launch_st = c->st;
+  c->cap_st = nullptr;
   c->launches = 0;
   c->ws = static_cast<uint8_t *>(workspace);
   c->ws_bytes = bytes;
@@ -395,7 +409,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->last_E = 0; c->last_M = 0;
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
-  c->use_graphs = true;
+  c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess;
   if (gemm_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   *out = c;
@@ -465,6 +479,7 @@ void fvar_destroy(fvar_ctx *ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   ctx->drop_graphs();
+  if (ctx->cap_st) cudaStreamDestroy(ctx->cap_st);
   delete ctx;
 }
 
@@ -785,10 +800,12 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
     if (it == ctx->graphs.end()) {
       if (ctx->graphs.size() >= 256) ctx->drop_graphs();
       const long long l0 = ctx->launches;
-      FV_CUDA(ctx, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal), "begin capture");
+      FV_CUDA(ctx, cudaStreamBeginCapture(ctx->cap_st, cudaStreamCaptureModeThreadLocal), "begin capture");
+      st = ctx->launch_st = ctx->cap_st;
       s = body();
+      st = ctx->launch_st = ctx->st;
       cudaGraph_t graph = nullptr;
-      cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      cudaError_t ce = cudaStreamEndCapture(ctx->cap_st, &graph);
       if (s != FVAR_OK) {
         if (graph) cudaGraphDestroy(graph);
         return s;

@@ -185,6 +185,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -353,8 +355,7 @@ static cudaError_t launch_one(const CUtensorMap &tmA, const CUtensorMap &tmW, co
   const long long tiles = static_cast<long long>((a.R + kBlockM - 1) / kBlockM) * ((a.N + BN - 1) / BN) * a.nbatch;
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
-  gemm_kernel<BN, EPI><<<grid, kGemmThreads, Cfg::kSmemBytes, st>>>(tmA, tmW, a);
-  return cudaGetLastError();
+  return launch_pdl(gemm_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), Cfg::kSmemBytes, st, tmA, tmW, a);
 }
 
 template <int BN>

@@ -27,6 +27,17 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// ------------------------------------------------------------------------------------ dependent launch
+// Every kernel of the library is launched with programmatic stream serialization: its CTAs may be
+// scheduled while the previous kernel on the stream is still draining, so that launch latency and
+// the prologue (barrier init, TMEM allocation, descriptor prefetch) overlap the predecessor's tail.
+// pdl_wait() blocks until the predecessor grid has completed and its writes are visible; nothing
+// that reads or overwrites global memory may precede it.  pdl_launch_dependents() then lets the
+// successor begin its own prologue.  Because every kernel waits before it releases its successor,
+// at most two grids are in flight and completion order is transitive along the stream.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
