@@ -95,6 +95,8 @@ struct fvar_ctx {
   cudaStream_t st;         // the caller's stream
   cudaStream_t launch_st;  // where launches go: st, or cap_st while a graph is being captured
   cudaStream_t cap_st;     // private stream used only for capture (the legacy default stream cannot be captured)
+  cudaStream_t cap_st2;    // second capture stream: the selection / fill branch of a late group runs beside the blocks
+  cudaEvent_t ev_fork, ev_join;
   std::string err;
   long long launches;
   // weights (device pointers per block)
@@ -325,6 +327,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->st = static_cast<cudaStream_t>(cuda_stream);
   c->launch_st = c->st;
   c->cap_st = nullptr;
+  c->cap_st2 = nullptr;
+  c->ev_fork = c->ev_join = nullptr;
   c->launches = 0;
   c->ws = static_cast<uint8_t *>(workspace);
   c->ws_bytes = bytes;
@@ -409,7 +413,10 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->last_E = 0; c->last_M = 0;
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
-  c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess;
+  c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
   if (gemm_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   *out = c;
@@ -480,6 +487,9 @@ void fvar_destroy(fvar_ctx *ctx) {
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   ctx->drop_graphs();
   if (ctx->cap_st) cudaStreamDestroy(ctx->cap_st);
+  if (ctx->cap_st2) cudaStreamDestroy(ctx->cap_st2);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   delete ctx;
 }
 
@@ -665,20 +675,35 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
     int *inv_g = ctx->inv + static_cast<size_t>(g) * ctx->Bmax * ctx->Mmax;
     const RowMap smap{1, 0, r};                  // the compact work stream of this group
 
+    // While a graph is being captured, the index selection and the restoration fill of a late group
+    // go to a second stream: they depend only on the group's input and on the previous scale's
+    // cache, so they run beside the projection and the blocks and join before the scatter.
+    const bool forked = late && st == ctx->cap_st;
     if (late) {
+      cudaStream_t side = st;
+      if (forked) {
+        FV_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st), "fork record");
+        FV_CUDA(ctx, cudaStreamWaitEvent(ctx->cap_st2, ctx->ev_fork, 0), "fork wait");
+        side = ctx->cap_st2;
+      }
       if (pol->forced_indices) {
         ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * E * (M + 2.0 * r));
         FV_CUDA(ctx, launch_copy_indices(pol->forced_indices + static_cast<size_t>(g) * E * r_max, E, M, r, r_max, idx_g,
-                                         inv_g, ctx->status, st), "copy_indices");
+                                         inv_g, ctx->status, side), "copy_indices");
         ctx->launched();
       } else {
         ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
-        FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C, ctx->scores, st), "row_scores");
+        FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C, ctx->scores, side), "row_scores");
         ctx->launched();
         ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r));
-        FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, st), "select_topr");
+        FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, side), "select_topr");
         ctx->launched();
       }
+      // restoration fill: rows outside the index set, from the upsampled cache of the previous scale
+      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M);
+      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, side), "rtr_fill");
+      ctx->launched();
+      if (forked) FV_CUDA(ctx, cudaEventRecord(ctx->ev_join, side), "join record");
       const int Mk = static_cast<int>(align_up(M, 64));
       ctx->prof_begin(FVAR_KCLASS_TRANSPOSE, 0.0, 4.0 * E * M * C + 4.0 * E * C * Mk);
       FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mk, ctx->xt, st), "transpose");
@@ -770,6 +795,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         ga.resid = ctx->xs; ga.rmap = smap; ga.ld_out = C;
         ga.gate = ada + 5 * C; ga.gate_stride = 6 * C;
         if (last) {
+          if (forked) FV_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0), "join wait");
           ga.out_f32 = gout; ga.omap = bmap;
           ga.scatter = late ? idx_g : nullptr;
         } else {
@@ -778,11 +804,6 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         if ((s = run_gemm(ctx, EPI_RESID, ctx->h_map, blk, W_FC2, ga, "fc2 gemm")) != FVAR_OK) return s;
       }
       ctx->staged[blk] = r;
-    }
-    if (late) {
-      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M);
-      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, st), "rtr_fill");
-      ctx->launched();
     }
     X_in = gout;
     ctx->last_rank[g] = r;
