@@ -147,6 +147,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d16_late3_b16", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="for runs under ncu: skip the host-buffer leg, the event pass and the CPU baseline")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
@@ -258,12 +260,12 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     ms_total, launches = timed(step_device, args.steps, warm)
     clocks = sampler.stop() if sampler else None
-    ms_e2e, _ = timed(step_host, args.steps, 2)
+    ms_e2e, _ = (ms_total, 0) if args.profile_run else timed(step_host, args.steps, 2)
     assert ctx.poll_status() == fv.OK, "device status word reports an error"
 
     # per-kernel-class event timing: a separate pass over the same steps, events around every launch
     ctx.profile_enable(True)
-    prof_steps = max(1, min(args.steps, 10))
+    prof_steps = 0 if args.profile_run else max(1, min(args.steps, 10))
     for _ in range(prof_steps):
         step_device()
     classes = {}
@@ -300,7 +302,7 @@ def main():
                 "d2h_bytes_per_step": sum(E * Ms[k] * shp.width * 2 for k in late_scales)},
         "roofline": roofline,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not args.profile_run:
         tps, dt, desc, threads = oracle_leg(wl, 1, 0)
         line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc,
                                 "seconds": dt}

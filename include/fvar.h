@@ -150,8 +150,11 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx);
  * its input and output conversions into a CUDA graph the first time it sees a combination of scale,
  * ranks, cache lengths and batch, and replays the graph afterwards (the launches only touch the
  * workspace).  Instantiating a graph is the one place where the CUDA driver may allocate memory on the
- * library's behalf.  Steps with forced_indices or with profiling enabled are launched directly. */
-enum { FVAR_OPT_CUDA_GRAPHS = 0 };
+ * library's behalf.  Steps with forced_indices or with profiling enabled are launched directly.
+ * FVAR_OPT_GEMM_MAX_SPLITS (default 1; 1, 2 or 4): largest split-K factor the GEMM tile picker may use.
+ * Partial tiles go through a scratch area of the workspace and are added in a fixed order, so results do
+ * not depend on timing.  On the measured workloads splitting did not pay, hence the default. */
+enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1 };
 fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value);
 
 /* Measurement aid: while enabled, every kernel launch of this context is bracketed by CUDA events on

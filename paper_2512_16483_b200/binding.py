@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libfvar.so")
 OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
-OPT_CUDA_GRAPHS = 0
+OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS = 0, 1
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")

@@ -80,6 +80,8 @@ void set_global_error(const char *msg) { g_init_error = msg ? msg : ""; }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
 static const int kBNs[3] = {64, 128, 256};
+constexpr size_t kSplitScratchBytes = 64u << 20;   // split-K partial tiles
+constexpr size_t kSplitCounters = 4096;            // one arrival counter per tile
 
 enum WeightId { W_QKV = 0, W_O, W_FC1, W_FC2, W_ADA, W_CQ, W_CKV, W_CO, W_COUNT };
 
@@ -108,8 +110,8 @@ struct fvar_ctx {
   size_t ws_bytes;
   unsigned *status;
   bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *xt, *qt_pool;
-  float *ada, *gcache, *x0, *xs, *scores;
-  int *idx, *inv;
+  float *ada, *gcache, *x0, *xs, *scores, *split_partial;
+  int *idx, *inv, *split_counters;
   std::vector<size_t> qt_off;          // [scale][group] offset (elements) into qt_pool
   std::vector<int> qt_r;               // [scale][group] rank of the stored projection (0: none)
   std::vector<CUtensorMap> qt_map;     // [scale][group]
@@ -134,6 +136,7 @@ struct fvar_ctx {
   struct GraphEntry { cudaGraphExec_t exec; long long kernels; };
   std::map<std::string, GraphEntry> graphs;
   bool use_graphs;
+  int max_splits;                      // largest split-K factor the tile picker may use (1, 2 or 4)
   void drop_graphs() {
     for (auto &kv : graphs) cudaGraphExecDestroy(kv.second.exec);
     graphs.clear();
@@ -173,7 +176,7 @@ struct fvar_ctx {
 namespace {
 
 struct Layout {
-  size_t status, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
+  size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
   std::vector<size_t> qt_off;
 };
 
@@ -207,6 +210,8 @@ Layout make_layout(const fvar_cfg *c) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; };
   L.status = take(256);
+  L.split_partial = take(kSplitScratchBytes);
+  L.split_counters = take(kSplitCounters * 4);
   L.kc = take(nb * B * L_cap * C * 2);
   L.vt = take(nb * B * L_cap * C * 2);
   L.ckc = take(nb * B * ctx_cap * C * 2);
@@ -257,7 +262,11 @@ fvar_status cuda_fail(fvar_ctx *ctx, cudaError_t e, const char *what) {
 // out = A W^T (+ epilogue) on the context's stream; picks the tile width from the problem size.
 fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
   const int tiles_m = (g.R + 127) / 128 * g.nbatch;
-  const int bn = gemm_pick_block_n(tiles_m, g.N, g.K, ctx->num_sms);
+  int bn = 64, sp = 1;
+  gemm_pick_tile(tiles_m, g.N, g.K, ctx->num_sms, ctx->max_splits, kSplitScratchBytes, &bn, &sp);
+  g.splits = sp;
+  g.partial = ctx->split_partial;
+  g.counters = ctx->split_counters;
   g.status = ctx->status;
   ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
                   2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
@@ -334,6 +343,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->ws_bytes = bytes;
   auto at = [&](size_t off) { return c->ws + off; };
   c->status = reinterpret_cast<unsigned *>(at(L.status));
+  c->split_partial = reinterpret_cast<float *>(at(L.split_partial));
+  c->split_counters = reinterpret_cast<int *>(at(L.split_counters));
   c->kc = reinterpret_cast<bf16 *>(at(L.kc)); c->vt = reinterpret_cast<bf16 *>(at(L.vt));
   c->ckc = reinterpret_cast<bf16 *>(at(L.ckc)); c->cvt = reinterpret_cast<bf16 *>(at(L.cvt));
   c->ada = reinterpret_cast<float *>(at(L.ada)); c->silu_c = reinterpret_cast<bf16 *>(at(L.silu_c));
@@ -413,6 +424,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->last_E = 0; c->last_M = 0;
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
+  c->max_splits = 1;
   c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
@@ -454,6 +466,13 @@ fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value) {
       FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
       ctx->drop_graphs();
     }
+    return FVAR_OK;
+  }
+  if (option == FVAR_OPT_GEMM_MAX_SPLITS) {
+    if (value != 1 && value != 2 && value != 4) return fail(ctx, FVAR_EINVAL, "set_option: max splits must be 1, 2 or 4");
+    FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+    ctx->drop_graphs();
+    ctx->max_splits = value;
     return FVAR_OK;
   }
   return fail(ctx, FVAR_EINVAL, "set_option: unknown option");

@@ -148,6 +148,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t tmem_base_holder;
   __shared__ volatile int abort_flag;
+  __shared__ volatile int split_last;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bar_base = smem_base + S * Cfg::kStageBytes;
@@ -160,8 +161,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   const int tiles_m = (p.R + kBlockM - 1) / kBlockM;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int tiles_per_batch = tiles_m * tiles_n;
-  const int total_tiles = tiles_per_batch * p.nbatch;
+  const int splits = p.splits > 1 ? p.splits : 1;      // split-K: each work item covers a K range of one tile
+  const int total_tiles = tiles_per_batch * p.nbatch * splits;
   const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+  const int kb_per_split = (num_kb + splits - 1) / splits;
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -196,12 +199,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t armed = 0;                      // bit s set: stage s has been armed at least once
       uint32_t last_parity = 0;                // bit s: parity of the phase last armed on stage s
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+      for (int work = blockIdx.x; ok && work < total_tiles; work += gridDim.x) {
+        const int tile = work / splits, sp = work - tile * splits;
         const int e = tile / tiles_per_batch, rem = tile - e * tiles_per_batch;
         const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
         const int row_a = e * p.a_batch_rows + m_idx * kBlockM;
         const int row_w = e * p.b_batch_rows + n_idx * BN;
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), Cfg::kStageBytes);
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
@@ -229,20 +234,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+      for (int work = blockIdx.x; ok && work < total_tiles; work += gridDim.x, ++it) {
+        const int sp = work % splits;
+        const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         const int a = it & 1;
         const uint32_t aphase = (it >> 1) & 1u;
         if (!mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, p.status, &abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
           const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + Cfg::kStageBytesA);
 #pragma unroll
           for (int k = 0; k < kBlockK / 16; ++k)
-            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb > kb0) || (k != 0));
           umma_commit(empty_bar(stage));
           if (++stage == S) { stage = 0; phase ^= 1u; }
         }
@@ -254,7 +261,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int quad = warp & 3;                 // TMEM lanes [32 * quad, 32 * quad + 32)
     int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++it) {
+    for (int work = blockIdx.x; ok && work < total_tiles; work += gridDim.x, ++it) {
+      const int tile = work / splits, sp = work - tile * splits;
       const int e = tile / tiles_per_batch, rem = tile - e * tiles_per_batch;
       const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
       const int a = it & 1;
@@ -262,19 +270,69 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag));
       if (!ok) break;
       tc_fence_after();
-      const int row = m_idx * kBlockM + quad * 32 + lane;
+      const int row_local = quad * 32 + lane;
+      const int row = m_idx * kBlockM + row_local;
       const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
+      if (splits == 1) {
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = n_idx * BN + c * 32;
-        if (col0 >= p.N) break;                // uniform across the warp
-        uint32_t acc[32];
-        tmem_ld32(taddr + c * 32, acc);
-        tmem_ld_wait();
-        if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0);
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col0 = n_idx * BN + c * 32;
+          if (col0 >= p.N) break;                // uniform across the warp
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+          if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0);
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(a));
+      } else {
+        // Split-K: park this K range's partial tile in the scratch area; the CTA that finishes a
+        // tile last adds the partials in split order (so the sum does not depend on timing) and
+        // applies the epilogue.
+        float *mine = p.partial + (static_cast<size_t>(tile) * splits + sp) * (kBlockM * BN) + row_local * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            __stcg(reinterpret_cast<float4 *>(mine + c * 32) + q,
+                   make_float4(__uint_as_float(acc[q * 4]), __uint_as_float(acc[q * 4 + 1]),
+                               __uint_as_float(acc[q * 4 + 2]), __uint_as_float(acc[q * 4 + 3])));
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(a));
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64) split_last = (atomicAdd(p.counters + tile, 1) == splits - 1) ? 1 : 0;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (split_last) {
+          __threadfence();
+          const float *base = p.partial + static_cast<size_t>(tile) * splits * (kBlockM * BN) + row_local * BN;
+#pragma unroll 1
+          for (int c = 0; c < BN / 32; ++c) {
+            const int col0 = n_idx * BN + c * 32;
+            if (col0 >= p.N) break;
+            float sum[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum[i] = 0.f;
+            for (int s2 = 0; s2 < splits; ++s2) {
+              const float4 *src = reinterpret_cast<const float4 *>(base + static_cast<size_t>(s2) * (kBlockM * BN) + c * 32);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                const float4 v = __ldcg(src + q);
+                sum[q * 4] += v.x; sum[q * 4 + 1] += v.y; sum[q * 4 + 2] += v.z; sum[q * 4 + 3] += v.w;
+              }
+            }
+            uint32_t acc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(sum[i]);
+            if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0);
+          }
+          if (threadIdx.x == 64) p.counters[tile] = 0;      // ready for the next launch
+        }
       }
-      tc_fence_before();
-      mbar_arrive(tempty_bar(a));
     }
   }
 
@@ -297,26 +355,42 @@ static int forced_block_n() {
   return v;
 }
 
-int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms) {
-  if (forced_block_n()) return forced_block_n();
-  // Cost model fitted to measurements on B200: an SM takes in about 100 GB/s from L2, so one K step
-  // of a 128 x BN tile (16 KiB of A + BN * 128 B of W) costs t_k microseconds; a wave of tiles costs
-  // num_kb * t_k plus an epilogue that is only hidden behind the next tile of the same CTA.
+// Cost model fitted to measurements on B200: an SM takes in about 100 GB/s from L2, so one K step
+// of a 128 x BN tile (16 KiB of A + BN * 128 B of W) costs t_k microseconds; a wave of work items
+// costs its K steps plus an epilogue that is only hidden behind the next item of the same CTA.
+// Splitting K trades a reduction through the scratch area for more CTAs streaming the operands.
+void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits, size_t scratch_bytes, int *block_n,
+                    int *splits) {
   const int cand[3] = {64, 128, 256};
   const float t_k[3] = {0.31f, 0.36f, 0.47f}, t_epi[3] = {1.0f, 1.5f, 2.5f};
   const int num_kb = (K + kBlockK - 1) / kBlockK;
-  int best = 64;
   float best_cost = 1e30f;
+  *block_n = 64;
+  *splits = 1;
   for (int i = 0; i < 3; ++i) {
+    if (forced_block_n() && cand[i] != forced_block_n()) continue;
     const long long tiles = static_cast<long long>(tiles_m_total) * ((N + cand[i] - 1) / cand[i]);
-    const long long waves = (tiles + num_sms - 1) / num_sms;
-    const float cost = waves * (num_kb * t_k[i] + t_epi[i]);
-    if (cost < best_cost) {
-      best_cost = cost;
-      best = cand[i];
+    for (int sp = 1; sp <= max_splits; sp *= 2) {
+      if (sp > 1 && (num_kb / sp < 8 || tiles > 4096 ||
+                     static_cast<size_t>(tiles) * sp * kBlockM * cand[i] * 4 > scratch_bytes))
+        break;
+      const long long waves = (tiles * sp + num_sms - 1) / num_sms;
+      const int kb = (num_kb + sp - 1) / sp;
+      float cost = waves * (kb * t_k[i] + t_epi[i]);
+      if (sp > 1) cost += 1.5f + 0.6f * sp * cand[i] / 128.0f;      // park + fixed-order reduction by one CTA
+      if (cost < best_cost) {
+        best_cost = cost;
+        *block_n = cand[i];
+        *splits = sp;
+      }
     }
   }
-  return best;
+}
+
+int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms) {
+  int bn, sp;
+  gemm_pick_tile(tiles_m_total, N, K, num_sms, 1, 0, &bn, &sp);
+  return bn;
 }
 
 template <int BN, int EPI>
@@ -352,7 +426,8 @@ static cudaError_t launch_one(const CUtensorMap &tmA, const CUtensorMap &tmW, co
   using Cfg = GemmCfg<BN>;
   cudaError_t err = set_attr<BN, EPI>();
   if (err != cudaSuccess) return err;
-  const long long tiles = static_cast<long long>((a.R + kBlockM - 1) / kBlockM) * ((a.N + BN - 1) / BN) * a.nbatch;
+  const long long tiles = static_cast<long long>((a.R + kBlockM - 1) / kBlockM) * ((a.N + BN - 1) / BN) * a.nbatch *
+                          (a.splits > 1 ? a.splits : 1);
   if (tiles <= 0) return cudaSuccess;
   const int grid = static_cast<int>(tiles < num_sms ? tiles : num_sms);
   return launch_pdl(gemm_kernel<BN, EPI>, dim3(grid), dim3(kGemmThreads), Cfg::kSmemBytes, st, tmA, tmW, a);

@@ -39,6 +39,10 @@ struct GemmArgs {
   // EPI_QKV: virtual column = col + col_base; [0,C) -> q, [C,2C) -> K cache, [2C,3C) -> transposed V cache
   bf16 *kc, *vt;
   int C, H, D, L_cap, L_prev, col_base;
+  // split-K (splits > 1): fp32 partial tiles [tile][split][128][BN] and one arrival counter per tile
+  int splits;
+  float *partial;
+  int *counters;
   unsigned *status;
 };
 
@@ -50,6 +54,8 @@ bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_
              uint64_t ld2_elems, uint32_t box0, uint32_t box1);
 
 int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms);
+void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits, size_t scratch_bytes, int *block_n,
+                    int *splits);
 // Launches the tensor-core GEMM.  block_n in {64, 128, 256}: the W map's box must have block_n rows.
 cudaError_t launch_gemm(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
                         int num_sms, cudaStream_t st);
