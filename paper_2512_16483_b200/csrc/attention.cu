@@ -1,12 +1,14 @@
 // Flash-style attention of one scale's query rows over the multi-scale KV cache, sm_100a.
 //
-// One CTA handles 128 query rows of one (batch element, head).  Warp 0 streams K / V^T tiles of
-// 128 keys with TMA; warp 1 issues S = Q K^T and O_j = P V on the tensor cores (accumulators in
-// TMEM); warps 2-5 own one query row per thread: they read S from TMEM, keep the running max and
-// sum, write P (bf16) into a swizzled shared-memory tile for the second MMA, and fold each O_j
-// into a register accumulator with the usual rescaling.  S is double-buffered so that Q K^T of
-// block j+1 overlaps the softmax of block j.  Keys at or beyond L are masked.  Every wait is
-// bounded (see ptx.cuh).
+// One CTA handles up to 256 query rows (two tiles of 128) of one (batch element, head).
+//   warp 0      streams K and V^T tiles of 128 keys through a ring of shared-memory slots (TMA);
+//   warp 1      issues S_t = Q_t K^T and O_t += P_t V on the tensor cores, accumulators in TMEM;
+//   warps 2-5   softmax of tile 0, one query row per thread;   warps 6-9: softmax of tile 1.
+// The two tiles run out of phase: while one warp-group turns S into P (row max, exp2, bf16 P into
+// a swizzled shared tile), the tensor core works for the other tile (P V of block j, then Q K^T
+// of block j+1).  O stays in TMEM for the whole key loop; its rows are rescaled only when the
+// running maximum has grown by more than 2^8 since the last rescale, so the common case costs no
+// TMEM round trip.  Keys at or beyond L are masked.  Every wait is bounded (see ptx.cuh).
 #include <math.h>
 
 #include "internal.h"
@@ -14,23 +16,24 @@
 
 namespace fvar {
 
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 320;
 constexpr int kQRows = 128;
 constexpr int kKeys = 128;
 constexpr int kAtomBytes = 128 * 128;   // [128 rows][64 bf16] swizzled tile
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
 
 template <int D>
 struct AttnCfg {
-  static constexpr int kStages = (D == 64) ? 4 : 2;
-  static constexpr int kQBytes = kQRows * D * 2;
-  static constexpr int kKBytes = kKeys * D * 2;
-  static constexpr int kVBytes = D * kKeys * 2;
-  static constexpr int kStageBytes = kKBytes + kVBytes;
-  static constexpr int kPBytes = kQRows * kKeys * 2;
-  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kPBytes + 1024 + 256;
-  static constexpr int kTmemCols = 512;   // S0 [0,128), S1 [128,256), O [256, 256 + D)
+  static constexpr int kTileBytes = 128 * D * 2;          // a Q tile, a K tile [128 keys][D] or a V^T tile [D][128 keys]
+  static constexpr int kRing = (D == 64) ? 6 : 3;         // K_j, V_j, K_{j+1}, ...
+  static constexpr int kQBytes = 2 * kTileBytes;
+  static constexpr int kPTile = kQRows * kKeys * 2;
+  static constexpr int kPBytes = 2 * kPTile;
+  static constexpr int kSmemBytes = kQBytes + kRing * kTileBytes + kPBytes + 1024 + 256;
+  static constexpr int kTmemCols = 512;   // S0 [0,128), S1 [128,256), O0 [256,256+D), O1 [256+D,256+2D)
   static_assert(kSmemBytes > 116 * 1024, "one CTA per SM (the CTA allocates all of TMEM)");
-  static_assert(kSmemBytes <= 227 * 1024, "shared memory");
+  static_assert(kSmemBytes + 64 <= 227 * 1024, "shared memory");
+  static_assert(256 + 2 * D <= 512, "TMEM columns");
 };
 
 template <int D>
@@ -38,40 +41,42 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ AttnArgs p) {
   using Cfg = AttnCfg<D>;
-  constexpr int S = Cfg::kStages;
+  constexpr int NR = Cfg::kRing;
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t tmem_base_holder;
   __shared__ volatile int abort_flag;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = smem_base;
-  const uint32_t kv_smem = q_smem + Cfg::kQBytes;
-  const uint32_t p_smem = kv_smem + S * Cfg::kStageBytes;
+  const uint32_t ring_smem = q_smem + Cfg::kQBytes;
+  const uint32_t p_smem = ring_smem + NR * Cfg::kTileBytes;
   const uint32_t bar_base = p_smem + Cfg::kPBytes;
   const uint32_t q_full = bar_base;
-  auto kv_full = [&](int s) { return bar_base + 8u * (1 + s); };
-  auto kv_empty = [&](int s) { return bar_base + 8u * (1 + S + s); };
-  auto s_full = [&](int b) { return bar_base + 8u * (1 + 2 * S + b); };
-  const uint32_t p_full = bar_base + 8u * (3 + 2 * S);
-  const uint32_t o_full = bar_base + 8u * (4 + 2 * S);
+  auto ring_full = [&](int s) { return bar_base + 8u * (1 + s); };
+  auto ring_empty = [&](int s) { return bar_base + 8u * (1 + NR + s); };
+  auto s_full = [&](int t) { return bar_base + 8u * (1 + 2 * NR + t); };
+  auto p_full = [&](int t) { return bar_base + 8u * (3 + 2 * NR + t); };
+  auto o_full = [&](int t) { return bar_base + 8u * (5 + 2 * NR + t); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qt = blockIdx.x, h = blockIdx.y, e = blockIdx.z;
   const int b = e * p.bmul + p.boff;
   const int bh = b * p.H + h;
   const int nkv = (p.L + kKeys - 1) / kKeys;
+  const int ntiles = (p.r - qt * 2 * kQRows > kQRows) ? 2 : 1;     // query tiles this CTA really has
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
     mbar_init(q_full, 1);
-    for (int s = 0; s < S; ++s) {
-      mbar_init(kv_full(s), 1);
-      mbar_init(kv_empty(s), 1);
+    for (int s = 0; s < NR; ++s) {
+      mbar_init(ring_full(s), 1);
+      mbar_init(ring_empty(s), 1);
     }
-    mbar_init(s_full(0), 1);
-    mbar_init(s_full(1), 1);
-    mbar_init(p_full, 128);
-    mbar_init(o_full, 1);
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(s_full(t), 1);
+      mbar_init(p_full(t), 128);
+      mbar_init(o_full(t), 1);
+    }
     mbar_fence_init();
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
@@ -85,40 +90,43 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
-  const uint32_t tmem_o = tmem_base + 256;
   pdl_wait();
   pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {
       // ---------------------------------------------------------------- TMA producer
-      mbar_expect_tx(q_full, Cfg::kQBytes);
-      const int qrow0 = e * p.r + qt * kQRows;
+      mbar_expect_tx(q_full, ntiles * Cfg::kTileBytes);
+      const int qrow0 = e * p.r + qt * 2 * kQRows;
+      for (int t = 0; t < ntiles; ++t)
 #pragma unroll
-      for (int a = 0; a < D / 64; ++a) tma_load_2d(q_smem + a * kAtomBytes, &tmQ, q_full, h * D + a * 64, qrow0);
+        for (int a = 0; a < D / 64; ++a)
+          tma_load_2d(q_smem + t * Cfg::kTileBytes + a * kAtomBytes, &tmQ, q_full, h * D + a * 64, qrow0 + t * kQRows);
       uint32_t armed = 0, last_parity = 0;
       bool ok = true;
-      for (int j = 0; j < nkv; ++j) {
-        const int stage = j % S;
-        const uint32_t phase = (j / S) & 1u;
-        if (!mbar_wait(kv_empty(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
-        mbar_expect_tx(kv_full(stage), Cfg::kStageBytes);
-        const uint32_t ks = kv_smem + stage * Cfg::kStageBytes;
-        const uint32_t vs = ks + Cfg::kKBytes;
+      for (int i = 0; i < 2 * nkv; ++i) {            // even i: K of block i/2, odd i: V^T of block i/2
+        const int slot = i % NR, j = i >> 1;
+        const uint32_t phase = (i / NR) & 1u;
+        if (!mbar_wait(ring_empty(slot), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+        mbar_expect_tx(ring_full(slot), Cfg::kTileBytes);
+        const uint32_t dst = ring_smem + slot * Cfg::kTileBytes;
+        if ((i & 1) == 0) {
 #pragma unroll
-        for (int a = 0; a < D / 64; ++a) tma_load_3d(ks + a * kAtomBytes, &tmK, kv_full(stage), a * 64, j * kKeys, bh);
+          for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * kAtomBytes, &tmK, ring_full(slot), a * 64, j * kKeys, bh);
+        } else {
 #pragma unroll
-        for (int a = 0; a < 2; ++a) tma_load_3d(vs + a * (D * 128), &tmV, kv_full(stage), j * kKeys + a * 64, 0, bh);
-        armed |= 1u << stage;
-        last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
+          for (int a = 0; a < 2; ++a) tma_load_3d(dst + a * (D * 128), &tmV, ring_full(slot), j * kKeys + a * 64, 0, bh);
+        }
+        armed |= 1u << slot;
+        last_parity = (last_parity & ~(1u << slot)) | (phase << slot);
       }
-      if (!ok) {
+      if (!ok) {   // let every copy that was issued land before the shared memory is released
         const long long t0 = clock64();
         while (!mbar_try_wait(q_full, 0) && clock64() - t0 < kWaitCycles) {}
-        for (int s = 0; s < S; ++s)
+        for (int s = 0; s < NR; ++s)
           if (armed & (1u << s)) {
             const long long t1 = clock64();
-            while (!mbar_try_wait(kv_full(s), (last_parity >> s) & 1u) && clock64() - t1 < kWaitCycles) {}
+            while (!mbar_try_wait(ring_full(s), (last_parity >> s) & 1u) && clock64() - t1 < kWaitCycles) {}
           }
       }
     }
@@ -127,143 +135,164 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // ---------------------------------------------------------------- MMA issuer
       constexpr uint32_t idesc_s = umma_idesc_bf16(kQRows, kKeys);
       constexpr uint32_t idesc_o = umma_idesc_bf16(kQRows, D);
-      auto issue_s = [&](int j) {
-        const uint32_t ks = kv_smem + (j % S) * Cfg::kStageBytes;
-        const uint32_t d_tmem = tmem_base + (j & 1) * kKeys;
+      auto issue_s = [&](int t, int slot) {          // S_t = Q_t K^T
+        const uint32_t ks = ring_smem + slot * Cfg::kTileBytes, qs = q_smem + t * Cfg::kTileBytes;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint64_t da = smem_desc_sw128(q_smem + (k / 4) * kAtomBytes) + 2 * (k % 4);
+          const uint64_t da = smem_desc_sw128(qs + (k / 4) * kAtomBytes) + 2 * (k % 4);
           const uint64_t db = smem_desc_sw128(ks + (k / 4) * kAtomBytes) + 2 * (k % 4);
-          umma_bf16(d_tmem, da, db, idesc_s, k != 0);
+          umma_bf16(tmem_base + t * kKeys, da, db, idesc_s, k != 0);
         }
-        umma_commit(s_full(j & 1));
+        umma_commit(s_full(t));
       };
-      bool ok = mbar_wait(q_full, 0, p.status, &abort_flag);
-      if (ok) ok = mbar_wait(kv_full(0), 0, p.status, &abort_flag);
-      if (ok) {
-        tc_fence_after();
-        issue_s(0);
-      }
-      for (int j = 0; ok && j < nkv; ++j) {
-        if (j + 1 < nkv) {
-          if (!mbar_wait(kv_full((j + 1) % S), ((j + 1) / S) & 1u, p.status, &abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          issue_s(j + 1);
-        }
-        if (!mbar_wait(p_full, j & 1u, p.status, &abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t vs = kv_smem + (j % S) * Cfg::kStageBytes + Cfg::kKBytes;
+      auto issue_pv = [&](int t, int slot, bool accumulate) {   // O_t (+)= P_t V
+        const uint32_t vs = ring_smem + slot * Cfg::kTileBytes, ps = p_smem + t * Cfg::kPTile;
 #pragma unroll
         for (int k = 0; k < kKeys / 16; ++k) {
-          const uint64_t da = smem_desc_sw128(p_smem + (k / 4) * kAtomBytes) + 2 * (k % 4);
+          const uint64_t da = smem_desc_sw128(ps + (k / 4) * kAtomBytes) + 2 * (k % 4);
           const uint64_t db = smem_desc_sw128(vs + (k / 4) * (D * 128)) + 2 * (k % 4);
-          umma_bf16(tmem_o, da, db, idesc_o, k != 0);
+          umma_bf16(tmem_base + 256 + t * D, da, db, idesc_o, (accumulate || k != 0) ? 1u : 0u);
         }
-        umma_commit(kv_empty(j % S));
-        umma_commit(o_full);
+        umma_commit(o_full(t));
+      };
+      bool ok = mbar_wait(q_full, 0, p.status, &abort_flag);
+      if (ok) ok = mbar_wait(ring_full(0), 0, p.status, &abort_flag);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < ntiles; ++t) issue_s(t, 0);
+        umma_commit(ring_empty(0));
+      }
+      for (int j = 0; ok && j < nkv; ++j) {
+        const int vi = 2 * j + 1, ki = 2 * j + 2;
+        for (int t = 0; ok && t < ntiles; ++t) {
+          if (!mbar_wait(p_full(t), j & 1u, p.status, &abort_flag)) { ok = false; break; }
+          if (t == 0 && !mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(t, vi % NR, j > 0);
+          if (t == ntiles - 1) umma_commit(ring_empty(vi % NR));
+          if (j + 1 < nkv) {
+            if (t == 0 && !mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            issue_s(t, ki % NR);
+            if (t == ntiles - 1) umma_commit(ring_empty(ki % NR));
+          }
+        }
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax / accumulate
-    const int quad = warp & 3;
-    const int row_local = quad * 32 + lane;
-    const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-    const float c = p.scale_log2;
-    float o_acc[D];
-#pragma unroll
-    for (int i = 0; i < D; ++i) o_acc[i] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
-    bool ok = true;
+    // ------------------------------------------------------------------ softmax warp-groups
+    const int t = (warp - 2) >> 2;                       // query tile of this warp-group
+    if (t < ntiles) {
+      const int quad = warp & 3;                         // TMEM lanes [32 * quad, 32 * quad + 32)
+      const int row_local = quad * 32 + lane;
+      const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+      const uint32_t s_addr = tmem_base + t * kKeys + lane_addr;
+      const uint32_t o_addr = tmem_base + 256 + t * D + lane_addr;
+      const uint32_t p_row = p_smem + t * Cfg::kPTile + row_local * 128;
+      const float c = p.scale_log2;
+      float m_ref = -INFINITY, l_run = 0.f;
+      bool ok = true;
 
-    auto fold_o = [&](float alpha) {          // o_acc = o_acc * alpha + O_j (from TMEM)
-#pragma unroll
-      for (int cc = 0; cc < D / 32; ++cc) {
-        uint32_t t[32];
-        tmem_ld32(tmem_o + lane_addr + cc * 32, t);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o_acc[cc * 32 + i] = fmaf(o_acc[cc * 32 + i], alpha, __uint_as_float(t[i]));
-      }
-    };
-
-    for (int j = 0; j < nkv; ++j) {
-      ok = __all_sync(0xffffffffu, mbar_wait(s_full(j & 1), (j >> 1) & 1u, p.status, &abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t s_addr = tmem_base + (j & 1) * kKeys + lane_addr;
-      const int valid = p.L - j * kKeys;        // keys of this block below L (>= 128: all)
-      float m_blk = -INFINITY;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t t[32];
-        tmem_ld32(s_addr + cc * 32, t);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float s = (cc * 32 + i < valid) ? __uint_as_float(t[i]) : -INFINITY;
-          m_blk = fmaxf(m_blk, s);
-        }
-      }
-      const float m_new = fmaxf(m_run, m_blk);
-      const float alpha = exp2f((m_run - m_new) * c);
-      const float neg_mc = -m_new * c;
-      if (j > 0) {
-        // O_{j-1} must be folded (and P's buffer released by the tensor core) before P_j is written.
-        ok = __all_sync(0xffffffffu, mbar_wait(o_full, (j - 1) & 1u, p.status, &abort_flag));
+      for (int j = 0; j < nkv; ++j) {
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full(t), j & 1u, p.status, &abort_flag));
         if (!ok) break;
         tc_fence_after();
-        fold_o(alpha_prev);
-      }
-      float l_blk = 0.f;
-#pragma unroll 1
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t t[32];
-        tmem_ld32(s_addr + cc * 32, t);
+        const int valid = p.L - j * kKeys;               // keys of this block below L (>= 128: all)
+        // the whole S row (128 fp32) in registers: four TMEM loads in flight, one wait
+        uint32_t v[4][32];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) tmem_ld32(s_addr + cc * 32, v[cc]);
         tmem_ld_wait();
-        uint32_t pk[16];
+        if (valid < kKeys) {                             // last block: mask keys at or beyond L
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float p0 = (cc * 32 + i < valid) ? exp2f(fmaf(__uint_as_float(t[i]), c, neg_mc)) : 0.f;
-          float p1 = (cc * 32 + i + 1 < valid) ? exp2f(fmaf(__uint_as_float(t[i + 1]), c, neg_mc)) : 0.f;
-          l_blk += p0 + p1;
-          __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-          pk[i >> 1] = *reinterpret_cast<uint32_t *>(&v2);
+          for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (cc * 32 + i >= valid) v[cc][i] = 0xff800000u;   // -inf
         }
-        // columns cc*32 .. cc*32+31 of row row_local: four 16-byte chunks of the swizzled tile
-        const uint32_t atom = p_smem + (cc >> 1) * kAtomBytes + row_local * 128;
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t chunk = static_cast<uint32_t>((cc & 1) * 4 + q);
-          const uint32_t addr = atom + ((chunk ^ (row_local & 7)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q * 4]), "r"(pk[q * 4 + 1]),
-                       "r"(pk[q * 4 + 2]), "r"(pk[q * 4 + 3])
-                       : "memory");
+        for (int cc = 0; cc < 4; ++cc)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(v[cc][i]));
+        const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        const float m_cand = fmaxf(m_ref, m_blk);
+        const bool need = (m_cand - m_ref) * c > kRescaleThreshold;      // true on the first block (m_ref = -inf)
+        if (j > 0) {
+          // P V of block j-1 must be complete before P's buffer is overwritten or O is touched
+          ok = __all_sync(0xffffffffu, mbar_wait(o_full(t), (j - 1) & 1u, p.status, &abort_flag));
+          if (!ok) break;
+          tc_fence_after();
         }
-      }
-      l_run = l_run * alpha + l_blk;
-      m_run = m_new;
-      alpha_prev = alpha;
-      fence_proxy_async_smem();
-      tc_fence_before();
-      mbar_arrive(p_full);
-    }
-    if (ok && nkv > 0) {
-      if (__all_sync(0xffffffffu, mbar_wait(o_full, (nkv - 1) & 1u, p.status, &abort_flag))) {
-        tc_fence_after();
-        fold_o(alpha_prev);
-        const int rib = qt * kQRows + row_local;
-        if (rib < p.r) {
-          const float inv_l = 1.0f / l_run;
-          bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? exp2f((m_ref - m_cand) * c) : 1.0f;
+          if (need) m_ref = m_cand;
+          l_run *= alpha;
+          if (j > 0) {
+#pragma unroll 1
+            for (int cc = 0; cc < D / 32; ++cc) {
+              uint32_t o[32];
+              tmem_ld32(o_addr + cc * 32, o);
+              tmem_ld_wait();
 #pragma unroll
-          for (int q = 0; q < D / 8; ++q) {
-            uint32_t w[4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              __nv_bfloat162 v2 = __floats2bfloat162_rn(o_acc[q * 8 + t * 2] * inv_l, o_acc[q * 8 + t * 2 + 1] * inv_l);
-              w[t] = *reinterpret_cast<uint32_t *>(&v2);
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st32(o_addr + cc * 32, o);
             }
-            reinterpret_cast<uint4 *>(dst)[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            tmem_st_wait();
+          }
+        }
+        const float neg_mc = -m_ref * c;
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float p0 = exp2f(fmaf(__uint_as_float(v[cc][i]), c, neg_mc));       // exp2(-inf) = 0 for masked keys
+            const float p1 = exp2f(fmaf(__uint_as_float(v[cc][i + 1]), c, neg_mc));
+            ls[(i >> 1) & 3] += p0 + p1;
+            __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+            pk[i >> 1] = *reinterpret_cast<uint32_t *>(&v2);
+          }
+          // columns cc*32 .. cc*32+31 of this row: four 16-byte chunks of the swizzled tile
+          const uint32_t atom = p_row + (cc >> 1) * kAtomBytes;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t chunk = static_cast<uint32_t>((cc & 1) * 4 + q);
+            const uint32_t addr = atom + ((chunk ^ (row_local & 7)) << 4);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q * 4]), "r"(pk[q * 4 + 1]),
+                         "r"(pk[q * 4 + 2]), "r"(pk[q * 4 + 3])
+                         : "memory");
+          }
+        }
+        const float l_blk = (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        l_run += l_blk;
+        fence_proxy_async_smem();
+        tc_fence_before();
+        mbar_arrive(p_full(t));
+      }
+      if (ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag))) {
+        tc_fence_after();
+        const int rib = qt * 2 * kQRows + t * kQRows + row_local;
+        const float inv_l = 1.0f / l_run;
+        bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;
+#pragma unroll 1
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(o_addr + cc * 32, v);
+          tmem_ld_wait();
+          if (rib < p.r) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              uint32_t w[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + u * 2]) * inv_l,
+                                                          __uint_as_float(v[q * 8 + u * 2 + 1]) * inv_l);
+                w[u] = *reinterpret_cast<uint32_t *>(&v2);
+              }
+              reinterpret_cast<uint4 *>(dst + cc * 32)[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
           }
         }
       }
@@ -300,7 +329,7 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   using Cfg = AttnCfg<D>;
   cudaError_t err = set_attr<D>();
   if (err != cudaSuccess) return err;
-  dim3 grid((a.r + kQRows - 1) / kQRows, a.H, a.B_eff);
+  dim3 grid((a.r + 2 * kQRows - 1) / (2 * kQRows), a.H, a.B_eff);
   return launch_pdl(attention_kernel<D>, grid, dim3(kAttnThreads), Cfg::kSmemBytes, st, tmQ, tmK, tmV, a);
 }
 

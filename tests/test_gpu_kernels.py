@@ -6,7 +6,7 @@ import torch
 
 import synth_inputs as si
 from oracle import fvar_oracle as orc
-from helpers import assert_close, bf16_to_numpy, to_bf16_cuda
+from helpers import assert_close, assert_out_close, bf16_to_numpy, to_bf16_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -133,7 +133,8 @@ def test_attention(fv, B, H, D, r, L, L_cap):
     _poll(fv)
     ref = np.stack([orc.attention(q[b].astype(np.float64), K[b].astype(np.float64), V[b].astype(np.float64), H)
                     for b in range(B)])
-    assert_close(got, ref, max_rel=2e-2, min_cos=0.9995, what="attention")
+    assert_out_close(got, ref, what="attention")      # bf16 result: the bar plus the rounding of the output
+    assert_close(got, ref, max_rel=1.0, min_cos=0.9995, what="attention cosine")
 
 
 def test_attention_scaled_down_scores_uniform(fv):
