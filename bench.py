@@ -35,11 +35,36 @@ WORKLOADS = {
     "var_d16_dense3_b16": dict(shape="d16", B=16, first_late=7, keep=1.0, null_only=False),
     "var_d30_late2_b32": dict(shape="d30", B=32, first_late=8, keep=0.5, null_only=True),
     "var_d30_dense2_b32": dict(shape="d30", B=32, first_late=8, keep=1.0, null_only=False),
+    # Infinity-2B-shaped generator (32 blocks in 8 groups, cross-attention to 256 context tokens), B = 2 (one
+    # CFG pair), the three fidelity-refinement scales 40 / 48 / 64 over a cache pre-filled with 2521 rows:
+    # null-only + RP + RTR at the tabulated rank of every block group (alpha = 0.96) at all three scales ...
+    "infinity2b_late3_b2": dict(shape="inf2b", B=2, first_late=10, keep="table", null_only=True),
+    # ... the schedule of Sec. 4.1 (alpha = {0.96, 0, 0}: scale 40 approximated, 48 and 64 skipped) ...
+    "infinity2b_paper_b2": dict(shape="inf2b", B=2, first_late=10, keep="paper", null_only=True),
+    # ... and the unpruned dense path with both CFG branches.
+    "infinity2b_dense3_b2": dict(shape="inf2b", B=2, first_late=10, keep=1.0, null_only=False),
 }
 
 
+def scale_plan(wl, shp):
+    """Per late scale index: None (skip) or the list of ranks per block group (M = dense)."""
+    from paper_2512_16483_b200 import schedule
+    Ms, plan = shp.tokens_per_scale(), {}
+    for k in range(wl["first_late"], len(Ms)):
+        keep = wl["keep"]
+        if keep in ("table", "paper"):
+            side = shp.scales[k]
+            if keep == "paper" and schedule.INFINITY_ALPHA[schedule.INFINITY_LATE_SCALES.index(side)] == 0.0:
+                plan[k] = None
+            else:
+                plan[k] = schedule.infinity_group_ranks(side, shp.width, shp.n_groups)
+        else:
+            plan[k] = [schedule.rank_from_keep_ratio(Ms[k], keep)] * shp.n_groups
+    return plan
+
+
 def make_shape(name):
-    return {"d16": si.shape_var_d16, "d30": si.shape_var_d30}[name]()
+    return {"d16": si.shape_var_d16, "d30": si.shape_var_d30, "inf2b": si.shape_infinity_2b}[name]()
 
 
 def peaks():
@@ -89,41 +114,53 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------------------------- the oracle leg
 
-def oracle_leg(wl, steps, warmup, sample_pairs=2):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload: `sample_pairs` CFG
-    pairs, every block, every late scale.  Returns (tokens/s, seconds per step, description, threads)."""
+def oracle_leg(wl, steps, warmup):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  VAR shapes: 2 of the CFG
+    pairs, every block, every late scale.  Infinity shape: the one CFG pair, the first block group of the 8,
+    every non-skipped late scale, extrapolated x 8 groups.  Returns (tokens/s, seconds per step,
+    description, threads)."""
     from oracle import fvar_oracle as orc
     try:
         from threadpoolctl import threadpool_info
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
     except Exception:
         threads = os.cpu_count() or 1
+    full = make_shape(wl["shape"])
+    plan_full = scale_plan(wl, full)
     shp = make_shape(wl["shape"])
-    B = 2 * sample_pairs
+    big = wl["shape"] == "inf2b"
+    groups = 1 if big else full.n_groups
+    shp.n_blocks = groups * shp.blocks_per_group
+    B = 2 if big else 4
     Ms = shp.tokens_per_scale()
     k0 = wl["first_late"]
     weights = si.make_weights(SEED, shp)
     o = orc.Oracle(weights, shp.n_heads, shp.blocks_per_group, shp.hw(), shp.ln_eps)
-    o.set_cond(si.make_cond(SEED, B, shp.width))
+    ctx = si.make_context(SEED, B, shp.ctx_len, shp.ctx_width) if shp.has_cross_attn else None
+    o.set_cond(si.make_cond(SEED, B, shp.width), ctx)
     L0 = sum(Ms[:k0])
     K, V = si.make_kv_prefill(SEED, shp.n_blocks, B, L0, shp.width)
     gc = si.make_group_cache(SEED, shp.n_groups, B, Ms[k0 - 1], shp.width)
-    toks = {k: si.make_tokens(SEED, B, Ms[k], shp.width) for k in range(k0, len(Ms))}
-    late = wl["keep"] < 1.0
-    if late:
-        for k in range(k0, len(Ms)):
-            r = orc.rank_from_keep_ratio(Ms[k], wl["keep"])
-            for g in range(shp.n_groups):
+    toks = {k: si.make_tokens(SEED, B, Ms[k], shp.width) for k in plan_full}
+    pols = {}
+    for k, ranks in plan_full.items():
+        if ranks is None:
+            continue
+        ranks = ranks[:groups]
+        late = any(r < Ms[k] for r in ranks)
+        for g, r in enumerate(ranks):
+            if r < Ms[k]:
                 o.set_projection(k, g, si.make_projection(SEED, k, g, Ms[k], r))
-    pol = orc.Policy("lowrank_rtr" if late else "dense", "null_only" if wl["null_only"] else "pair", wl["keep"])
+        pols[k] = orc.Policy("lowrank_rtr" if late else "dense", "null_only" if wl["null_only"] else "pair",
+                             rank_per_group=ranks if late else None)
     E = B // 2 if wl["null_only"] else B
-    tokens_per_step = E * sum(Ms[k0:])
+    tokens_per_step = E * sum(Ms[k] for k in plan_full)       # skipped scales deliver their positions too
 
     def one():
         o.load_kv(K, V)
         o.load_group_cache(k0 - 1, gc)
-        for k in range(k0, len(Ms)):
-            o.scale_step(toks[k], k, pol)
+        for k in sorted(pols):
+            o.scale_step(toks[k], k, pols[k])
             o.kv_append(k)
 
     for _ in range(warmup):
@@ -131,9 +168,10 @@ def oracle_leg(wl, steps, warmup, sample_pairs=2):
     t0 = time.perf_counter()
     for _ in range(steps):
         one()
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    desc = "%d of the workload's CFG pairs, all %d blocks, all %d late scales, fp64 numpy" % (
-        sample_pairs, shp.n_blocks, len(Ms) - k0)
+    dt = (time.perf_counter() - t0) / max(steps, 1) * (full.n_groups / groups)
+    desc = "%d CFG pair(s), %d of %d block groups%s, %d late scale(s) run, fp64 numpy" % (
+        B // 2, groups, full.n_groups, " (time extrapolated x %d)" % (full.n_groups // groups) if groups < full.n_groups else "",
+        len(pols))
     return tokens_per_step / dt, dt, desc, threads
 
 
@@ -147,6 +185,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="var_d16_late3_b16", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--max-splits", type=int, default=0, help="tuning: largest split-K factor (1, 2, 4); 0 = library default")
     ap.add_argument("--profile-run", action="store_true",
                     help="for runs under ncu: skip the host-buffer leg, the event pass and the CPU baseline")
     args = ap.parse_args()
@@ -156,7 +195,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     metric = "tokens/s over the late scale steps (output positions delivered per second)"
     config = {"workload": args.workload, "shape": wl["shape"], "batch": wl["B"],
-              "late_scale_sides": list(make_shape(wl["shape"]).scales[wl["first_late"]:]), "keep_ratio": wl["keep"],
+              "late_scale_sides": list(make_shape(wl["shape"]).scales[wl["first_late"]:]), "keep": wl["keep"],
               "cfg": "null_only" if wl["null_only"] else "pair",
               "l2": "inputs_exceed_l2 (the stack's weights, streamed every step, are larger than L2)"}
 
@@ -191,46 +230,87 @@ def main():
     shp = make_shape(wl["shape"])
     B, k0 = wl["B"], wl["first_late"]
     Ms = shp.tokens_per_scale()
-    late_scales = list(range(k0, len(Ms)))
-    late = wl["keep"] < 1.0
-    mode = fv.LOWRANK_RTR if late else fv.DENSE
+    plan = scale_plan(wl, shp)
+    late_scales = sorted(plan)
     cfg_mode = fv.CFG_NULL_ONLY if wl["null_only"] else fv.CFG_PAIR
     E = B // 2 if wl["null_only"] else B
+    seed = SEED + rank
+    big = wl["shape"] == "inf2b"
 
     def bf16_cuda(a):
         return torch.from_numpy(si.bf16_bits(a).view(np.int16).reshape(a.shape)).view(torch.bfloat16).cuda()
 
-    seed = SEED + rank
-    weights = [{k: bf16_cuda(v) for k, v in blk.items()} for blk in si.make_weights(seed, shp)]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+
+    def randn_bf16(shape, std=1.0):          # large tensors are drawn on the device (same recipe, torch's generator)
+        return (torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+
+    if big:
+        C, F, W = shp.width, shp.ffn_dim, shp.ctx_width
+        dims = {"w_qkv": (3 * C, C), "b_qkv": (3 * C,), "w_o": (C, C), "b_o": (C,), "w_fc1": (F, C), "b_fc1": (F,),
+                "w_fc2": (C, F), "b_fc2": (C,), "w_ada": (6 * C, C), "b_ada": (6 * C,), "w_cq": (C, C),
+                "w_ckv": (2 * C, W), "w_co": (C, C)}
+        weights = []
+        for _ in range(shp.n_blocks):
+            blk = {n: randn_bf16(d, 0.02) for n, d in dims.items()}
+            blk["ln_c_gamma"] = (1.0 + 0.1 * torch.randn(C, generator=gen, device="cuda")).to(torch.bfloat16)
+            weights.append(blk)
+    else:
+        weights = [{k: bf16_cuda(v) for k, v in blk.items()} for blk in si.make_weights(seed, shp)]
     ctx = fv.Fvar(weights, blocks_per_group=shp.blocks_per_group, n_heads=shp.n_heads, head_dim=shp.head_dim,
-                  ffn_dim=shp.ffn_dim, scale_hw=shp.hw(), max_batch=B, ln_eps=shp.ln_eps)
-    ctx.set_cond(bf16_cuda(si.make_cond(seed, B, shp.width)))
+                  ffn_dim=shp.ffn_dim, scale_hw=shp.hw(), max_batch=B, ctx_len=shp.ctx_len, ctx_width=shp.ctx_width,
+                  ln_eps=shp.ln_eps)
+    if args.max_splits:
+        ctx.set_option(fv.OPT_GEMM_MAX_SPLITS, args.max_splits)
+    context = bf16_cuda(si.make_context(seed, B, shp.ctx_len, shp.ctx_width)) if shp.has_cross_attn else None
+    ctx.set_cond(bf16_cuda(si.make_cond(seed, B, shp.width)), context)
     L0 = sum(Ms[:k0])
-    K, V = si.make_kv_prefill(seed, shp.n_blocks, B, L0, shp.width)
-    ctx.load_kv(bf16_cuda(K), bf16_cuda(V))
-    ctx.load_group_cache(k0 - 1, torch.from_numpy(si.make_group_cache(seed, shp.n_groups, B, Ms[k0 - 1], shp.width)).cuda())
-    del K, V
-    if late:
-        for k in late_scales:
-            r = schedule.rank_from_keep_ratio(Ms[k], wl["keep"])
-            for g in range(shp.n_groups):
-                ctx.set_projection(k, g, bf16_cuda(np.ascontiguousarray(si.make_projection(seed, k, g, Ms[k], r).T)))
-    toks = {k: bf16_cuda(si.make_tokens(seed, B, Ms[k], shp.width)) for k in late_scales}
+    if big:
+        ctx.load_kv(randn_bf16((shp.n_blocks, B, L0, shp.width)), randn_bf16((shp.n_blocks, B, L0, shp.width)))
+        ctx.load_group_cache(k0 - 1, torch.randn((shp.n_groups, B, Ms[k0 - 1], shp.width), generator=gen, device="cuda"))
+    else:
+        K, V = si.make_kv_prefill(seed, shp.n_blocks, B, L0, shp.width)
+        ctx.load_kv(bf16_cuda(K), bf16_cuda(V))
+        ctx.load_group_cache(k0 - 1, torch.from_numpy(si.make_group_cache(seed, shp.n_groups, B, Ms[k0 - 1], shp.width)).cuda())
+        del K, V
+    torch.cuda.synchronize()
+    modes = {}
+    for k in late_scales:
+        ranks = plan[k]
+        if ranks is None:
+            modes[k] = (fv.SKIP, None)
+            continue
+        late = any(r < Ms[k] for r in ranks)
+        modes[k] = (fv.LOWRANK_RTR if late else fv.DENSE, ranks if late else None)
+        for g, r in enumerate(ranks):
+            if r < Ms[k]:
+                qt = randn_bf16((r, Ms[k]), 1.0 / np.sqrt(r)) if big else \
+                    bf16_cuda(np.ascontiguousarray(si.make_projection(seed, k, g, Ms[k], r).T))
+                ctx.set_projection(k, g, qt)
+    toks = {k: (randn_bf16((B, Ms[k], shp.width)) if big else bf16_cuda(si.make_tokens(seed, B, Ms[k], shp.width)))
+            for k in late_scales}
     outs = {k: torch.empty((E, Ms[k], shp.width), dtype=torch.bfloat16, device="cuda") for k in late_scales}
     toks_host = {k: toks[k].cpu().pin_memory() for k in late_scales}
     outs_host = {k: torch.empty((E, Ms[k], shp.width), dtype=torch.bfloat16).pin_memory() for k in late_scales}
-    tokens_per_step = E * sum(Ms[k] for k in late_scales)
+    tokens_per_step = E * sum(Ms[k] for k in late_scales)     # a skipped scale still delivers its positions
 
     def step_device():
         ctx.restore_loaded()
         for k in late_scales:
-            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_mode, keep_ratio=wl["keep"], out=outs[k])
+            mode, ranks = modes[k]
+            if mode == fv.SKIP:
+                continue
+            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_mode, rank_per_group=ranks, out=outs[k])
             ctx.kv_append(k)
 
     def step_host():
         ctx.restore_loaded()
         for k in late_scales:
-            ctx.scale_step_host(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_mode, keep_ratio=wl["keep"])
+            mode, ranks = modes[k]
+            if mode == fv.SKIP:
+                continue
+            ctx.scale_step_host(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_mode, rank_per_group=ranks)
             ctx.kv_append(k)
 
     def barrier():
@@ -294,12 +374,12 @@ def main():
                 "classes": classes}
     line = {
         "metric": metric, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
-        "ms_per_step": ms_step, "ms_per_scale_step": ms_step / len(late_scales), "higher_is_better": True,
+        "ms_per_step": ms_step, "ms_per_scale_step": ms_step / max(1, sum(1 for k in late_scales if modes[k][0] != fv.SKIP)), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e, "unit": "tokens/s",
-                "h2d_bytes_per_step": sum(B * Ms[k] * shp.width * 2 for k in late_scales),
-                "d2h_bytes_per_step": sum(E * Ms[k] * shp.width * 2 for k in late_scales)},
+                "h2d_bytes_per_step": sum(B * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP),
+                "d2h_bytes_per_step": sum(E * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP)},
         "roofline": roofline,
     }
     if world == 1 and not args.no_cpu_baseline and not args.profile_run:
