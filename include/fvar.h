@@ -167,6 +167,9 @@ enum { FVAR_KCLASS_GEMM = 0, FVAR_KCLASS_ATTENTION = 1, FVAR_KCLASS_LN = 2, FVAR
 fvar_status fvar_profile_enable(fvar_ctx *ctx, int on);
 fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long long *launches, double *flops,
                               double *bytes);
+/* Per-launch event times (ms) of one kernel class in launch order: up to `capacity` values into ms_host;
+ * *count_host receives the number of launches recorded. */
+fvar_status fvar_profile_dump(fvar_ctx *ctx, int kclass, float *ms_host, int capacity, int *count_host);
 
 /* Committed cache rows of `block` (host value). */
 int fvar_cache_len(const fvar_ctx *ctx, int block);

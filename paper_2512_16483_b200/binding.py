@@ -84,6 +84,7 @@ def load_library() -> ct.CDLL:
         "fvar_set_option": (i, [vp, i, i]),
         "fvar_profile_enable": (i, [vp, i]),
         "fvar_profile_read": (i, [vp, i, P(ct.c_double), P(ll), P(ct.c_double), P(ct.c_double)]),
+        "fvar_profile_dump": (i, [vp, i, P(ct.c_float), i, P(i)]),
         "fvar_destroy": (None, [vp]),
         "fvar_last_error": (ct.c_char_p, [vp]),
         "fvar_row_scores": (i, [vp, i, i, i, vp, vp]),
@@ -104,7 +105,7 @@ def load_library() -> ct.CDLL:
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
-            "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read",
+            "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
             "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
@@ -352,6 +353,13 @@ class Fvar:
 
     def profile_enable(self, on: bool):
         self._check(self.lib.fvar_profile_enable(self.ctx, int(on)))
+
+    def profile_dump(self, kclass: int, capacity: int = 4096):
+        """Per-launch times in ms of one kernel class, in launch order."""
+        buf = (ct.c_float * capacity)()
+        n = ct.c_int(0)
+        self._check(self.lib.fvar_profile_dump(self.ctx, kclass, buf, capacity, ct.byref(n)))
+        return [buf[j] for j in range(min(n.value, capacity))]
 
     def profile_read(self, kclass: int):
         """(total ms, launches, algorithmic flops, algorithmic bytes) of one kernel class."""

@@ -117,7 +117,10 @@ struct fvar_ctx {
   std::vector<CUtensorMap> qt_map;     // [scale][group]
   std::vector<CUtensorMap> xt_map;     // [scale][3]
   std::vector<CUtensorMap> kmap, vmap, ckmap, cvmap;   // per block
-  CUtensorMap y_map, a_map, q_map, h_map, silu_map;
+  // GEMM A operands: one map per box height (16, 32, 64, 128 rows); q_map feeds the attention kernel
+  struct ActMaps { CUtensorMap m[4]; };
+  ActMaps y_map, a_map, h_map, silu_map;
+  CUtensorMap q_map;
   // state
   int B;                               // batch of the current generation (0: no cond set)
   std::vector<int> len;                // committed cache rows per block
@@ -260,7 +263,18 @@ fvar_status cuda_fail(fvar_ctx *ctx, cudaError_t e, const char *what) {
   } while (0)
 
 // out = A W^T (+ epilogue) on the context's stream; picks the tile width from the problem size.
-fvar_status run_gemm(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
+fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what);
+
+// A operand from one of the library's activation buffers: a single row tile takes the shortest box
+// that covers its rows.
+fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int blk, int wid, GemmArgs &g, const char *what) {
+  int t = 3;
+  if (g.nbatch == 1 && g.R <= 64) t = g.R <= 16 ? 0 : (g.R <= 32 ? 1 : 2);
+  g.a_box_rows = 16 << t;
+  return run_gemm_map(ctx, epi, maps.m[t], blk, wid, g, what);
+}
+
+fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
   const int tiles_m = (g.R + 127) / 128 * g.nbatch;
   int bn = 64, sp = 1;
   gemm_pick_tile(tiles_m, g.N, g.K, ctx->num_sms, ctx->max_splits, kSplitScratchBytes, &bn, &sp);
@@ -394,9 +408,12 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
       for (int t = 0; t < 3 && ok; ++t)
         ok = tmap_2d(&c->wmap[(b * W_COUNT + i) * 3 + t], c->w[i][b], w_cols[i], w_rows[i], w_cols[i], kBNs[t]);
   const size_t act_rows = static_cast<size_t>(c->Bmax) * c->Mmax;
-  ok = ok && tmap_2d(&c->y_map, c->y, C, act_rows, C, 128) && tmap_2d(&c->a_map, c->a, C, act_rows, C, 128) &&
-       tmap_2d(&c->q_map, c->q, C, act_rows, C, 128) && tmap_2d(&c->h_map, c->hbuf, F, act_rows, F, 128) &&
-       tmap_2d(&c->silu_map, c->silu_c, C, c->Bmax, C, 128);
+  for (int t = 0; t < 4 && ok; ++t) {
+    const uint32_t box = 16u << t;
+    ok = tmap_2d(&c->y_map.m[t], c->y, C, act_rows, C, box) && tmap_2d(&c->a_map.m[t], c->a, C, act_rows, C, box) &&
+         tmap_2d(&c->h_map.m[t], c->hbuf, F, act_rows, F, box) && tmap_2d(&c->silu_map.m[t], c->silu_c, C, c->Bmax, C, box);
+  }
+  ok = ok && tmap_2d(&c->q_map, c->q, C, act_rows, C, 128);
   c->xt_map.resize(static_cast<size_t>(cfg->n_scales) * 3);
   for (int k = 0; k < cfg->n_scales && ok; ++k)
     for (int t = 0; t < 3 && ok; ++t)
@@ -487,6 +504,19 @@ fvar_status fvar_profile_enable(fvar_ctx *ctx, int on) {
   return FVAR_OK;
 }
 
+fvar_status fvar_profile_dump(fvar_ctx *ctx, int kclass, float *ms_host, int capacity, int *count_host) {
+  if (!ctx || !ms_host || !count_host || capacity < 0) return FVAR_EINVAL;
+  FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  int n = 0;
+  for (const auto &r : ctx->prof) {
+    if (r.kclass != kclass) continue;
+    if (n < capacity) FV_CUDA(ctx, cudaEventElapsedTime(&ms_host[n], r.e0, r.e1), "event elapsed");
+    ++n;
+  }
+  *count_host = n;
+  return FVAR_OK;
+}
+
 fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long long *launches, double *flops,
                               double *bytes) {
   if (!ctx || !total_ms || !launches || !flops || !bytes) return FVAR_EINVAL;
@@ -567,7 +597,7 @@ fvar_status fvar_set_cond(fvar_ctx *ctx, int B, const void *cond, const void *co
       g.vt = ctx->cvt + blk * ctx->ckv_block_elems();
       g.C = C; g.H = ctx->H; g.D = ctx->D; g.L_cap = ctx->ctx_cap; g.L_prev = 0; g.col_base = C;
       g.out_bf16 = ctx->q; g.ld_out = C;           // unused: no column maps to the q part
-      fvar_status s = run_gemm(ctx, EPI_QKV, ctx_map, blk, W_CKV, g, "context kv gemm");
+      fvar_status s = run_gemm_map(ctx, EPI_QKV, ctx_map, blk, W_CKV, g, "context kv gemm");
       if (s != FVAR_OK) return s;
     }
   }

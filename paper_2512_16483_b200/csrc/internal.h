@@ -20,6 +20,7 @@ enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU_BF16 = 2, EPI_QKV = 3, EPI_RE
 
 struct GemmArgs {
   int R, N, K;            // out[R][N] = A[R][K] * W[N][K]^T, per batch
+  int a_box_rows;         // rows of the A tensor map's box (0 = 128)
   int nbatch;             // number of independent problems sharing the launch
   int a_batch_rows;       // row offset of batch e in the A tensor map (0: A shared by all)
   int b_batch_rows;       // row offset of batch e in the W tensor map (0: W shared by all)
