@@ -45,6 +45,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t tmem_base_holder;
   __shared__ volatile int abort_flag;
+  __shared__ volatile int merge_last[2];
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = smem_base;
@@ -59,10 +60,16 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   auto o_full = [&](int t) { return bar_base + 8u * (5 + 2 * NR + t); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qt = blockIdx.x, h = blockIdx.y, e = blockIdx.z;
+  // Split-KV: kv_splits CTAs share one query tile pair, each covering a contiguous range of key
+  // blocks; their unnormalised results are merged by whichever of them finishes last.
+  const int splits = p.kv_splits > 1 ? p.kv_splits : 1;
+  const int qt = blockIdx.x / splits, sp = blockIdx.x - qt * splits, h = blockIdx.y, e = blockIdx.z;
   const int b = e * p.bmul + p.boff;
   const int bh = b * p.H + h;
-  const int nkv = (p.L + kKeys - 1) / kKeys;
+  const int nkv_total = (p.L + kKeys - 1) / kKeys;
+  const int kv_per = (nkv_total + splits - 1) / splits;
+  const int jb0 = sp * kv_per;                                    // first key block of this CTA
+  const int nkv = min(kv_per, nkv_total - jb0);                   // >= 1: the host sizes splits so
   const int ntiles = (p.r - qt * 2 * kQRows > kQRows) ? 2 : 1;     // query tiles this CTA really has
 
   if (threadIdx.x == 0) {
@@ -112,10 +119,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t dst = ring_smem + slot * Cfg::kTileBytes;
         if ((i & 1) == 0) {
 #pragma unroll
-          for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * kAtomBytes, &tmK, ring_full(slot), a * 64, j * kKeys, bh);
+          for (int a = 0; a < D / 64; ++a) tma_load_3d(dst + a * kAtomBytes, &tmK, ring_full(slot), a * 64, (jb0 + j) * kKeys, bh);
         } else {
 #pragma unroll
-          for (int a = 0; a < 2; ++a) tma_load_3d(dst + a * (D * 128), &tmV, ring_full(slot), j * kKeys + a * 64, 0, bh);
+          for (int a = 0; a < 2; ++a) tma_load_3d(dst + a * (D * 128), &tmV, ring_full(slot), (jb0 + j) * kKeys + a * 64, 0, bh);
         }
         armed |= 1u << slot;
         last_parity = (last_parity & ~(1u << slot)) | (phase << slot);
@@ -197,7 +204,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         ok = __all_sync(0xffffffffu, mbar_wait(s_full(t), j & 1u, p.status, &abort_flag));
         if (!ok) break;
         tc_fence_after();
-        const int valid = p.L - j * kKeys;               // keys of this block below L (>= 128: all)
+        const int valid = p.L - (jb0 + j) * kKeys;       // keys of this block below L (>= 128: all)
         // the whole S row (128 fp32) in registers: four TMEM loads in flight, one wait
         uint32_t v[4][32];
 #pragma unroll
@@ -274,25 +281,86 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag))) {
         tc_fence_after();
         const int rib = qt * 2 * kQRows + t * kQRows + row_local;
-        const float inv_l = 1.0f / l_run;
         bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;
-#pragma unroll 1
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t v[32];
-          tmem_ld32(o_addr + cc * 32, v);
-          tmem_ld_wait();
-          if (rib < p.r) {
+        auto store_chunk = [&](int cc, const float (&o)[32], float scale) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              uint32_t w[4];
+          for (int q = 0; q < 4; ++q) {
+            uint32_t w[4];
 #pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + u * 2]) * inv_l,
-                                                          __uint_as_float(v[q * 8 + u * 2 + 1]) * inv_l);
-                w[u] = *reinterpret_cast<uint32_t *>(&v2);
-              }
-              reinterpret_cast<uint4 *>(dst + cc * 32)[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int u = 0; u < 4; ++u) {
+              __nv_bfloat162 v2 = __floats2bfloat162_rn(o[q * 8 + u * 2] * scale, o[q * 8 + u * 2 + 1] * scale);
+              w[u] = *reinterpret_cast<uint32_t *>(&v2);
             }
+            reinterpret_cast<uint4 *>(dst + cc * 32)[q] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        };
+        if (splits == 1) {
+          const float inv_l = 1.0f / l_run;
+#pragma unroll 1
+          for (int cc = 0; cc < D / 32; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + cc * 32, v);
+            tmem_ld_wait();
+            float o[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+            if (rib < p.r) store_chunk(cc, o, inv_l);
+          }
+        } else {
+          // Park (O, m, l) of this key range.  Layout per (tile slot, split): float4 number d4 * 128 + row
+          // (coalesced across the lanes of a warp), then m[128] and l[128].
+          const int tslot = ((e * p.H + h) * static_cast<int>(gridDim.x / splits) + qt) * 2 + t;
+          const size_t per_split = static_cast<size_t>(D + 2) * kQRows;            // floats
+          float *mine = p.part + (static_cast<size_t>(tslot) * splits + sp) * per_split;
+#pragma unroll 1
+          for (int cc = 0; cc < D / 32; ++cc) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + cc * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              __stcg(reinterpret_cast<float4 *>(mine) + (cc * 8 + q) * kQRows + row_local,
+                     make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]), __uint_as_float(v[q * 4 + 2]),
+                                 __uint_as_float(v[q * 4 + 3])));
+          }
+          __stcg(mine + D * kQRows + row_local, m_ref);
+          __stcg(mine + (D + 1) * kQRows + row_local, l_run);
+          __threadfence();
+          if (t == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
+          if (row_local == 0) merge_last[t] = (atomicAdd(p.counters + tslot, 1) == splits - 1) ? 1 : 0;
+          if (t == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
+          if (merge_last[t]) {
+            __threadfence();
+            const float *base = p.part + static_cast<size_t>(tslot) * splits * per_split;
+            float m_all = -INFINITY;
+            for (int s2 = 0; s2 < splits; ++s2) m_all = fmaxf(m_all, __ldcg(base + s2 * per_split + D * kQRows + row_local));
+            float l_all = 0.f;
+            for (int s2 = 0; s2 < splits; ++s2) {
+              const float *ps = base + s2 * per_split;
+              l_all += __ldcg(ps + (D + 1) * kQRows + row_local) * exp2f((__ldcg(ps + D * kQRows + row_local) - m_all) * c);
+            }
+            const float inv_l = 1.0f / l_all;
+#pragma unroll 1
+            for (int cc = 0; cc < D / 32; ++cc) {
+              float o[32];
+#pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = 0.f;
+              for (int s2 = 0; s2 < splits; ++s2) {                 // fixed order: the sum does not depend on timing
+                const float *ps = base + s2 * per_split;
+                const float w = exp2f((__ldcg(ps + D * kQRows + row_local) - m_all) * c);
+                const float4 *src = reinterpret_cast<const float4 *>(ps) + cc * 8 * kQRows + row_local;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                  const float4 v = __ldcg(src + q * kQRows);
+                  o[q * 4] = fmaf(w, v.x, o[q * 4]);
+                  o[q * 4 + 1] = fmaf(w, v.y, o[q * 4 + 1]);
+                  o[q * 4 + 2] = fmaf(w, v.z, o[q * 4 + 2]);
+                  o[q * 4 + 3] = fmaf(w, v.w, o[q * 4 + 3]);
+                }
+              }
+              if (rib < p.r) store_chunk(cc, o, inv_l);
+            }
+            if (row_local == 0) p.counters[tslot] = 0;               // ready for the next launch
           }
         }
       }
@@ -329,8 +397,24 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   using Cfg = AttnCfg<D>;
   cudaError_t err = set_attr<D>();
   if (err != cudaSuccess) return err;
-  dim3 grid((a.r + 2 * kQRows - 1) / (2 * kQRows), a.H, a.B_eff);
+  const int splits = a.kv_splits > 1 ? a.kv_splits : 1;
+  dim3 grid((a.r + 2 * kQRows - 1) / (2 * kQRows) * splits, a.H, a.B_eff);
   return launch_pdl(attention_kernel<D>, grid, dim3(kAttnThreads), Cfg::kSmemBytes, st, tmQ, tmK, tmV, a);
+}
+
+int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms, size_t scratch_bytes, int max_counters) {
+  const int qtiles = (r + 2 * kQRows - 1) / (2 * kQRows);
+  const long long ctas = static_cast<long long>(qtiles) * H * B_eff;
+  const int nkv = (L + kKeys - 1) / kKeys;
+  if (ctas * 2 > num_sms || nkv < 8) return 1;            // enough CTAs already, or too few key blocks to share
+  int splits = static_cast<int>(num_sms / ctas);
+  if (splits > nkv / 4) splits = nkv / 4;                  // at least four key blocks per range
+  if (splits > 16) splits = 16;
+  while (splits > 1 && (static_cast<size_t>(ctas) * 2 * splits * (D + 2) * kQRows * 4 > scratch_bytes || ctas * 2 > max_counters))
+    --splits;
+  if (splits < 2) return 1;
+  const int per = (nkv + splits - 1) / splits;
+  return (nkv + per - 1) / per;                            // every range gets at least one block
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,

@@ -796,7 +796,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         if ((s = run_gemm(ctx, EPI_QKV, ctx->y_map, blk, W_QKV, ga, "qkv gemm")) != FVAR_OK) return s;
       }
       {
-        AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, ctx->split_partial,
+                    ctx->split_counters};
+        aa.kv_splits = attention_pick_splits(E, H, r, D, L_prev + r, ctx->num_sms, kSplitScratchBytes, kSplitCounters);
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * (L_prev + r) * C, 4.0 * E * (L_prev + r) * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
         ctx->launched();
@@ -818,7 +820,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         GemmArgs gq = gemm_args(R, C, C);
         gq.out_bf16 = ctx->q; gq.ld_out = C;
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
-        AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status};
+        AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, nullptr, nullptr};
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
         ctx->launched();
@@ -1034,7 +1036,7 @@ fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B,
       !tmap_3d(&tv, Vt, L_cap, D, BH, L_cap, static_cast<uint64_t>(L_cap) * D, 64, D))
     return kfail(FVAR_EINVAL, "attention: operands must be 16-byte aligned");
   AttnArgs a{B, H, r, D, L, L_cap, 1, 0, static_cast<bf16 *>(out), 1.4426950408889634f / sqrtf(static_cast<float>(D)),
-             kernel_status_ptr()};
+             kernel_status_ptr(), 1, nullptr, nullptr};
   if (!a.status) return kfail(FVAR_ECUDA, "attention: status word");
   FK_CUDA(launch_attention(tq, tk, tv, a, static_cast<cudaStream_t>(stream)), "attention");
   return FVAR_OK;
