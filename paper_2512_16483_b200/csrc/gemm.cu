@@ -391,7 +391,8 @@ void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits
     if (forced_block_n() && cand[i] != forced_block_n()) continue;
     const long long tiles = static_cast<long long>(tiles_m_total) * ((N + cand[i] - 1) / cand[i]);
     for (int sp = 1; sp <= max_splits; sp *= 2) {
-      if (sp > 1 && (num_kb / sp < 8 || tiles > 4096 ||
+      // splitting pays only for long reductions that would otherwise leave most SMs idle (measured)
+      if (sp > 1 && (num_kb < 64 || tiles * sp > num_sms || tiles > 4096 ||
                      static_cast<size_t>(tiles) * sp * kBlockM * cand[i] * 4 > scratch_bytes))
         break;
       const long long waves = (tiles * sp + num_sms - 1) / num_sms;
