@@ -20,6 +20,12 @@ __host__ __device__ constexpr int k_atoms(int bn) { return bn <= 128 ? 2 : 1; }
 constexpr int kGemmThreads = 192;
 constexpr int kSmemBudget = 196608;     // bytes of operand stages per CTA (192 KiB)
 
+#ifdef FVAR_TRACE
+// Debug build only (-DFVAR_TRACE): CTA 0 records, per K stage, the cycles its producer spent waiting
+// for a free slot / issuing the copies and its MMA thread spent waiting for data / issuing.
+__device__ long long g_gemm_trace[4 * 1024];
+#endif
+
 template <int BN>
 struct GemmCfg {
   static constexpr int kAtomBytesA = kBlockM * kBlockK * 2;
@@ -217,7 +223,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int row_w = e * p.b_batch_rows + n_idx * BN;
         const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
+#ifdef FVAR_TRACE
+          const long long tr0 = clock64();
+#endif
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+#ifdef FVAR_TRACE
+          const long long tr1 = clock64();
+#endif
           mbar_expect_tx(full_bar(stage), a_tx_bytes + Cfg::kStageBytesB);
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
 #pragma unroll
@@ -229,6 +241,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           armed |= 1u << stage;
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == S) { stage = 0; phase ^= 1u; }
+#ifdef FVAR_TRACE
+          if (blockIdx.x == 0 && work == 0 && kb - kb0 < 1024) {
+            g_gemm_trace[4 * (kb - kb0)] = tr1 - tr0;
+            g_gemm_trace[4 * (kb - kb0) + 1] = clock64() - tr1;
+          }
+#endif
         }
       }
       if (!ok) {
@@ -241,8 +259,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {
       // ---------------------------------------------------------------- MMA issuer
+      // The whole warp walks the loop (so that stage counters, addresses and descriptors are
+      // warp-uniform values); one elected lane issues the MMAs and the commits.
+      const bool leader = elect_one();
       constexpr uint32_t idesc = umma_idesc_bf16(kBlockM, BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -253,25 +274,49 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         const int a = it & 1;
         const uint32_t aphase = (it >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag));
+        if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, p.status, &abort_flag)) { ok = false; break; }
+#ifdef FVAR_TRACE
+          const long long tr0 = clock64();
+#endif
+          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, p.status, &abort_flag));
+          if (!ok) break;
+#ifdef FVAR_TRACE
+          const long long tr1 = clock64();
+#endif
           tc_fence_after();
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
+          // descriptors are computed by the whole warp (warp-uniform values); only the issue is elected
+          uint64_t da[kKAtoms], db[kKAtoms];
 #pragma unroll
           for (int ka = 0; ka < kKAtoms; ++ka) {
-            const uint64_t da = smem_desc_sw128(sa + ka * Cfg::kAtomBytesA);
-            const uint64_t db = smem_desc_sw128(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB);
+            da[ka] = smem_desc_sw128(sa + ka * Cfg::kAtomBytesA);
+            db[ka] = smem_desc_sw128(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB);
+          }
+          const uint32_t acc_first = (kb > kb0) ? 1u : 0u;
+          if (leader) {
+#pragma unroll
+          for (int ka = 0; ka < kKAtoms; ++ka) {
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)
-              umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb > kb0) || (ka != 0) || (k != 0));
+              umma_bf16(d_tmem, da[ka] + 2 * k, db[ka] + 2 * k, idesc, (ka != 0 || k != 0) ? 1u : acc_first);
           }
           umma_commit(empty_bar(stage));
+          }
+          __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
+#ifdef FVAR_TRACE
+          if (leader && blockIdx.x == 0 && work == 0 && kb - kb0 < 1024) {
+            g_gemm_trace[4 * (kb - kb0) + 2] = tr1 - tr0;
+            g_gemm_trace[4 * (kb - kb0) + 3] = clock64() - tr1;
+          }
+#endif
         }
-        if (ok) umma_commit(tfull_bar(a));
+        if (ok && leader) umma_commit(tfull_bar(a));
+        __syncwarp();
       }
     }
   } else {
@@ -315,6 +360,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           uint32_t acc[32];
           tmem_ld32(taddr + c * 32, acc);
           tmem_ld_wait();
+          if (row < p.R)                       // rows past the end carry nothing anybody reads
 #pragma unroll
           for (int q = 0; q < 8; ++q)
             __stcg(mine + (c * 8 + q) * kBlockM,
@@ -337,7 +383,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             float sum[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) sum[i] = 0.f;
-            for (int s2 = 0; s2 < splits; ++s2) {
+            for (int s2 = 0; s2 < splits && row < p.R; ++s2) {
               const float4 *src = base + static_cast<size_t>(s2) * (kBlockM * BN / 4) + c * 8 * kBlockM;
 #pragma unroll
               for (int q = 0; q < 8; ++q) {
@@ -407,6 +453,12 @@ void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits
     }
   }
 }
+
+#ifdef FVAR_TRACE
+extern "C" int fvar_debug_read_gemm_trace(long long *host, int n) {
+  return cudaMemcpyFromSymbol(host, g_gemm_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms) {
   int bn, sp;
