@@ -289,11 +289,96 @@ __global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__
   }
 }
 
+// Warp-per-row variant for C <= 256 * T: the row lives in the registers of one warp (T groups of 8
+// elements per lane), statistics by shuffles only, no block-wide barrier; 8 rows per CTA.
+template <int T>
+__global__ void __launch_bounds__(256) ln_modulate_warp_kernel(const float *__restrict__ x, RowMap xmap, int rows, int total_rows,
+                                                               int C, const float *__restrict__ shift,
+                                                               const float *__restrict__ scale, long long vec_stride,
+                                                               int bmul, int boff, const bf16 *__restrict__ gamma, float eps,
+                                                               bf16 *__restrict__ y) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int grow = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (grow >= total_rows) return;
+  const int lane = threadIdx.x & 31;
+  const int e = grow / rows, j = grow - e * rows;
+  const float *xr = x + (static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb + j) * C;
+  bf16 *yr = y + static_cast<long long>(grow) * C;
+  const int nvec = C / 8;
+  float v[T][8];
+  float sum = 0.f;
+#pragma unroll
+  for (int t = 0; t < T; ++t) {
+    const int g = lane + t * 32;
+    if (g < nvec) {
+      const float4 a = __ldg(reinterpret_cast<const float4 *>(xr) + 2 * g), c = __ldg(reinterpret_cast<const float4 *>(xr) + 2 * g + 1);
+      v[t][0] = a.x; v[t][1] = a.y; v[t][2] = a.z; v[t][3] = a.w;
+      v[t][4] = c.x; v[t][5] = c.y; v[t][6] = c.z; v[t][7] = c.w;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sum += v[t][i];
+    }
+  }
+  const float mean = warp_sum(sum) / C;
+  float sq = 0.f;
+#pragma unroll
+  for (int t = 0; t < T; ++t)
+    if (lane + t * 32 < nvec) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float d = v[t][i] - mean;
+        sq = fmaf(d, d, sq);
+      }
+    }
+  const float rstd = rsqrtf(warp_sum(sq) / C + eps);
+  const long long voff = static_cast<long long>(e * bmul + boff) * vec_stride;
+#pragma unroll
+  for (int t = 0; t < T; ++t) {
+    const int g = lane + t * 32;
+    if (g < nvec) {
+      float o[8];
+      if (gamma != nullptr) {
+        const uint4 gu = __ldg(reinterpret_cast<const uint4 *>(gamma) + g);
+        const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&gu);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 gf = __bfloat1622float2(gh[i]);
+          o[2 * i] = (v[t][2 * i] - mean) * rstd * gf.x;
+          o[2 * i + 1] = (v[t][2 * i + 1] - mean) * rstd * gf.y;
+        }
+      } else {
+        const float4 *sc = reinterpret_cast<const float4 *>(scale + voff) + 2 * g;
+        const float4 *sh = reinterpret_cast<const float4 *>(shift + voff) + 2 * g;
+        const float4 s0 = __ldg(sc), s1 = __ldg(sc + 1), h0 = __ldg(sh), h1 = __ldg(sh + 1);
+        const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        const float shv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o[i] = fmaf((v[t][i] - mean) * rstd, 1.0f + scv[i], shv[i]);
+      }
+      uint32_t w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&h2);
+      }
+      reinterpret_cast<uint4 *>(yr)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
 cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int C, const float *shift,
                                const float *scale, long long vec_stride, int bmul, int boff, const bf16 *gamma,
                                float eps, bf16 *y, cudaStream_t st) {
   if (E * rows <= 0) return cudaSuccess;
   if (C % 8 != 0 || C > 8 * kLnThreads * kLnMaxVec) return cudaErrorInvalidValue;
+  const int total = E * rows;
+  // few rows: a CTA per row finishes sooner (more threads per row); many rows: a warp per row streams better
+  if (total >= 4096 && C <= 1024)
+    return launch_pdl(ln_modulate_warp_kernel<4>, dim3((total + 7) / 8), dim3(256), 0, st, x, xmap, rows, total, C, shift, scale,
+                      vec_stride, bmul, boff, gamma, eps, y);
+  if (total >= 4096 && C <= 2048)
+    return launch_pdl(ln_modulate_warp_kernel<8>, dim3((total + 7) / 8), dim3(256), 0, st, x, xmap, rows, total, C, shift, scale,
+                      vec_stride, bmul, boff, gamma, eps, y);
   return launch_pdl(ln_modulate_kernel, dim3(E * rows), dim3(kLnThreads), 0, st, x, xmap, rows, C, shift, scale, vec_stride, bmul, boff, gamma,
                                                       eps, y);
 }
@@ -326,6 +411,7 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
   const float4 *p11 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y1) * w0 + x1) * C);
   float4 *dst = reinterpret_cast<float4 *>(out + (static_cast<long long>(b) * M1 + i) * C);
   const float w00 = (1.f - fy) * (1.f - fx), w01 = (1.f - fy) * fx, w10 = fy * (1.f - fx), w11 = fy * fx;
+#pragma unroll 4
   for (int c = threadIdx.x & 31; c < C / 4; c += 32) {
     const float4 a = __ldg(p00 + c), bq = __ldg(p01 + c), cq = __ldg(p10 + c), d = __ldg(p11 + c);
     float4 o;
@@ -333,7 +419,7 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
     o.y = w00 * a.y + w01 * bq.y + w10 * cq.y + w11 * d.y;
     o.z = w00 * a.z + w01 * bq.z + w10 * cq.z + w11 * d.z;
     o.w = w00 * a.w + w01 * bq.w + w10 * cq.w + w11 * d.w;
-    dst[c] = o;
+    __stcs(dst + c, o);                          // written once, read by a later kernel: stream it
   }
 }
 
@@ -349,37 +435,38 @@ cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int 
 // Transposed two-term bf16 split of the fp32 rows for the projection GEMM:
 // xt[e][c][m] = hi(x[row(e, m)][c]) and xt[e][c][Mk + m] = lo(...), hi = bf16(x), lo = bf16(x - hi),
 // so that the tensor-core product Q^T (hi + lo) carries ~16 mantissa bits of x.  Mk = M rounded up
-// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  32 x 32 tiles
-// through shared memory.
+// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  64 x 32 tiles
+// through shared memory, two tokens (one bf16x2) per lane on the way out.
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
                                                              int Mk, bf16 *__restrict__ xt) {
   pdl_wait();
   pdl_launch_dependents();
-  __shared__ float tile[32][33];
-  const int e = blockIdx.z, m0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  __shared__ float tile[64][33];                 // 64 token rows x 32 channels
+  const int e = blockIdx.z, m0 = blockIdx.x * 64, c0 = blockIdx.y * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const float *src = x + static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb * C;
-  for (int k = ty; k < 32; k += 8) {
+  for (int k = ty; k < 64; k += 8) {
     const int m = m0 + k, c = c0 + tx;
     tile[k][tx] = (m < M && c < C) ? src[static_cast<long long>(m) * C + c] : 0.f;
   }
   __syncthreads();
   bf16 *dst = xt + static_cast<long long>(e) * C * 2 * Mk;
-  for (int k = ty; k < 32; k += 8) {
-    const int c = c0 + k, m = m0 + tx;
-    if (c < C && m < Mk) {
-      const float v = tile[tx][k];
-      const bf16 hi = __float2bfloat16_rn(v);
-      const bf16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-      dst[static_cast<long long>(c) * 2 * Mk + m] = hi;
-      dst[static_cast<long long>(c) * 2 * Mk + Mk + m] = lo;
+  for (int k = ty; k < 32; k += 8) {             // one channel per warp pass; each lane writes two tokens
+    const int c = c0 + k, m = m0 + 2 * tx;
+    if (c < C) {                                 // m + 1 < Mk always: Mk is a multiple of 64
+      const float v0 = tile[2 * tx][k], v1 = tile[2 * tx + 1][k];
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
+      const float2 hf = __bfloat1622float2(hi);
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - hf.x, v1 - hf.y);
+      *reinterpret_cast<__nv_bfloat162 *>(dst + static_cast<long long>(c) * 2 * Mk + m) = hi;
+      *reinterpret_cast<__nv_bfloat162 *>(dst + static_cast<long long>(c) * 2 * Mk + Mk + m) = lo;
     }
   }
 }
 
 cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
                                   cudaStream_t st) {
-  dim3 grid((Mk + 31) / 32, (C + 31) / 32, E);
+  dim3 grid(Mk / 64, (C + 31) / 32, E);
   return launch_pdl(transpose_bf16_kernel, dim3(grid), dim3(256), 0, st, x, xmap, M, C, Mk, xt);
 }
 
