@@ -63,6 +63,11 @@ def scale_plan(wl, shp):
     return plan
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel class, from the ncu capture
+# summarised in profiles/launches_var_d16_late3_b16.md (None: not captured for this workload / kernel changed since)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"var_d16_late3_b16": 9.72e6}
+
+
 def make_shape(name):
     return {"d16": si.shape_var_d16, "d30": si.shape_var_d30, "inf2b": si.shape_infinity_2b}[name]()
 
@@ -370,7 +375,8 @@ def main():
     roofline = {"bound": "tensor", "kernel": "gemm_kernel (every tile width and epilogue the step launches)",
                 "achieved": g["tflops"], "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                 "frac": g["tflops"] / pk["bf16_sustained"], "peak_source": pk["source"] + ", sustained bf16",
-                "traffic": None, "how": "separate pass of %d steps with CUDA events around every launch" % prof_steps,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload), "traffic_unit": "bytes per launch (ncu, cold cache)",
+                "algorithmic_bytes_per_launch": (g["gbs"] * 1e9 * g["avg_us"] * 1e-6) if "gbs" in g else None, "how": "separate pass of %d steps with CUDA events around every launch" % prof_steps,
                 "classes": classes}
     line = {
         "metric": metric, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,
