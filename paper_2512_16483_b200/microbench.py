@@ -1,0 +1,107 @@
+"""Stand-alone timings of the library's kernels through the C ABI (CUDA events, one GPU).
+
+    python -m paper_2512_16483_b200.microbench gemm        # tile-width sweep: FVAR_GEMM_BLOCK_N=64|128|256 forces a width
+    python -m paper_2512_16483_b200.microbench attention
+    python -m paper_2512_16483_b200.microbench memory      # score, LayerNorm + modulate, restoration fill, selection
+
+GEMM calls rotate over several weight copies (more than L2 holds) and are captured in one CUDA graph so
+that host launch cost does not enter the time.
+"""
+from __future__ import annotations
+
+import os
+import sys
+
+import torch
+
+from . import binding as fv
+
+
+def _time(fn, n=20, warm=3):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / n          # microseconds
+
+
+def gemm():
+    lib = fv.load_library()
+    bn = os.environ.get("FVAR_GEMM_BLOCK_N", "auto")
+    shapes = [(1024, 3072, 1024), (1024, 1024, 1024), (1024, 4096, 1024), (1024, 1024, 4096), (400, 3072, 1024),
+              (16, 2048, 2048), (16, 2048, 8192), (336, 8192, 2048), (4096, 4096, 1024), (8192, 8192, 2048),
+              (16384, 4096, 4096)]
+    for R, N, K in shapes:
+        ncopy = max(2, min(32, int(300e6 // (N * K * 2))))
+        A = torch.randn(R, K, device="cuda").bfloat16()
+        Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(ncopy)]
+        out = torch.empty(R, N, device="cuda", dtype=torch.float32)
+
+        def call(i):
+            lib.fvar_gemm_bf16(A.data_ptr(), Ws[i % ncopy].data_ptr(), None, R, N, K, out.data_ptr(),
+                               torch.cuda.current_stream().cuda_stream)
+        for i in range(ncopy):
+            call(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(ncopy):
+                call(i)
+        us = _time(g.replay, n=5, warm=1) / ncopy
+        print("BN=%s R=%d N=%d K=%d: %.2f us  %.1f TFLOP/s  weights %.0f GB/s" % (
+            bn, R, N, K, us, 2 * R * N * K / us / 1e6, N * K * 2 / us / 1e3))
+
+
+def attention():
+    lib = fv.load_library()
+    cases = [(2, 16, 128, 4096, 10521, 10624), (2, 16, 128, 1600, 4121, 4224), (2, 16, 128, 4096, 256, 256),
+             (16, 16, 64, 256, 680, 768), (32, 30, 64, 256, 680, 768), (8, 16, 64, 128, 552, 768),
+             (1, 16, 128, 170, 6595, 10624)]
+    for B, H, D, r, L, Lc in cases:
+        C = H * D
+        q = torch.randn(B, r, C, device="cuda").bfloat16()
+        Kc = torch.randn(B, H, Lc, D, device="cuda").bfloat16()
+        Vt = torch.randn(B, H, D, Lc, device="cuda").bfloat16()
+        out = torch.empty_like(q)
+        us = _time(lambda: lib.fvar_attention(q.data_ptr(), Kc.data_ptr(), Vt.data_ptr(), B, H, r, D, L, Lc,
+                                              out.data_ptr(), torch.cuda.current_stream().cuda_stream), n=10)
+        print("B=%d H=%d D=%d r=%d L=%d: %.1f us  %.1f TFLOP/s  K/V %.0f GB/s" % (
+            B, H, D, r, L, us, 4.0 * B * r * L * C / us / 1e6, 4.0 * B * L * C / us / 1e3))
+    assert fv.kernel_poll_status() == fv.OK
+
+
+def memory():
+    for B, M, C in [(2, 4096, 2048), (32, 4096, 2048), (32, 1600, 1024)]:
+        xs = [torch.randn(B, M, C, device="cuda") for _ in range(2)]
+        k = [0]
+
+        def nxt():
+            k[0] += 1
+            return xs[k[0] % 2]
+        us = _time(lambda: fv.fvar_row_scores(nxt()))
+        print("row_scores   B=%d M=%d C=%d: %.1f us  %.0f GB/s" % (B, M, C, us, B * M * C * 4 / us / 1e3))
+        sh, sc = torch.randn(B, C, device="cuda"), torch.randn(B, C, device="cuda")
+        us = _time(lambda: fv.fvar_ln_modulate(nxt(), sh, sc, 1e-6))
+        print("ln_modulate  B=%d M=%d C=%d: %.1f us  %.0f GB/s" % (B, M, C, us, B * M * C * 6 / us / 1e3))
+        if M == 4096:
+            prev = torch.randn(B, 2304, C, device="cuda")
+            out = torch.empty(B, M, C, device="cuda")
+            inv = torch.full((B, M), -1, dtype=torch.int32, device="cuda")
+            inv[:, ::24] = 1
+            us = _time(lambda: fv.fvar_rtr_fill(prev, (48, 48), (64, 64), inv, out))
+            nfill = int((inv < 0).sum().item())
+            print("rtr_fill     B=%d M=%d C=%d: %.1f us  %.0f GB/s (rows written once + cache read once)" % (
+                B, M, C, us, (nfill * C * 4 + B * 2304 * C * 4) / us / 1e3))
+        s = torch.rand(B, M, device="cuda")
+        us = _time(lambda: fv.fvar_select_topr(s, M // 4))
+        print("select_topr  B=%d M=%d r=%d: %.1f us (includes ~10 us of host call overhead)" % (B, M, M // 4, us))
+
+
+if __name__ == "__main__":
+    which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
+    {"gemm": gemm, "attention": attention, "memory": memory}[which]()
