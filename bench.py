@@ -68,6 +68,21 @@ def scale_plan(wl, shp):
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {"var_d16_late3_b16": 9.72e6}
 
 
+def max_over_ranks(ms_local, dist, device):
+    """Replicas only: every rank runs the same independent workload; the job's time is the slowest rank's."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_per_step, steps, world, ms_total_max):
+    """Whole-job throughput: all ranks' units over the max-over-ranks time of `steps` steps."""
+    return world * units_per_rank_per_step * steps / (ms_total_max * 1e-3)
+
+
 def make_shape(name):
     return {"d16": si.shape_var_d16, "d30": si.shape_var_d30, "inf2b": si.shape_infinity_2b}[name]()
 
@@ -334,11 +349,7 @@ def main():
             fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
         return ms, ctx.launch_count() - n0
 
     warm = max(args.warmup, 3)
@@ -369,8 +380,8 @@ def main():
 
     pk = peaks()
     ms_step = ms_total / args.steps
-    value = world * tokens_per_step / (ms_step * 1e-3)
-    e2e = world * tokens_per_step / (ms_e2e / args.steps * 1e-3)
+    value = whole_job_value(tokens_per_step, args.steps, world, ms_total)
+    e2e = whole_job_value(tokens_per_step, args.steps, world, ms_e2e)
     g = classes.get("gemm", {"tflops": 0.0})
     roofline = {"bound": "tensor", "kernel": "gemm_kernel (every tile width and epilogue the step launches)",
                 "achieved": g["tflops"], "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
