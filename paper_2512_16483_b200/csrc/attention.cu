@@ -142,15 +142,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       // ---------------------------------------------------------------- MMA issuer
       constexpr uint32_t idesc_s = umma_idesc_bf16(kQRows, kKeys);
       constexpr uint32_t idesc_o = umma_idesc_bf16(kQRows, D);
-      auto issue_s = [&](int t, int slot) {          // S_t = Q_t K^T
+      auto issue_s = [&](int t, int buf, int slot) {   // S buffer `buf` = Q_t K^T
         const uint32_t ks = ring_smem + slot * Cfg::kTileBytes, qs = q_smem + t * Cfg::kTileBytes;
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
           const uint64_t da = smem_desc_sw128(qs + (k / 4) * kAtomBytes) + 2 * (k % 4);
           const uint64_t db = smem_desc_sw128(ks + (k / 4) * kAtomBytes) + 2 * (k % 4);
-          umma_bf16(tmem_base + t * kKeys, da, db, idesc_s, k != 0);
+          umma_bf16(tmem_base + buf * kKeys, da, db, idesc_s, k != 0);
         }
-        umma_commit(s_full(t));
+        umma_commit(s_full(buf));
       };
       auto issue_pv = [&](int t, int slot, bool accumulate) {   // O_t (+)= P_t V
         const uint32_t vs = ring_smem + slot * Cfg::kTileBytes, ps = p_smem + t * Cfg::kPTile;
@@ -166,9 +166,27 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (ok) ok = mbar_wait(ring_full(0), 0, p.status, &abort_flag);
       if (ok) {
         tc_fence_after();
-        for (int t = 0; t < ntiles; ++t) issue_s(t, 0);
+        for (int t = 0; t < ntiles; ++t) issue_s(t, t, 0);
         umma_commit(ring_empty(0));
       }
+      if (ntiles == 1) {
+        // A single query tile has no partner to alternate with: the idle tile's S columns serve as
+        // a second S buffer, so that Q K^T of block j+1 runs while the softmax works on block j.
+        for (int j = 0; ok && j < nkv; ++j) {
+          const int vi = 2 * j + 1, ki = 2 * j + 2;
+          if (j + 1 < nkv) {
+            if (!mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            issue_s(0, (j + 1) & 1, ki % NR);
+            umma_commit(ring_empty(ki % NR));
+          }
+          if (!mbar_wait(p_full(0), j & 1u, p.status, &abort_flag)) { ok = false; break; }
+          if (!mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(0, vi % NR, j > 0);
+          umma_commit(ring_empty(vi % NR));
+        }
+      } else
       for (int j = 0; ok && j < nkv; ++j) {
         const int vi = 2 * j + 1, ki = 2 * j + 2;
         for (int t = 0; ok && t < ntiles; ++t) {
@@ -180,7 +198,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (j + 1 < nkv) {
             if (t == 0 && !mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
             tc_fence_after();
-            issue_s(t, ki % NR);
+            issue_s(t, t, ki % NR);
             if (t == ntiles - 1) umma_commit(ring_empty(ki % NR));
           }
         }
@@ -193,7 +211,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const int quad = warp & 3;                         // TMEM lanes [32 * quad, 32 * quad + 32)
       const int row_local = quad * 32 + lane;
       const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-      const uint32_t s_addr = tmem_base + t * kKeys + lane_addr;
+      const bool single = (ntiles == 1);               // then S alternates between the two S buffers
+      const uint32_t s_base = tmem_base + lane_addr;
       const uint32_t o_addr = tmem_base + 256 + t * D + lane_addr;
       const uint32_t p_row = p_smem + t * Cfg::kPTile + row_local * 128;
       const float c = p.scale_log2;
@@ -201,7 +220,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       bool ok = true;
 
       for (int j = 0; j < nkv; ++j) {
-        ok = __all_sync(0xffffffffu, mbar_wait(s_full(t), j & 1u, p.status, &abort_flag));
+        const int sbuf = single ? (j & 1) : t;
+        const uint32_t s_addr = s_base + sbuf * kKeys;
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full(sbuf), (single ? (j >> 1) : j) & 1u, p.status, &abort_flag));
         if (!ok) break;
         tc_fence_after();
         const int valid = p.L - (jb0 + j) * kKeys;       // keys of this block below L (>= 128: all)
