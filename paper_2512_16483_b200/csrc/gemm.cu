@@ -60,7 +60,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Epilogue for one thread: one output row, 32 consecutive columns starting at col0 (col0 % 32 == 0).
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t (&acc)[32], int batch, int row,
-                                               int col0) {
+                                               int col0, const float4 *resid_pre = nullptr) {
   float v[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
@@ -139,7 +139,7 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t
     const float *g = p.gate ? p.gate + static_cast<long long>(b) * p.gate_stride + col0 : nullptr;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-      float4 r4 = reinterpret_cast<const float4 *>(res)[q];
+      float4 r4 = resid_pre ? resid_pre[q] : reinterpret_cast<const float4 *>(res)[q];
       float4 g4 = g ? __ldg(reinterpret_cast<const float4 *>(g) + q) : make_float4(1.f, 1.f, 1.f, 1.f);
       float4 o;
       o.x = fmaf(g4.x, v[q * 4], r4.x);
@@ -330,22 +330,44 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
       const int a = it & 1;
       const uint32_t aphase = (it >> 1) & 1u;
+      const int row_local = quad * 32 + lane;
+      const int row = m_idx * kBlockM + row_local;
+      // The residual rows of the first two column chunks are fetched while the main loop still runs:
+      // with one tile per CTA nothing else hides that latency.
+      constexpr int kPre = (BN / 32 < 2) ? BN / 32 : 2;
+      float4 pre[kPre][8];
+      bool have_pre = false;
+      if constexpr (EPI == EPI_RESID) {
+        if (splits == 1 && row < p.R) {
+          const int e2 = row / p.rows_per_batch, j2 = row - e2 * p.rows_per_batch;
+          const float *res = p.resid + (static_cast<long long>(e2 * p.rmap.bmul + p.rmap.boff) * p.rmap.rpb + j2) * p.ld_out + n_idx * BN;
+#pragma unroll
+          for (int c = 0; c < kPre; ++c)
+            if (n_idx * BN + c * 32 < p.N) {
+#pragma unroll
+              for (int q = 0; q < 8; ++q) pre[c][q] = reinterpret_cast<const float4 *>(res + c * 32)[q];
+            }
+          have_pre = true;
+        }
+      }
       ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag));
       if (!ok) break;
       tc_fence_after();
-      const int row_local = quad * 32 + lane;
-      const int row = m_idx * kBlockM + row_local;
       const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
       if (splits == 1) {
-#pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        auto do_chunk = [&](int c, const float4 *prep) {
           const int col0 = n_idx * BN + c * 32;
-          if (col0 >= p.N) break;                // uniform across the warp
-          uint32_t acc[32];
-          tmem_ld32(taddr + c * 32, acc);
-          tmem_ld_wait();
-          if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0);
-        }
+          if (col0 < p.N) {                      // uniform across the warp
+            uint32_t acc[32];
+            tmem_ld32(taddr + c * 32, acc);
+            tmem_ld_wait();
+            if (row < p.R) epilogue_chunk<EPI>(p, acc, e, row, col0, prep);
+          }
+        };
+#pragma unroll
+        for (int c = 0; c < kPre; ++c) do_chunk(c, have_pre ? pre[c] : nullptr);
+#pragma unroll 1
+        for (int c = kPre; c < BN / 32; ++c) do_chunk(c, nullptr);
         tc_fence_before();
         mbar_arrive(tempty_bar(a));
       } else {
