@@ -111,6 +111,15 @@ def select_top_r(scores: np.ndarray, r: int) -> np.ndarray:
     return np.array(sorted(order[:r]), dtype=np.int32)
 
 
+def sampling_keys(scores: np.ndarray, noise: np.ndarray) -> np.ndarray:
+    """Keys for drawing rows without replacement with probability proportional to the row score
+    (Sec. 3.3 RTR: "each row i chosen with probability P_i" proportional to ||F^(i)||^2): with
+    E_i ~ Exp(1) independent, the r largest s_i / E_i are a sample without replacement in which the
+    first pick is row i with probability s_i / sum_j s_j (exponential race).  The noise E is an
+    input; the keys are one fp32 division each, the precision the kernel decides in."""
+    return (np.asarray(scores, dtype=np.float32) / np.asarray(noise, dtype=np.float32)).astype(np.float32)
+
+
 def random_projection(Q: np.ndarray, X: np.ndarray) -> np.ndarray:
     """F_r = Q^T X: [r][C] from Q [M][r] and X [M][C] (Algorithm 1, RP step)."""
     return Q.T @ X
@@ -223,12 +232,13 @@ class Policy:
     """Per-call policy of a scale step (mirrors the C ABI's keep policy)."""
 
     def __init__(self, mode: str = "dense", cfg_mode: str = "pair", keep_ratio: float = 1.0,
-                 rank_per_group: Optional[Sequence[int]] = None, forced_indices=None):
+                 rank_per_group: Optional[Sequence[int]] = None, forced_indices=None, sample_noise=None):
         assert mode in ("dense", "lowrank_rtr", "skip")
         assert cfg_mode in ("pair", "null_only")
         self.mode, self.cfg_mode = mode, cfg_mode
         self.keep_ratio, self.rank_per_group = keep_ratio, rank_per_group
         self.forced_indices = forced_indices      # [B_eff][G] -> int array, or None
+        self.sample_noise = sample_noise          # [G][B_eff][M] Exp(1) variates: sampled selection; None: top-r
 
 
 class Oracle:
@@ -327,6 +337,8 @@ class Oracle:
                 else:
                     if pol.forced_indices is not None:
                         idx = np.asarray(pol.forced_indices[e][g], dtype=np.int32)
+                    elif pol.sample_noise is not None:
+                        idx = select_top_r(sampling_keys(row_scores(X, np.float32), pol.sample_noise[g][e]), r)
                     else:
                         idx = select_top_r(row_scores(X, np.float32), r)
                     x = random_projection(self.proj[(scale_idx, g)], X)

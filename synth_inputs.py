@@ -175,3 +175,9 @@ def make_group_cache(seed: int, G: int, B: int, M_prev: int, C: int) -> np.ndarr
     """Stand-in for the previous scale's block-group outputs: [G][B][M_prev][C], N(0,1) in fp32."""
     rng = np.random.default_rng([seed, 7])
     return rng.standard_normal((G, B, M_prev, C), dtype=np.float32)
+
+
+def make_sample_noise(seed: int, scale_idx: int, G: int, B_eff: int, M: int) -> np.ndarray:
+    """Exp(1) variates [G][B_eff][M] (fp32) for the sampled row selection; one draw per (scale, group, element, row)."""
+    rng = np.random.default_rng([seed, 8, scale_idx])
+    return rng.standard_exponential(size=(G, B_eff, M)).astype(np.float32) + np.float32(1e-30)

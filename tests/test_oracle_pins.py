@@ -453,3 +453,21 @@ def test_forced_indices_are_used():
     forced = [[np.array([0, 2, 5, 8])], [np.array([1, 3, 4, 7])]]
     o.scale_step(toks[1], 1, orc.Policy("lowrank_rtr", rank_per_group=[4], forced_indices=forced))
     assert list(o.last_indices[0][0]) == [0, 2, 5, 8] and list(o.last_indices[1][0]) == [1, 3, 4, 7]
+
+
+def test_sampling_keys_exponential_race():
+    """The first pick of the sampled selection is row i with probability s_i / sum s (property of the
+    exponential race), r picks are distinct, and equal noise reduces the rule to plain top-r."""
+    s = np.array([5.0, 1.0, 3.0, 0.5, 0.5], dtype=np.float32)
+    n = 20000
+    noise = si.make_sample_noise(3, 0, 1, n, 5)[0]
+    first = np.array([orc.select_top_r(orc.sampling_keys(s, noise[t]), 1)[0] for t in range(n)])
+    freq = np.bincount(first, minlength=5) / n
+    expect = s / s.sum()
+    assert np.all(np.abs(freq - expect) < 4 * np.sqrt(expect * (1 - expect) / n) + 1e-3)
+    picks = orc.select_top_r(orc.sampling_keys(s, noise[0]), 3)
+    assert len(set(picks.tolist())) == 3 and list(picks) == sorted(picks)
+    ones = np.ones(5, dtype=np.float32)
+    assert list(orc.select_top_r(orc.sampling_keys(s, ones), 2)) == list(orc.select_top_r(s, 2))
+    k = orc.sampling_keys(np.array([3.0], np.float32), np.array([7.0], np.float32))
+    assert k.dtype == np.float32 and k[0] == np.float32(3.0) / np.float32(7.0)
