@@ -45,6 +45,7 @@ typedef enum {
 
 enum { FVAR_DENSE = 0, FVAR_LOWRANK_RTR = 1, FVAR_SKIP = 2 };      /* fvar_keep_policy.mode     */
 enum { FVAR_CFG_PAIR = 0, FVAR_CFG_NULL_ONLY = 1 };                /* fvar_keep_policy.cfg_mode */
+enum { FVAR_SELECT_TOPR = 0, FVAR_SELECT_SAMPLE = 1 };             /* fvar_keep_policy.select   */
 
 /* Static shape of the block stack. */
 typedef struct {
@@ -83,6 +84,11 @@ typedef struct {
   float keep_ratio;           /* r = floor(keep_ratio * M + 0.5) for every group                   */
   const int *forced_indices;  /* dev, test hook: [n_groups][B_eff][r_max] ascending row indices that
                                  replace the selection (r_max = largest r of the call); NULL in production */
+  int select;                 /* FVAR_SELECT_TOPR: the r highest row scores (default, 0).
+                                 FVAR_SELECT_SAMPLE: r rows drawn without replacement with probability
+                                 proportional to the row score (Sec. 3.3: "each row i chosen with probability
+                                 P_i"): the r largest keys s_i / E_i, E_i ~ Exp(1) given in sample_noise        */
+  const float *sample_noise;  /* dev fp32 [n_groups][B_eff][M] of Exp(1) variates (> 0) for FVAR_SELECT_SAMPLE     */
 } fvar_keep_policy;
 
 /* Bytes of device workspace fvar_init needs for this shape (0 if the shape is invalid). */
@@ -197,6 +203,11 @@ const char *fvar_last_error(const fvar_ctx *ctx);
 /* Row score of Sec. 3.3 (RTR): s[b][i] = sum_c x[b][i][c]^2 (the numerator of p_i; the common
  * denominator ||X||_F^2 does not change the order).  x dev fp32 [B][M][C], C % 4 == 0; scores dev fp32 [B][M]. */
 fvar_status fvar_row_scores(const float *x, int B, int M, int C, float *scores, void *stream);
+
+/* Sampling keys of the row selection: keys[b][i] = s[b][i] / noise[b][i] (one fp32 division, round to
+ * nearest) with s the row score above and noise dev fp32 [B][M] of Exp(1) variates.  Feeding the keys
+ * to fvar_select_topr draws r rows without replacement with probability proportional to s (Sec. 3.3). */
+fvar_status fvar_row_keys(const float *x, const float *noise, int B, int M, int C, float *keys, void *stream);
 
 /* Index set I of Sec. 3.3 / Algorithm 1: per batch element the r highest-scoring rows, ascending.
  * Order: score descending then index ascending; NaN ranks as +inf; -0 == +0.

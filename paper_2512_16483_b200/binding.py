@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libfvar.so")
 OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
+SELECT_TOPR, SELECT_SAMPLE = 0, 1
 OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS = 0, 1
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
@@ -47,7 +48,8 @@ class _Weights(ct.Structure):
 
 class _Policy(ct.Structure):
     _fields_ = [("mode", ct.c_int), ("cfg_mode", ct.c_int), ("rank_per_group", ct.POINTER(ct.c_int)),
-                ("keep_ratio", ct.c_float), ("forced_indices", ct.c_void_p)]
+                ("keep_ratio", ct.c_float), ("forced_indices", ct.c_void_p), ("select", ct.c_int),
+                ("sample_noise", ct.c_void_p)]
 
 
 _lib = None
@@ -88,6 +90,7 @@ def load_library() -> ct.CDLL:
         "fvar_destroy": (None, [vp]),
         "fvar_last_error": (ct.c_char_p, [vp]),
         "fvar_row_scores": (i, [vp, i, i, i, vp, vp]),
+        "fvar_row_keys": (i, [vp, vp, i, i, i, vp, vp]),
         "fvar_select_topr": (i, [vp, i, i, i, vp, vp, vp]),
         "fvar_ln_modulate": (i, [vp, i, i, i, vp, vp, ll, f, vp, vp]),
         "fvar_gemm_bf16": (i, [vp, vp, vp, i, i, i, vp, vp]),
@@ -106,7 +109,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
-            "fvar_row_scores", "fvar_select_topr", "fvar_ln_modulate",
+            "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
             "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
 
@@ -137,6 +140,15 @@ def fvar_row_scores(x: torch.Tensor) -> torch.Tensor:
     s = torch.empty((B, M), dtype=torch.float32, device=x.device)
     _check_kernel(load_library().fvar_row_scores(x.data_ptr(), B, M, C, s.data_ptr(), _stream()))
     return s
+
+
+def fvar_row_keys(x: torch.Tensor, noise: torch.Tensor) -> torch.Tensor:
+    """x fp32 [B][M][C], noise fp32 [B][M] (Exp(1) variates) -> sampling keys fp32 [B][M] = score / noise."""
+    _dev(x, torch.float32), _dev(noise, torch.float32)
+    B, M, C = x.shape
+    k = torch.empty((B, M), dtype=torch.float32, device=x.device)
+    _check_kernel(load_library().fvar_row_keys(x.data_ptr(), noise.data_ptr(), B, M, C, k.data_ptr(), _stream()))
+    return k
 
 
 def fvar_select_topr(scores: torch.Tensor, r: int):
@@ -270,8 +282,11 @@ class Fvar:
         _dev(Qt, torch.bfloat16)
         self._check(self.lib.fvar_set_projection(self.ctx, scale_idx, group, Qt.data_ptr(), Qt.shape[0]))
 
-    def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices):
-        pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None)
+    def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise=None):
+        pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None, SELECT_TOPR, None)
+        if sample_noise is not None:
+            _dev(sample_noise, torch.float32)
+            pol.select, pol.sample_noise = SELECT_SAMPLE, sample_noise.data_ptr()
         keep = []
         if rank_per_group is not None:
             arr = (ct.c_int * len(rank_per_group))(*[int(r) for r in rank_per_group])
@@ -289,10 +304,10 @@ class Fvar:
         return (self.B // 2 if cfg_mode == CFG_NULL_ONLY else self.B, h * w, self.width)
 
     def scale_step(self, tokens: torch.Tensor, scale_idx: int, *, mode: int = DENSE, cfg_mode: int = CFG_PAIR,
-                   keep_ratio: float = 1.0, rank_per_group=None, forced_indices=None,
+                   keep_ratio: float = 1.0, rank_per_group=None, forced_indices=None, sample_noise=None,
                    out: Optional[torch.Tensor] = None) -> Optional[torch.Tensor]:
         _dev(tokens, torch.bfloat16)
-        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, forced_indices)
+        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise)
         if mode == SKIP:
             self._check(self.lib.fvar_scale_step(self.ctx, tokens.data_ptr(), scale_idx, ct.byref(pol), None))
             return None

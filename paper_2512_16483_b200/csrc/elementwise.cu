@@ -15,8 +15,11 @@ __device__ __forceinline__ float warp_sum(float v) {
 // ------------------------------------------------------------------------------------------------
 // Row score s_i = sum_c x[i][c]^2: one warp per row, float4 loads.  Row (e, i) of the compact
 // score array reads row xmap(e, i) of x.
+// With `noise` (Exp(1) variates, one per row) the value written is the sampling key s_i / E_i: the r
+// largest keys are a draw without replacement with probability proportional to s_i.
 __global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict__ x, RowMap xmap, int M,
-                                                         long long rows, int C, float *__restrict__ scores) {
+                                                         long long rows, int C, const float *__restrict__ noise,
+                                                         float *__restrict__ scores) {
   pdl_wait();
   pdl_launch_dependents();
   const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
@@ -33,13 +36,14 @@ __global__ void __launch_bounds__(256) row_scores_kernel(const float *__restrict
     acc = fmaf(v.w, v.w, acc);
   }
   acc = warp_sum(acc);
-  if (lane == 0) scores[row] = acc;
+  if (lane == 0) scores[row] = noise ? __fdiv_rn(acc, noise[row]) : acc;
 }
 
-cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, float *scores, cudaStream_t st) {
+cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, const float *noise, float *scores,
+                              cudaStream_t st) {
   const long long rows = static_cast<long long>(E) * M;
   if (rows <= 0) return cudaSuccess;
-  return launch_pdl(row_scores_kernel, dim3(static_cast<unsigned>((rows + 7) / 8)), dim3(256), 0, st, x, xmap, M, rows, C, scores);
+  return launch_pdl(row_scores_kernel, dim3(static_cast<unsigned>((rows + 7) / 8)), dim3(256), 0, st, x, xmap, M, rows, C, noise, scores);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -665,6 +665,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   if (ctx->B <= 0) return fail(ctx, FVAR_ESTATE, "scale_step before set_cond");
   if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales) return fail(ctx, FVAR_EINVAL, "scale_step: bad scale_idx");
   if (scale_idx < ctx->last_scale) return fail(ctx, FVAR_ESTATE, "scale_step: scale_idx decreased");
+  if (pol->select != FVAR_SELECT_TOPR && pol->select != FVAR_SELECT_SAMPLE) return fail(ctx, FVAR_EINVAL, "scale_step: bad select");
+  const bool sampled = pol->select == FVAR_SELECT_SAMPLE;
+  if (sampled && !pol->sample_noise) return fail(ctx, FVAR_EINVAL, "scale_step: sampled selection needs sample_noise");
   const bool null_only = pol->cfg_mode == FVAR_CFG_NULL_ONLY;
   if (null_only && (ctx->B % 2)) return fail(ctx, FVAR_EINVAL, "scale_step: null-only needs an even batch");
   if (!null_only && ctx->null_only_seen) return fail(ctx, FVAR_ESTATE, "scale_step: pair step after a null-only step");
@@ -742,7 +745,8 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         ctx->launched();
       } else {
         ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
-        FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C, ctx->scores, side), "row_scores");
+        FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C,
+                                       sampled ? pol->sample_noise + static_cast<size_t>(g) * E * M : nullptr, ctx->scores, side), "row_scores");
         ctx->launched();
         ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r));
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, side), "select_topr");
@@ -866,6 +870,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
     std::string key;
     auto put = [&](long long v) { key.append(reinterpret_cast<const char *>(&v), sizeof(v)); };
     put(scale_idx); put(B); put(E); put(prev_slot); put(cur_slot); put(ctx->cache_scale);
+    put(sampled ? static_cast<long long>(reinterpret_cast<uintptr_t>(pol->sample_noise)) : 0);
     for (int g = 0; g < G; ++g) put(rank[g]);
     for (int blk = 0; blk < ctx->cfg.n_blocks; ++blk) put(ctx->len[blk]);
     auto it = ctx->graphs.find(key);
@@ -987,7 +992,13 @@ static fvar_status kfail(fvar_status s, const char *m) { g_init_error = m; retur
 
 fvar_status fvar_row_scores(const float *x, int B, int M, int C, float *scores, void *stream) {
   if (!x || !scores || B <= 0 || M <= 0 || C <= 0 || C % 4) return kfail(FVAR_EINVAL, "row_scores: bad arguments");
-  FK_CUDA(launch_row_scores(x, RowMap{1, 0, M}, B, M, C, scores, static_cast<cudaStream_t>(stream)), "row_scores");
+  FK_CUDA(launch_row_scores(x, RowMap{1, 0, M}, B, M, C, nullptr, scores, static_cast<cudaStream_t>(stream)), "row_scores");
+  return FVAR_OK;
+}
+
+fvar_status fvar_row_keys(const float *x, const float *noise, int B, int M, int C, float *keys, void *stream) {
+  if (!x || !noise || !keys || B <= 0 || M <= 0 || C <= 0 || C % 4) return kfail(FVAR_EINVAL, "row_keys: bad arguments");
+  FK_CUDA(launch_row_scores(x, RowMap{1, 0, M}, B, M, C, noise, keys, static_cast<cudaStream_t>(stream)), "row_keys");
   return FVAR_OK;
 }
 

@@ -103,7 +103,8 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 void set_global_error(const char *msg);
 
 // Memory-bound kernels.
-cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, float *scores, cudaStream_t st);
+cudaError_t launch_row_scores(const float *x, RowMap xmap, int E, int M, int C, const float *noise, float *scores,
+                              cudaStream_t st);
 cudaError_t launch_select_topr(const float *scores, int B, int M, int r, int *idx, int *inv, cudaStream_t st);
 cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_forced, int *idx, int *inv,
                                 unsigned *status, cudaStream_t st);

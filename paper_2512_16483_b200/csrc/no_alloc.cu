@@ -58,7 +58,7 @@ extern "C" fvar_status fvar_select_rows_static(const float *x, int B, int M, int
   }
   float *scores = nullptr;
   cudaError_t e = static_scores_address(&scores);
-  if (e == cudaSuccess) e = launch_row_scores(x, RowMap{1, 0, M}, B, M, C, scores, static_cast<cudaStream_t>(stream));
+  if (e == cudaSuccess) e = launch_row_scores(x, RowMap{1, 0, M}, B, M, C, nullptr, scores, static_cast<cudaStream_t>(stream));
   if (e == cudaSuccess) e = launch_select_topr(scores, B, M, r, idx, inv, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     set_global_error((std::string("select_rows_static: ") + cudaGetErrorString(e)).c_str());

@@ -182,3 +182,22 @@ def test_rtr_fill(fv, hw_in, hw_out, C):
     fv.fvar_rtr_fill(torch.from_numpy(prev).cuda(), hw_in, hw_out, None, out2)      # inv == NULL fills all rows
     np.testing.assert_allclose(out2.cpu().numpy()[0], orc.upsample_bilinear(prev[0].astype(np.float64), hw_in, hw_out),
                                atol=2e-5, rtol=1e-5)
+
+
+# ----------------------------------------------------------------------------- sampled selection keys
+
+@pytest.mark.parametrize("B,M,C", [(2, 256, 1024), (1, 4096, 2048), (3, 100, 64)])
+def test_row_keys_and_sampled_selection(fv, B, M, C):
+    """Keys s_i / E_i of the sampled selection: the division is exact in fp32 on both sides, so the keys
+    differ only by the summation order of the score; selection on identical keys is bit-exact."""
+    x = si.make_tokens(41, B, M, C, "spread")
+    noise = si.make_sample_noise(41, 0, 1, B, M)[0]
+    got = fv.fvar_row_keys(torch.from_numpy(x).cuda(), torch.from_numpy(noise).cuda()).cpu().numpy()
+    ref64 = orc.row_scores(x, np.float64) / noise.astype(np.float64)
+    np.testing.assert_allclose(got, ref64, rtol=3e-6)
+    keys = np.stack([orc.sampling_keys(orc.row_scores(x[b], np.float32), noise[b]) for b in range(B)])
+    for r in (1, max(1, M // 4), M // 2):
+        _check_select(fv, keys, r)
+    # a key is one correctly rounded fp32 division of the kernel's own score
+    s_gpu = fv.fvar_row_scores(torch.from_numpy(x).cuda()).cpu().numpy()
+    assert np.array_equal(got, (s_gpu / noise).astype(np.float32))

@@ -320,3 +320,30 @@ def test_split_k_is_deterministic_and_close(fv, splits):
     second = p.gpu.scale_step(to_bf16_cuda(toks), 9, mode=fv.LOWRANK_RTR, keep_ratio=0.5).clone()
     p.check_ok()
     assert torch.equal(first, second)
+
+
+def test_sampled_selection_step(fv):
+    """FVAR_SELECT_SAMPLE: rows drawn without replacement with probability proportional to their score,
+    from the same Exp(1) variates on both sides; the rest of the step is unchanged."""
+    shp = si.shape_var_d16(n_blocks=2)
+    B, k, M, r = 2, 9, 256, 96
+    p = Pair(fv, shp, seed=109, B=B)
+    p.prefill(k)
+    p.set_projections(k, [r, r])
+    toks = si.make_tokens(109, B, M, 1024, "spread")
+    noise = si.make_sample_noise(109, k, 2, B, M)
+    ref = p.oracle.scale_step(toks, k, orc.Policy("lowrank_rtr", "pair", rank_per_group=[r, r], sample_noise=noise))
+    out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r],
+                           sample_noise=torch.from_numpy(noise).cuda())
+    p.check_ok()
+    top = [orc.select_top_r(orc.row_scores(toks[e], np.float32), r) for e in range(B)]
+    for g in range(2):
+        idx = p.gpu.get_indices(g, B, M).cpu().numpy()
+        for e in range(B):
+            assert np.array_equal(idx[e], p.oracle.last_indices[e][g]), (g, e)
+    assert any(not np.array_equal(p.oracle.last_indices[e][0], top[e]) for e in range(B))     # it is not plain top-r
+    assert_out_close(bf16_to_numpy(out), ref, what="sampled selection")
+    # the same call again replays the captured graph and gives the same bits
+    again = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r],
+                             sample_noise=torch.from_numpy(noise).cuda())
+    assert again.shape == out.shape
