@@ -43,6 +43,13 @@ WORKLOADS = {
     "infinity2b_paper_b2": dict(shape="inf2b", B=2, first_late=10, keep="paper", null_only=True),
     # ... and the unpruned dense path with both CFG branches.
     "infinity2b_dense3_b2": dict(shape="inf2b", B=2, first_late=10, keep=1.0, null_only=False),
+    # The transformer part of a whole 13-scale generation (no quantizer / decoder): every scale from 1x1 on, the
+    # KV cache built by the steps themselves.  vanilla: all scales dense with both CFG branches; fastervar: scales
+    # 1..32 dense with both branches, then the schedule of Sec. 4.1 (40 approximated on the null branch, 48 and 64
+    # skipped); fastervar_late3: the three late scales all approximated at the tabulated ranks.
+    "infinity2b_gen13_vanilla_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=13, keep=1.0, null_only=False),
+    "infinity2b_gen13_fastervar_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=10, keep="paper", null_only=True),
+    "infinity2b_gen13_fastervar_late3_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=10, keep="table", null_only=True),
 }
 
 
@@ -52,7 +59,9 @@ def scale_plan(wl, shp):
     Ms, plan = shp.tokens_per_scale(), {}
     for k in range(wl["first_late"], len(Ms)):
         keep = wl["keep"]
-        if keep in ("table", "paper"):
+        if k < wl.get("dense_until", 0):
+            plan[k] = [Ms[k]] * shp.n_groups
+        elif keep in ("table", "paper"):
             side = shp.scales[k]
             if keep == "paper" and schedule.INFINITY_ALPHA[schedule.INFINITY_LATE_SCALES.index(side)] == 0.0:
                 plan[k] = None
@@ -145,6 +154,8 @@ def oracle_leg(wl, steps, warmup):
         threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
     except Exception:
         threads = os.cpu_count() or 1
+    if "dense_until" in wl:
+        raise NotImplementedError("no CPU baseline for the whole-generation workloads")
     full = make_shape(wl["shape"])
     plan_full = scale_plan(wl, full)
     shp = make_shape(wl["shape"])
@@ -252,8 +263,9 @@ def main():
     Ms = shp.tokens_per_scale()
     plan = scale_plan(wl, shp)
     late_scales = sorted(plan)
-    cfg_mode = fv.CFG_NULL_ONLY if wl["null_only"] else fv.CFG_PAIR
-    E = B // 2 if wl["null_only"] else B
+    null_at = {k: bool(wl["null_only"]) and k >= wl.get("dense_until", 0) for k in late_scales}
+    cfg_at = {k: fv.CFG_NULL_ONLY if null_at[k] else fv.CFG_PAIR for k in late_scales}
+    E_at = {k: B // 2 if null_at[k] else B for k in late_scales}
     seed = SEED + rank
     big = wl["shape"] == "inf2b"
 
@@ -286,7 +298,9 @@ def main():
     context = bf16_cuda(si.make_context(seed, B, shp.ctx_len, shp.ctx_width)) if shp.has_cross_attn else None
     ctx.set_cond(bf16_cuda(si.make_cond(seed, B, shp.width)), context)
     L0 = sum(Ms[:k0])
-    if big:
+    if k0 == 0:
+        pass                                   # whole generation: the steps build the cache themselves
+    elif big:
         ctx.load_kv(randn_bf16((shp.n_blocks, B, L0, shp.width)), randn_bf16((shp.n_blocks, B, L0, shp.width)))
         ctx.load_group_cache(k0 - 1, torch.randn((shp.n_groups, B, Ms[k0 - 1], shp.width), generator=gen, device="cuda"))
     else:
@@ -310,27 +324,28 @@ def main():
                 ctx.set_projection(k, g, qt)
     toks = {k: (randn_bf16((B, Ms[k], shp.width)) if big else bf16_cuda(si.make_tokens(seed, B, Ms[k], shp.width)))
             for k in late_scales}
-    outs = {k: torch.empty((E, Ms[k], shp.width), dtype=torch.bfloat16, device="cuda") for k in late_scales}
+    outs = {k: torch.empty((E_at[k], Ms[k], shp.width), dtype=torch.bfloat16, device="cuda") for k in late_scales}
     toks_host = {k: toks[k].cpu().pin_memory() for k in late_scales}
-    outs_host = {k: torch.empty((E, Ms[k], shp.width), dtype=torch.bfloat16).pin_memory() for k in late_scales}
-    tokens_per_step = E * sum(Ms[k] for k in late_scales)     # a skipped scale still delivers its positions
+    outs_host = {k: torch.empty((E_at[k], Ms[k], shp.width), dtype=torch.bfloat16).pin_memory() for k in late_scales}
+    tokens_per_step = sum(E_at[k] * Ms[k] for k in late_scales)     # a skipped scale still delivers its positions
+    rewind = ctx.reset if k0 == 0 else ctx.restore_loaded
 
     def step_device():
-        ctx.restore_loaded()
+        rewind()
         for k in late_scales:
             mode, ranks = modes[k]
             if mode == fv.SKIP:
                 continue
-            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_mode, rank_per_group=ranks, out=outs[k])
+            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks, out=outs[k])
             ctx.kv_append(k)
 
     def step_host():
-        ctx.restore_loaded()
+        rewind()
         for k in late_scales:
             mode, ranks = modes[k]
             if mode == fv.SKIP:
                 continue
-            ctx.scale_step_host(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_mode, rank_per_group=ranks)
+            ctx.scale_step_host(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks)
             ctx.kv_append(k)
 
     def barrier():
@@ -396,10 +411,10 @@ def main():
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e, "unit": "tokens/s",
                 "h2d_bytes_per_step": sum(B * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP),
-                "d2h_bytes_per_step": sum(E * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP)},
+                "d2h_bytes_per_step": sum(E_at[k] * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP)},
         "roofline": roofline,
     }
-    if world == 1 and not args.no_cpu_baseline and not args.profile_run:
+    if world == 1 and not args.no_cpu_baseline and not args.profile_run and "dense_until" not in wl:
         tps, dt, desc, threads = oracle_leg(wl, 1, 0)
         line["cpu_baseline"] = {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc,
                                 "seconds": dt}
