@@ -347,3 +347,30 @@ def test_sampled_selection_step(fv):
     again = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r],
                              sample_noise=torch.from_numpy(noise).cuda())
     assert again.shape == out.shape
+
+
+@pytest.mark.parametrize("B,cfg", [(1, "pair"), (2, "null_only"), (3, "pair")])
+def test_edge_ranks_and_batches(fv, B, cfg):
+    """Degenerate cases of the method: r = 1 (one representative row), r = M - 1 (one filled row), a batch
+    of one element, an odd batch, non-square token maps."""
+    shp = si.shape_tiny(n_blocks=2, blocks_per_group=1, width=128, n_heads=2, head_dim=64, ffn_dim=192,
+                        scales=(1, 3, 5), scale_hw=((1, 2), (3, 2), (5, 4)))
+    p = Pair(fv, shp, seed=110, B=B, std=0.05)
+    Ms = shp.tokens_per_scale()
+    toks = [si.make_tokens(110, B, m, 128) for m in Ms]
+    got, ref = _step_both(p, toks[0], 0, mode=fv.DENSE)
+    assert_out_close(got, ref, what="dense 1x2 map")
+    p.gpu.kv_append(0)
+    p.oracle.kv_append(0)
+    ranks = [1, Ms[1] - 1]
+    p.set_projections(1, ranks)
+    got, ref = _step_both(p, toks[1], 1, mode=fv.LOWRANK_RTR, cfg=cfg, ranks=ranks)
+    assert_out_close(got, ref, what="r = 1 / r = M - 1")
+    p.gpu.kv_append(1)
+    p.oracle.kv_append(1)
+    ranks = [Ms[2] - 1, 1]
+    p.set_projections(2, ranks)
+    got, ref = _step_both(p, toks[2], 2, mode=fv.LOWRANK_RTR, cfg=cfg, ranks=ranks)
+    assert_out_close(got, ref, what="r = M - 1 / r = 1 after a late scale")
+    e0 = 1 if cfg == "null_only" else 0
+    assert p.gpu.cache_len(0) == p.oracle.cache_len(0, e0) and p.gpu.cache_len(1) == p.oracle.cache_len(1, e0)
