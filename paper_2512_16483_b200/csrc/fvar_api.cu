@@ -94,6 +94,7 @@ struct fvar_ctx {
   std::vector<int> hw;                 // 2 * n_scales
   std::vector<int> Mk;                 // tokens per scale
   int G, C, F, H, D, Bmax, Mmax, L_cap, ctx_cap, num_sms;
+  int max_clusters;                    // resident CTA pairs of the pair GEMM (0: pairs not used)
   cudaStream_t st;         // the caller's stream
   cudaStream_t launch_st;  // where launches go: st, or cap_st while a graph is being captured
   cudaStream_t cap_st;     // private stream used only for capture (the legacy default stream cannot be captured)
@@ -275,17 +276,21 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int 
 }
 
 fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk, int wid, GemmArgs &g, const char *what) {
-  const int tiles_m = (g.R + 127) / 128 * g.nbatch;
-  int bn = 64, sp = 1;
-  gemm_pick_tile(tiles_m, g.N, g.K, ctx->num_sms, ctx->max_splits, kSplitScratchBytes, &bn, &sp);
-  g.splits = sp;
+  // CTA pairs need the full 128-row A box (tmA is then the activation buffer's 128-row map)
+  const GemmPlan plan = gemm_plan(g.R, g.nbatch, g.N, g.K, ctx->num_sms, (g.a_box_rows == 128 || g.a_box_rows == 0) ? ctx->max_clusters : 0,
+                                  ctx->max_splits, kSplitScratchBytes);
+  const int bn = plan.block_n;
+  g.splits = plan.splits;
   g.partial = ctx->split_partial;
   g.counters = ctx->split_counters;
   g.status = ctx->status;
   ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
                   2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
                       (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N * g.nbatch);
-  FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->launch_st), what);
+  if (plan.pair)
+    FV_CUDA(ctx, launch_gemm_pair(epi, bn, tmA, ctx->wm(blk, wid, bn / 2), g, ctx->launch_st), what);
+  else
+    FV_CUDA(ctx, launch_gemm(epi, bn, tmA, ctx->wm(blk, wid, bn), g, ctx->num_sms, ctx->launch_st), what);
   ctx->launched();
   return FVAR_OK;
 }
@@ -446,8 +451,9 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
-  if (gemm_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
+  if (gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
+  c->max_clusters = gemm_pair_max_clusters();
   *out = c;
   return FVAR_OK;
 }
@@ -1023,16 +1029,21 @@ fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R
   int dev = 0, sms = 0;
   FK_CUDA(cudaGetDevice(&dev), "get device");
   FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
-  const int bn = gemm_pick_block_n((R + 127) / 128, N, K, sms);
+  const GemmPlan plan = gemm_plan(R, 1, N, K, sms, gemm_pair_max_clusters(), 1, 0);
+  const int bn = plan.block_n;
   CUtensorMap ta, tw;
-  if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, W, K, N, K, bn)) return kfail(FVAR_EINVAL, "gemm: operands must be 16-byte aligned");
+  if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, W, K, N, K, plan.pair ? bn / 2 : bn))
+    return kfail(FVAR_EINVAL, "gemm: operands must be 16-byte aligned");
   GemmArgs g = gemm_args(R, N, K);
   g.bias = static_cast<const bf16 *>(bias);
   g.out_f32 = out;
   g.ld_out = N;
   g.status = kernel_status_ptr();
   if (!g.status) return kfail(FVAR_ECUDA, "gemm: status word");
-  FK_CUDA(launch_gemm(EPI_F32, bn, ta, tw, g, sms, static_cast<cudaStream_t>(stream)), "gemm");
+  if (plan.pair)
+    FK_CUDA(launch_gemm_pair(EPI_F32, bn, ta, tw, g, static_cast<cudaStream_t>(stream)), "gemm");
+  else
+    FK_CUDA(launch_gemm(EPI_F32, bn, ta, tw, g, sms, static_cast<cudaStream_t>(stream)), "gemm");
   return FVAR_OK;
 }
 

@@ -2,22 +2,19 @@
 //
 // One persistent CTA per SM walks the tile list.  Warp 0 feeds a ring of shared-memory stages
 // with TMA (128-byte swizzle), warp 1 issues tcgen05.mma into one of two TMEM accumulators,
-// warps 2-5 drain the other accumulator (tcgen05.ld) and apply the epilogue, so the epilogue of
+// warps 2-9 drain the other accumulator (tcgen05.ld) and apply the epilogue, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  Every wait is bounded; on expiry the CTA flags the
 // status word, lets its outstanding copies land, frees its TMEM and returns.
 #include <stdlib.h>
 
-#include "internal.h"
-#include "ptx.cuh"
+#include "gemm_common.cuh"
 
 namespace fvar {
 
-constexpr int kBlockM = 128;
-constexpr int kBlockK = 64;             // 64 bf16 = one 128-byte swizzle row (one "atom" along K)
 // Atoms per pipeline stage: one barrier round trip covers 64 * atoms of K.  Narrow tiles are bound by
 // the round trip, not by bytes, so they take two atoms per stage (measured: 25 % faster at BN = 64).
 __host__ __device__ constexpr int k_atoms(int bn) { return bn <= 128 ? 2 : 1; }
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kSmemBudget = 196608;     // bytes of operand stages per CTA (192 KiB)
 
 #ifdef FVAR_TRACE
@@ -36,7 +33,7 @@ struct GemmCfg {
   static constexpr int kStageBytes = kStageBytesA + kStageBytesB;
   static constexpr int kStages = kSmemBudget / kStageBytes;
   static constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;     // two accumulators
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/ + 4 * 4096 /*epilogue staging*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/ + kEpiWarps * 4096 /*epilogue staging*/;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory");
   static_assert(kStages >= 2 && kStages <= 12, "stage count");
   static_assert((kTmemCols & (kTmemCols - 1)) == 0 && kTmemCols <= 512, "TMEM columns");
@@ -44,153 +41,6 @@ struct GemmCfg {
   // allocation (up to all 512 columns) can never wait on a co-resident CTA.
   static_assert(kSmemBytes > 116 * 1024, "one CTA per SM");
 };
-
-__device__ __forceinline__ float gelu_tanh_f(float x) {
-  const float k0 = 0.7978845608028654f, k1 = 0.044715f;
-  float u = k0 * (x + k1 * x * x * x);
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
-  return 0.5f * x * (1.0f + t);
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// Warp-wide row-major stores through a 4 KiB shared-memory staging tile.  After tcgen05.ld each lane
-// holds 32 consecutive columns of its own row; storing those directly makes every instruction touch
-// 32 different rows 16 bytes at a time.  Instead the lanes park their pieces in shared memory (16-byte
-// chunks XOR-swizzled by row, conflict-free both ways) and the warp writes whole 128-byte (fp32) or
-// 64-byte (bf16) row segments, 4 or 8 rows per instruction.  `dst` is this lane's row segment (nullptr:
-// row past the end); every lane of the warp must call.
-__device__ __forceinline__ void warp_store_f32(uint32_t stage, int lane, const float (&v)[32], float *dst) {
-#pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    const uint32_t addr = stage + lane * 128 + ((q ^ (lane & 7)) << 4);
-    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v[q * 4]), "f"(v[q * 4 + 1]), "f"(v[q * 4 + 2]),
-                 "f"(v[q * 4 + 3]) : "memory");
-  }
-  __syncwarp();
-  const int c = lane & 7;
-#pragma unroll
-  for (int it = 0; it < 8; ++it) {
-    const int r = it * 4 + (lane >> 3);
-    float4 o;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w)
-                 : "r"(stage + r * 128 + ((c ^ (r & 7)) << 4)));
-    float *pr = reinterpret_cast<float *>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(dst), r));
-    if (pr != nullptr) reinterpret_cast<float4 *>(pr)[c] = o;
-  }
-  __syncwarp();
-}
-
-__device__ __forceinline__ void warp_store_bf16(uint32_t stage, int lane, const float (&v)[32], bf16 *dst) {
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const uint32_t addr = stage + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4);
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(v[q * 8], v[q * 8 + 1])),
-                 "r"(pack_bf16(v[q * 8 + 2], v[q * 8 + 3])), "r"(pack_bf16(v[q * 8 + 4], v[q * 8 + 5])),
-                 "r"(pack_bf16(v[q * 8 + 6], v[q * 8 + 7])) : "memory");
-  }
-  __syncwarp();
-  const int c = lane & 3;
-#pragma unroll
-  for (int it = 0; it < 4; ++it) {
-    const int r = it * 8 + (lane >> 2);
-    uint4 o;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o.x), "=r"(o.y), "=r"(o.z), "=r"(o.w)
-                 : "r"(stage + r * 64 + ((c ^ ((r >> 1) & 3)) << 4)));
-    bf16 *pr = reinterpret_cast<bf16 *>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(dst), r));
-    if (pr != nullptr) reinterpret_cast<uint4 *>(pr)[c] = o;
-  }
-  __syncwarp();
-}
-
-// Epilogue of one warp for 32 rows x 32 consecutive columns starting at col0 (col0 % 32 == 0): each
-// lane owns one row (`valid` false: row past the end).  Every lane of the warp must call.
-template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t (&acc)[32], int batch, int row,
-                                               int col0, bool valid, uint32_t stage, int lane,
-                                               const float4 *resid_pre = nullptr) {
-  float v[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(acc[i]);
-  const bool full = (col0 + 32 <= p.N);
-  if (p.bias != nullptr) {
-    if (full) {
-      const uint4 *bp = reinterpret_cast<const uint4 *>(p.bias + col0);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 u = __ldg(bp + q);
-        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          float2 f = __bfloat1622float2(h[t]);
-          v[q * 8 + t * 2] += f.x;
-          v[q * 8 + t * 2 + 1] += f.y;
-        }
-      }
-    } else {
-      for (int i = 0; i < 32; ++i)
-        if (col0 + i < p.N) v[i] += __bfloat162float(p.bias[col0 + i]);
-    }
-  }
-  const long long grow = static_cast<long long>(batch) * p.R + row;   // row in the flattened output
-
-  if constexpr (EPI == EPI_F32) {
-    float *dst = p.out_f32 + grow * p.ld_out + col0;
-    if (full && (p.ld_out & 3) == 0) {            // uniform across the warp
-      warp_store_f32(stage, lane, v, valid ? dst : nullptr);
-    } else if (valid) {
-      for (int i = 0; i < 32; ++i)
-        if (col0 + i < p.N) dst[i] = v[i];
-    }
-  } else if constexpr (EPI == EPI_BF16 || EPI == EPI_GELU_BF16) {
-    if constexpr (EPI == EPI_GELU_BF16) {
-#pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_f(v[i]);
-    }
-    warp_store_bf16(stage, lane, v, valid ? p.out_bf16 + grow * p.ld_out + col0 : nullptr);
-  } else if constexpr (EPI == EPI_QKV) {
-    const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
-    const int b = e * p.bmul + p.boff;
-    const int vc = col0 + p.col_base;             // uniform across the warp
-    if (vc < p.C) {
-      warp_store_bf16(stage, lane, v, valid ? p.out_bf16 + static_cast<long long>(row) * p.ld_out + vc : nullptr);
-    } else if (vc < 2 * p.C) {
-      const int c = vc - p.C, h = c / p.D, d0 = c - h * p.D;
-      bf16 *base = p.kc + ((static_cast<long long>(b) * p.H + h) * p.L_cap + p.L_prev + j) * p.D + d0;
-      warp_store_bf16(stage, lane, v, valid ? base : nullptr);
-    } else if (valid) {
-      // transposed V cache: consecutive rows of the warp are consecutive addresses already
-      const int c = vc - 2 * p.C, h = c / p.D, d0 = c - h * p.D;
-      bf16 *base = p.vt + ((static_cast<long long>(b) * p.H + h) * p.D + d0) * p.L_cap + p.L_prev + j;
-#pragma unroll
-      for (int i = 0; i < 32; ++i) base[static_cast<long long>(i) * p.L_cap] = __float2bfloat16_rn(v[i]);
-    }
-  } else {  // EPI_RESID
-    float *dst = nullptr;
-    if (valid) {
-      const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
-      const int b = e * p.bmul + p.boff;
-      const float *res = p.resid + (static_cast<long long>(e * p.rmap.bmul + p.rmap.boff) * p.rmap.rpb + j) * p.ld_out + col0;
-      const int jo = p.scatter ? __ldg(p.scatter + static_cast<long long>(e) * p.rows_per_batch + j) : j;
-      dst = p.out_f32 + (static_cast<long long>(e * p.omap.bmul + p.omap.boff) * p.omap.rpb + jo) * p.ld_out + col0;
-      const float *g = p.gate ? p.gate + static_cast<long long>(b) * p.gate_stride + col0 : nullptr;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        float4 r4 = resid_pre ? resid_pre[q] : reinterpret_cast<const float4 *>(res)[q];
-        float4 g4 = g ? __ldg(reinterpret_cast<const float4 *>(g) + q) : make_float4(1.f, 1.f, 1.f, 1.f);
-        v[q * 4] = fmaf(g4.x, v[q * 4], r4.x);
-        v[q * 4 + 1] = fmaf(g4.y, v[q * 4 + 1], r4.y);
-        v[q * 4 + 2] = fmaf(g4.z, v[q * 4 + 2], r4.z);
-        v[q * 4 + 3] = fmaf(g4.w, v[q * 4 + 3], r4.w);
-      }
-    }
-    warp_store_f32(stage, lane, v, dst);
-  }
-}
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -231,7 +81,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 128);
+      mbar_init(tempty_bar(a), 32 * kEpiWarps);
     }
     mbar_fence_init();
     prefetch_tmap(&tmA);
@@ -361,8 +211,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // A warp reads the TMEM lanes of its quadrant (warp index mod 4); the two warps of a quadrant
+    // take alternate 32-column chunks of the tile.
     const int quad = warp & 3;                 // TMEM lanes [32 * quad, 32 * quad + 32)
+    const int cg = (warp - 2) >> 2;            // column group of this warp
+    constexpr int kChunks = (BN / 32 + kEpiColGroups - 1) / kEpiColGroups;   // chunks per warp
     const uint32_t ep_stage = bar_base + 256 + (warp - 2) * 4096;   // this warp's staging tile
     int it = 0;
     bool ok = true;
@@ -376,7 +230,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       const int row = m_idx * kBlockM + row_local;
       // The residual rows of the first two column chunks are fetched while the main loop still runs:
       // with one tile per CTA nothing else hides that latency.
-      constexpr int kPre = (BN / 32 < 2) ? BN / 32 : 2;
+      constexpr int kPre = (kChunks < 2) ? kChunks : 2;
       float4 pre[kPre][8];
       bool have_pre = false;
       if constexpr (EPI == EPI_RESID) {
@@ -384,11 +238,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           const int e2 = row / p.rows_per_batch, j2 = row - e2 * p.rows_per_batch;
           const float *res = p.resid + (static_cast<long long>(e2 * p.rmap.bmul + p.rmap.boff) * p.rmap.rpb + j2) * p.ld_out + n_idx * BN;
 #pragma unroll
-          for (int c = 0; c < kPre; ++c)
+          for (int ci = 0; ci < kPre; ++ci) {
+            const int c = ci * kEpiColGroups + cg;
             if (n_idx * BN + c * 32 < p.N) {
 #pragma unroll
-              for (int q = 0; q < 8; ++q) pre[c][q] = reinterpret_cast<const float4 *>(res + c * 32)[q];
+              for (int q = 0; q < 8; ++q) pre[ci][q] = reinterpret_cast<const float4 *>(res + c * 32)[q];
             }
+          }
           have_pre = true;
         }
       }
@@ -397,9 +253,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
       if (splits == 1) {
-        auto do_chunk = [&](int c, const float4 *prep) {
+        auto do_chunk = [&](int ci, const float4 *prep) {
+          const int c = ci * kEpiColGroups + cg;
           const int col0 = n_idx * BN + c * 32;
-          if (col0 < p.N) {                      // uniform across the warp
+          if (c * 32 < BN && col0 < p.N) {       // uniform across the warp
             uint32_t acc[32];
             tmem_ld32(taddr + c * 32, acc);
             tmem_ld_wait();
@@ -407,9 +264,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
         };
 #pragma unroll
-        for (int c = 0; c < kPre; ++c) do_chunk(c, have_pre ? pre[c] : nullptr);
+        for (int ci = 0; ci < kPre; ++ci) do_chunk(ci, have_pre ? pre[ci] : nullptr);
 #pragma unroll 1
-        for (int c = kPre; c < BN / 32; ++c) do_chunk(c, nullptr);
+        for (int ci = kPre; ci < kChunks; ++ci) do_chunk(ci, nullptr);
         tc_fence_before();
         mbar_arrive(tempty_bar(a));
       } else {
@@ -420,7 +277,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // warp (consecutive rows) touch 512 contiguous bytes per access.
         float4 *mine = reinterpret_cast<float4 *>(p.partial + (static_cast<size_t>(tile) * splits + sp) * (kBlockM * BN)) + row_local;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = cg; c < BN / 32; c += kEpiColGroups) {
           uint32_t acc[32];
           tmem_ld32(taddr + c * 32, acc);
           tmem_ld_wait();
@@ -434,14 +291,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         tc_fence_before();
         mbar_arrive(tempty_bar(a));
         __threadfence();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         if (threadIdx.x == 64) split_last = (atomicAdd(p.counters + tile, 1) == splits - 1) ? 1 : 0;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         if (split_last) {
           __threadfence();
           const float4 *base = reinterpret_cast<const float4 *>(p.partial + static_cast<size_t>(tile) * splits * (kBlockM * BN)) + row_local;
 #pragma unroll 1
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = cg; c < BN / 32; c += kEpiColGroups) {
             const int col0 = n_idx * BN + c * 32;
             if (col0 >= p.N) break;
             float sum[32];
@@ -523,6 +380,45 @@ extern "C" int fvar_debug_read_gemm_trace(long long *host, int n) {
   return cudaMemcpyFromSymbol(host, g_gemm_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
 }
 #endif
+
+// FVAR_GEMM_PAIR=0 never uses CTA pairs, =1 uses them whenever the problem allows; unset: cost model.
+static int forced_pair() {
+  static int v = -2;
+  if (v == -2) {
+    const char *e = getenv("FVAR_GEMM_PAIR");
+    v = e ? atoi(e) : -1;
+    if (v != 0 && v != 1) v = -1;
+  }
+  return v;
+}
+
+GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_clusters, int max_splits, size_t scratch_bytes) {
+  GemmPlan plan{false, 64, 1};
+  const int tiles_m = (R + kBlockM - 1) / kBlockM * nbatch;
+  gemm_pick_tile(tiles_m, N, K, num_sms, max_splits, scratch_bytes, &plan.block_n, &plan.splits);
+  if (nbatch != 1 || R <= kBlockM || max_clusters <= 0 || forced_pair() == 0) return plan;
+  // Cost of the single-CTA choice, recomputed with the same constants as gemm_pick_tile.
+  const float t_k1[3] = {0.24f, 0.30f, 0.47f}, t_epi1[3] = {1.0f, 1.5f, 2.5f};
+  const int num_kb = (K + kBlockK - 1) / kBlockK;
+  const int i1 = plan.block_n == 64 ? 0 : (plan.block_n == 128 ? 1 : 2);
+  const long long tiles1 = static_cast<long long>(tiles_m) * ((N + plan.block_n - 1) / plan.block_n) * plan.splits;
+  float cost1 = ((tiles1 + num_sms - 1) / num_sms) * (((num_kb + plan.splits - 1) / plan.splits) * t_k1[i1] + t_epi1[i1]);
+  if (plan.splits > 1) cost1 += 1.5f + 0.6f * plan.splits * plan.block_n / 128.0f;
+  // A pair CTA moves, per K step, what a single CTA of half the tile width moves, for twice the output.
+  const int cand2[2] = {128, 256};
+  const float t_k2[2] = {0.24f, 0.30f}, t_epi2[2] = {1.5f, 2.5f};
+  const int tiles_m2 = (R + 2 * kBlockM - 1) / (2 * kBlockM);
+  float best2 = 1e30f;
+  int bn2 = 0;
+  for (int i = 0; i < 2; ++i) {
+    if (forced_block_n() && cand2[i] != forced_block_n()) continue;
+    const long long t2 = static_cast<long long>(tiles_m2) * ((N + cand2[i] - 1) / cand2[i]);
+    const float c = ((t2 + max_clusters - 1) / max_clusters) * (num_kb * t_k2[i] + t_epi2[i]);
+    if (c < best2) { best2 = c; bn2 = cand2[i]; }
+  }
+  if (bn2 && (forced_pair() == 1 || best2 < cost1)) plan = GemmPlan{true, bn2, 1};
+  return plan;
+}
 
 int gemm_pick_block_n(int tiles_m_total, int N, int K, int num_sms) {
   int bn, sp;

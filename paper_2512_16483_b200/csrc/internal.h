@@ -61,8 +61,25 @@ void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits
 cudaError_t launch_gemm(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
                         int num_sms, cudaStream_t st);
 
+// CTA-pair form (gemm_pair.cu): 256 x block_n tiles, block_n in {128, 256}; the W map's box must have
+// block_n / 2 rows, the A map's box 128 rows.  One problem per launch (nbatch == 1), no split-K.
+cudaError_t launch_gemm_pair(int epi, int block_n, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a,
+                             cudaStream_t st);
+// Largest number of CTA pairs of the pair kernel that can be resident at once (0: pairs unavailable).
+int gemm_pair_max_clusters();
+// How a GEMM is launched: by single CTAs (block_n in {64, 128, 256}, optional split-K) or by CTA pairs
+// (block_n in {128, 256}).
+struct GemmPlan {
+  bool pair;
+  int block_n, splits;
+};
+// Picks the launch form and tile width from the measured cost model.  tiles_m_total: 128-row tiles over
+// all batches; pairs are considered only for a single problem with more than one row tile.
+GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_clusters, int max_splits, size_t scratch_bytes);
+
 // Set the dynamic shared-memory attribute of every instantiation (once, outside any stream capture).
 cudaError_t gemm_prepare();
+cudaError_t gemm_pair_prepare();
 cudaError_t attention_prepare();
 
 struct AttnArgs {
