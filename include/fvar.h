@@ -225,6 +225,19 @@ fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, c
 fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out,
                            void *stream);
 
+/* The same product with the launch form given instead of picked: form FVAR_GEMM_AUTO (the library's
+ * cost model, as fvar_gemm_bf16), FVAR_GEMM_SINGLE (one CTA per 128 x block_n tile, block_n in
+ * {64, 128, 256}) or FVAR_GEMM_PAIR (two CTAs on neighbouring SMs share one 256 x block_n tile through
+ * tcgen05.mma.cta_group::2, block_n in {128, 256}; needs R > 128).  block_n = 0 lets the cost model
+ * pick the width for the given form.  The transformer block of the step is the workload's own
+ * definition (the paper only names it a "VAR block", Sec. 3.1), so this is a kernel-level entry for
+ * tests and tuning.  FVAR_EINVAL for a form / width the problem does not allow. */
+#define FVAR_GEMM_AUTO 0
+#define FVAR_GEMM_SINGLE 1
+#define FVAR_GEMM_PAIR 2
+fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
+                                int block_n, float *out, void *stream);
+
 /* softmax(q k^T / sqrt(D)) v per head over the first L rows of a cache in the library's layout:
  * q dev bf16 [B][r][H*D]; Kc dev bf16 [B][H][L_cap][D]; Vt dev bf16 [B][H][D][L_cap] (values stored
  * transposed); out dev bf16 [B][r][H*D].  D in {64, 128}; L_cap % 8 == 0; 1 <= L <= L_cap. */

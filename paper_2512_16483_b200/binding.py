@@ -20,6 +20,7 @@ DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
 SELECT_TOPR, SELECT_SAMPLE = 0, 1
 OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS = 0, 1
+GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR = 0, 1, 2
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")
@@ -94,6 +95,7 @@ def load_library() -> ct.CDLL:
         "fvar_select_topr": (i, [vp, i, i, i, vp, vp, vp]),
         "fvar_ln_modulate": (i, [vp, i, i, i, vp, vp, ll, f, vp, vp]),
         "fvar_gemm_bf16": (i, [vp, vp, vp, i, i, i, vp, vp]),
+        "fvar_gemm_bf16_form": (i, [vp, vp, vp, i, i, i, i, i, vp, vp]),
         "fvar_attention": (i, [vp, vp, vp, i, i, i, i, i, i, vp, vp]),
         "fvar_rtr_fill": (i, [vp, i, i, i, i, i, i, vp, vp, vp]),
         "fvar_select_rows_static": (i, [vp, i, i, i, i, vp, vp, vp]),
@@ -110,7 +112,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
+            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
 
 def _stream() -> int:
@@ -173,11 +175,17 @@ def fvar_ln_modulate(x: torch.Tensor, shift: torch.Tensor, scale: torch.Tensor, 
 
 def fvar_gemm_bf16(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.Tensor] = None) -> torch.Tensor:
     """A bf16 [R][K], W bf16 [N][K], bias bf16 [N] -> fp32 [R][N] = A W^T + bias."""
+    return fvar_gemm_bf16_form(A, W, bias, GEMM_AUTO, 0)
+
+
+def fvar_gemm_bf16_form(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.Tensor], form: int, block_n: int) -> torch.Tensor:
+    """fvar_gemm_bf16 with the launch form (GEMM_AUTO / GEMM_SINGLE / GEMM_PAIR) and tile width given."""
     _dev(A, torch.bfloat16), _dev(W, torch.bfloat16)
     R, K = A.shape
     N = W.shape[0]
     out = torch.empty((R, N), dtype=torch.float32, device=A.device)
-    _check_kernel(load_library().fvar_gemm_bf16(A.data_ptr(), W.data_ptr(), _ptr(bias), R, N, K, out.data_ptr(), _stream()))
+    _check_kernel(load_library().fvar_gemm_bf16_form(A.data_ptr(), W.data_ptr(), _ptr(bias), R, N, K, form, block_n,
+                                                     out.data_ptr(), _stream()))
     return out
 
 

@@ -1024,12 +1024,25 @@ fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, c
   return FVAR_OK;
 }
 
-fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out, void *stream) {
+fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
+                                int block_n, float *out, void *stream) {
   if (!A || !W || !out || R <= 0 || N <= 0 || K <= 0 || K % 8) return kfail(FVAR_EINVAL, "gemm: bad arguments");
+  if (form != FVAR_GEMM_AUTO && form != FVAR_GEMM_SINGLE && form != FVAR_GEMM_PAIR) return kfail(FVAR_EINVAL, "gemm: bad form");
   int dev = 0, sms = 0;
   FK_CUDA(cudaGetDevice(&dev), "get device");
   FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
-  const GemmPlan plan = gemm_plan(R, 1, N, K, sms, gemm_pair_max_clusters(), 1, 0);
+  const int max_clusters = form == FVAR_GEMM_SINGLE ? 0 : gemm_pair_max_clusters();
+  GemmPlan plan = gemm_plan(R, 1, N, K, sms, max_clusters, 1, 0);
+  if (form == FVAR_GEMM_PAIR) {
+    if (R <= 128 || max_clusters <= 0) return kfail(FVAR_EINVAL, "gemm: the pair form needs R > 128 and a device that runs CTA pairs");
+    if (block_n != 0 && block_n != 128 && block_n != 256) return kfail(FVAR_EINVAL, "gemm: pair block_n must be 128 or 256");
+    if (!plan.pair) plan = GemmPlan{true, (N > 128) ? 256 : 128, 1};
+    if (block_n) plan.block_n = block_n;
+  } else if (block_n != 0) {
+    if (form == FVAR_GEMM_AUTO) return kfail(FVAR_EINVAL, "gemm: block_n needs an explicit form");
+    if (block_n != 64 && block_n != 128 && block_n != 256) return kfail(FVAR_EINVAL, "gemm: block_n must be 64, 128 or 256");
+    plan.block_n = block_n;
+  }
   const int bn = plan.block_n;
   CUtensorMap ta, tw;
   if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, W, K, N, K, plan.pair ? bn / 2 : bn))
@@ -1045,6 +1058,10 @@ fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R
   else
     FK_CUDA(launch_gemm(EPI_F32, bn, ta, tw, g, sms, static_cast<cudaStream_t>(stream)), "gemm");
   return FVAR_OK;
+}
+
+fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out, void *stream) {
+  return fvar_gemm_bf16_form(A, W, bias, R, N, K, FVAR_GEMM_AUTO, 0, out, stream);
 }
 
 fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B, int H, int r, int D, int L, int L_cap,

@@ -106,6 +106,37 @@ def test_gemm_bf16(fv, R, N, K, bias):
     np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
 
 
+# Every launch form and tile width against the same fp64 product: single CTAs (64 / 128 / 256 columns)
+# and CTA pairs (256-row tiles of 128 / 256 columns), on shapes with ragged row, column and K edges, an
+# odd number of 128-row tiles (the second CTA of the last pair has no rows) and more tiles than CTAs.
+@pytest.mark.parametrize("R,N,K", [(256, 256, 64), (129, 128, 72), (300, 200, 136), (641, 1000, 520),
+                                   (1024, 3072, 1024), (3000, 4096, 256), (4500, 512, 2048)])
+@pytest.mark.parametrize("form,block_n", [("single", 64), ("single", 128), ("single", 256), ("pair", 128), ("pair", 256)])
+def test_gemm_bf16_every_form(fv, R, N, K, form, block_n):
+    rng = np.random.default_rng(7 * R + N + K)
+    A = si.normal_bf16(rng, (R, K))
+    W = si.normal_bf16(rng, (N, K), 0.05)
+    b = si.normal_bf16(rng, (N,))
+    f = fv.GEMM_PAIR if form == "pair" else fv.GEMM_SINGLE
+    got = fv.fvar_gemm_bf16_form(to_bf16_cuda(A), to_bf16_cuda(W), to_bf16_cuda(b), f, block_n).cpu().numpy()
+    _poll(fv)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T + b.astype(np.float64)
+    tol = 1e-5 * (np.abs(A).astype(np.float64) @ np.abs(W).astype(np.float64).T).max() + 1e-6
+    np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
+
+
+def test_gemm_form_rejects_what_the_problem_does_not_allow(fv):
+    A = to_bf16_cuda(np.zeros((128, 64), np.float32))
+    W = to_bf16_cuda(np.zeros((128, 64), np.float32))
+    with pytest.raises(fv.FvarError):
+        fv.fvar_gemm_bf16_form(A, W, None, fv.GEMM_PAIR, 128)       # a single row tile has no partner
+    A2 = to_bf16_cuda(np.zeros((256, 64), np.float32))
+    with pytest.raises(fv.FvarError):
+        fv.fvar_gemm_bf16_form(A2, W, None, fv.GEMM_PAIR, 64)       # pairs come 128 or 256 columns wide
+    with pytest.raises(fv.FvarError):
+        fv.fvar_gemm_bf16_form(A2, W, None, fv.GEMM_SINGLE, 96)
+
+
 # ----------------------------------------------------------------------------- attention
 
 def _cache_layout(K, V, H, D, L_cap):
