@@ -14,6 +14,7 @@ What the paper fixes and this file follows:
   * index set I: the r most important rows, |I| = r       (Sec. 3.3; Algorithm 1)
   * random projection  F_r = Q^T F,  Q in R^{M x r}, Q_ij ~ N(0, 1/r)
                                                           (Sec. 3.3 RP; Algorithm 1)
+    Q is either given as data or drawn from a seed (Philox4x32-10 + Box-Muller, below)
   * cached output upsampled, F^{o,cache}_{k-1} = Up(F^o_{k-1})   (Eq. "upcache")
   * restoration F^o_k := {F^o_r rows at I} U {cache rows elsewhere} (Eq. "redefine")
   * CFG = 0 in the fidelity-refinement stage = null-prompt branch only
@@ -123,6 +124,74 @@ def sampling_keys(scores: np.ndarray, noise: np.ndarray) -> np.ndarray:
 def random_projection(Q: np.ndarray, X: np.ndarray) -> np.ndarray:
     """F_r = Q^T X: [r][C] from Q [M][r] and X [M][C] (Algorithm 1, RP step)."""
     return Q.T @ X
+
+
+# --------------------------------------------------------------------------- seeded projection
+# The method draws Q itself (Sec. 3.3 RP: Q_ij ~ N(0, 1/r); the robustness figure redraws it per
+# generation), so both sides need the same draws from a seed.  The generator is Philox4x32-10
+# (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11), a counter-based
+# generator: output = ten rounds of a fixed bijection of a 128-bit counter under a 64-bit key.
+
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57      # round multipliers
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85      # key increments (Weyl sequence)
+
+
+def philox4x32_10(counter: np.ndarray, key) -> np.ndarray:
+    """counter uint32 [..., 4], key (k0, k1) -> uint32 [..., 4].  One round maps (c0, c1, c2, c3) to
+    (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)); the key is bumped by (W0, W1)
+    between rounds."""
+    c = np.asarray(counter, dtype=np.uint64) & np.uint64(0xFFFFFFFF)
+    c0, c1, c2, c3 = c[..., 0], c[..., 1], c[..., 2], c[..., 3]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    mask, sh = np.uint64(0xFFFFFFFF), np.uint64(32)
+    for _ in range(10):
+        p0 = np.uint64(PHILOX_M0) * c0
+        p1 = np.uint64(PHILOX_M1) * c2
+        c0, c1, c2, c3 = ((p1 >> sh) ^ c1 ^ np.uint64(k0), p1 & mask, (p0 >> sh) ^ c3 ^ np.uint64(k1), p0 & mask)
+        k0, k1 = (k0 + PHILOX_W0) & 0xFFFFFFFF, (k1 + PHILOX_W1) & 0xFFFFFFFF
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def round_f64_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 value (ties to even) of each fp64 element, in ONE rounding, returned as fp32.
+    Going through fp32 first would round twice: when the fp32 result lands exactly on a bf16 tie the
+    direction has to come from the fp64 value."""
+    x = np.asarray(x, dtype=np.float64)
+    f = x.astype(np.float32)
+    u = f.view(np.uint32).astype(np.int64)
+    tie = (u & 0xFFFF) == 0x8000
+    back = f.astype(np.float64)
+    # magnitude of the fp32 value above / below the true one: step the bits off the tie accordingly
+    u = np.where(tie & (np.abs(back) > np.abs(x)), u - 1, u)
+    u = np.where(tie & (np.abs(back) < np.abs(x)), u + 1, u)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32)
+
+
+def generate_projection(seed: int, scale_idx: int, group: int, M: int, r: int) -> np.ndarray:
+    """Q [M][r] with Q_ij ~ N(0, 1/r) (Sec. 3.3 RP), bf16-rounded, from a 64-bit seed.
+
+    Layout of the draws: Q^T is flattened row-major (element n = j * M + i holds Q_ij); call t of the
+    generator, counter (t, group, scale_idx, 0) under key (seed low, seed high), yields elements
+    4t .. 4t + 3.  From its words x0..x3: u = (x + 0.5) 2^-32 in (0, 1); Box-Muller on (u0, u1) and
+    (u2, u3): z = sqrt(-2 ln u_a) * (cos 2 pi u_b, sin 2 pi u_b); Q = z / sqrt(r), all in fp64, then
+    one rounding to bf16."""
+    n = M * r
+    calls = (n + 3) // 4
+    ctr = np.zeros((calls, 4), dtype=np.uint32)
+    ctr[:, 0] = np.arange(calls, dtype=np.uint32)
+    ctr[:, 1] = group
+    ctr[:, 2] = scale_idx
+    x = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)).astype(np.float64)
+    u = (x + 0.5) * 2.0 ** -32
+    z = np.empty((calls, 4), dtype=np.float64)
+    for a in (0, 2):
+        rad = np.sqrt(-2.0 * np.log(u[:, a]))
+        ang = 2.0 * np.pi * u[:, a + 1]
+        z[:, a] = rad * np.cos(ang)
+        z[:, a + 1] = rad * np.sin(ang)
+    qt = (z.reshape(-1)[:n] / math.sqrt(r)).reshape(r, M)
+    return np.ascontiguousarray(round_f64_to_bf16(qt).T)
 
 
 def upsample_bilinear(F: np.ndarray, hw_in, hw_out) -> np.ndarray:

@@ -471,3 +471,83 @@ def test_sampling_keys_exponential_race():
     assert list(orc.select_top_r(orc.sampling_keys(s, ones), 2)) == list(orc.select_top_r(s, 2))
     k = orc.sampling_keys(np.array([3.0], np.float32), np.array([7.0], np.float32))
     assert k.dtype == np.float32 and k[0] == np.float32(3.0) / np.float32(7.0)
+
+
+# ----------------------------------------------------------------------------- seeded projection
+
+def test_philox_known_answers():
+    """The counter-based generator behind the seeded projection against its published vectors."""
+    n = 0
+    with open(os.path.join(GOLD, "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if not line.strip() or line.startswith("#"):
+                continue
+            v = [int(t, 16) for t in line.split()]
+            out = orc.philox4x32_10(np.array(v[0:4], dtype=np.uint32), (v[4], v[5]))
+            assert [int(o) for o in out] == v[6:10]
+            n += 1
+    assert n == 2
+    # a bijection of the counter: distinct counters, distinct outputs; vectorised == one by one
+    ctr = np.zeros((64, 4), dtype=np.uint32)
+    ctr[:, 0] = np.arange(64)
+    outs = orc.philox4x32_10(ctr, (7, 9))
+    assert len({tuple(int(x) for x in o) for o in outs}) == 64
+    assert np.array_equal(outs[5], orc.philox4x32_10(ctr[5], (7, 9)))
+
+
+def test_round_f64_to_bf16_is_one_correct_rounding():
+    """Against exact rational arithmetic on the two neighbouring bf16 values, including values that a
+    detour through fp32 would round the wrong way (fp32 result exactly on a bf16 tie)."""
+    from fractions import Fraction
+    rng = np.random.default_rng(3)
+    xs = list(rng.standard_normal(200) * 10.0 ** rng.integers(-3, 3, 200))
+    base = float(np.float32(1.0) + np.float32(2.0 ** -8))           # a bf16 tie: 1 + half an ulp (ulp = 2^-7)
+    xs += [base, base * (1 + 2.0 ** -40), base * (1 - 2.0 ** -40), -base * (1 + 2.0 ** -40), 3 * base, 0.0, 2.0 ** -7]
+    got = orc.round_f64_to_bf16(np.array(xs))
+    for x, g in zip(xs, got):
+        if x == 0.0:
+            assert g == 0.0
+            continue
+        # neighbours: truncate |x| to 8 significant bits, and the next one up
+        m, e = math.frexp(abs(x))                         # |x| = m 2^e, m in [0.5, 1)
+        lo = Fraction(int(m * 256), 256) * Fraction(2) ** e
+        hi = lo + Fraction(1, 256) * Fraction(2) ** e
+        fx = Fraction(abs(x))
+        if fx - lo < hi - fx:
+            want = lo
+        elif fx - lo > hi - fx:
+            want = hi
+        else:                                             # tie: even significand
+            want = lo if int(m * 256) % 2 == 0 else hi
+        assert Fraction(float(abs(g))) == want, (x, g)
+        assert (g < 0) == (x < 0)
+
+
+def test_generated_projection_layout_and_distribution():
+    from scipy import stats
+    seed, k, g, M, r = 0x1234567812345678, 9, 3, 256, 96
+    Q = orc.generate_projection(seed, k, g, M, r)
+    assert Q.shape == (M, r) and Q.dtype == np.float32
+    assert np.array_equal(si.round_to_bf16(Q), Q)                      # bf16-representable
+    # layout: element n = j * M + i of the flattened Q^T comes from call n // 4, word pair (n % 4) // 2
+    for (i, j) in [(0, 0), (5, 0), (255, 95), (17, 40)]:
+        n = j * M + i
+        x = orc.philox4x32_10(np.array([n // 4, g, k, 0], dtype=np.uint32), (seed & 0xFFFFFFFF, seed >> 32))
+        a = 2 * ((n % 4) // 2)
+        u0, u1 = (int(x[a]) + 0.5) / 2 ** 32, (int(x[a + 1]) + 0.5) / 2 ** 32
+        rad, ang = math.sqrt(-2.0 * math.log(u0)), 2.0 * math.pi * u1
+        z = rad * (math.cos(ang) if n % 2 == 0 else math.sin(ang)) / math.sqrt(r)
+        assert abs(float(Q[i, j]) - z) <= 2.0 ** -8 * abs(z) + 1e-12
+    # distribution: N(0, 1/r) by Kolmogorov-Smirnov (bf16 rounding moves the CDF by < 2^-8 relative)
+    z = Q.astype(np.float64).ravel() * math.sqrt(r)
+    assert stats.kstest(z, "norm").pvalue > 1e-3
+    assert abs(z.mean()) < 5.0 / math.sqrt(z.size) and abs(z.var() - 1.0) < 0.03
+    # E[Q Q^T] = I_M: diagonal near 1, off-diagonal near 0 with the spread 1/sqrt(r)
+    QQ = Q.astype(np.float64) @ Q.astype(np.float64).T
+    assert abs(np.diag(QQ).mean() - 1.0) < 0.03
+    off = QQ[~np.eye(M, dtype=bool)]
+    assert abs(off.mean()) < 0.01 and abs(off.std() - 1.0 / math.sqrt(r)) < 0.02
+    # other (seed, scale, group) give other draws; the same arguments give the same matrix
+    assert np.array_equal(Q, orc.generate_projection(seed, k, g, M, r))
+    assert not np.array_equal(Q, orc.generate_projection(seed, k, g + 1, M, r))
+    assert not np.array_equal(Q, orc.generate_projection(seed + 1, k, g, M, r))
