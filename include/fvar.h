@@ -113,6 +113,20 @@ fvar_status fvar_set_cond(fvar_ctx *ctx, int B, const void *cond, const void *co
  * set before a FVAR_LOWRANK_RTR step whose group rank is r < M. */
 fvar_status fvar_set_projection(fvar_ctx *ctx, int scale_idx, int group, const void *Qt, int r);
 
+/* The same matrix drawn on the device from a 64-bit seed instead of given (Sec. 3.3 RP: Q_ij ~
+ * N(0, 1/r); the paper redraws Q per generation).  Generator: Philox4x32-10 (Salmon et al., SC'11);
+ * call t with counter (t, group, scale_idx, 0) and key (seed low word, seed high word) yields elements
+ * 4t .. 4t + 3 of Q^T flattened row-major (element j * M + i is Q_ij); uniforms u = (x + 0.5) 2^-32;
+ * Box-Muller on the word pairs (0, 1) and (2, 3) in fp64: z = sqrt(-2 ln u_a) (cos, sin)(2 pi u_b);
+ * Q = z / sqrt(r), rounded once to bf16.  Replaces any projection stored for (scale, group).
+ * FVAR_EINVAL unless 0 < r <= M. */
+fvar_status fvar_generate_projection(fvar_ctx *ctx, int scale_idx, int group, int r, unsigned long long seed);
+
+/* Copies the stored projection of (scale, group), transposed as it was given or drawn, to
+ * Qt_out dev bf16 [r][M] (asynchronous on the context's stream) and its rank to *r_host.
+ * FVAR_ESTATE if none is stored. */
+fvar_status fvar_get_projection(fvar_ctx *ctx, int scale_idx, int group, void *Qt_out, int *r_host);
+
 /* One scale step (Algorithm 1: the dense loop body, or the fidelity-refinement loop body RP -> blocks
  * -> RTR).  tokens dev bf16 [B][M][C] with M = h_k * w_k; out dev bf16 [B_eff][M][C], B_eff = B
  * (pair) or B/2 (null-only).  Stages this scale's K/V rows at the cache tail; they become visible

@@ -72,6 +72,8 @@ def load_library() -> ct.CDLL:
         "fvar_init": (i, [P(_Weights), P(_Cfg), vp, ct.c_size_t, vp, P(vp)]),
         "fvar_set_cond": (i, [vp, i, vp, vp]),
         "fvar_set_projection": (i, [vp, i, i, vp, i]),
+        "fvar_generate_projection": (i, [vp, i, i, i, ct.c_ulonglong]),
+        "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
         "fvar_scale_step": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_scale_step_host": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_kv_append": (i, [vp, i]),
@@ -107,7 +109,8 @@ def load_library() -> ct.CDLL:
     return lib
 
 
-EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_scale_step",
+EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_generate_projection",
+            "fvar_get_projection", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
@@ -289,6 +292,17 @@ class Fvar:
         """Qt bf16 [r][M]: the projection matrix of Sec. 3.3, transposed."""
         _dev(Qt, torch.bfloat16)
         self._check(self.lib.fvar_set_projection(self.ctx, scale_idx, group, Qt.data_ptr(), Qt.shape[0]))
+
+    def generate_projection(self, scale_idx: int, group: int, r: int, seed: int):
+        """Draws the projection of (scale, group) on the device from a 64-bit seed (Philox4x32-10 + Box-Muller)."""
+        self._check(self.lib.fvar_generate_projection(self.ctx, scale_idx, group, r, seed & 0xFFFFFFFFFFFFFFFF))
+
+    def get_projection(self, scale_idx: int, group: int, M: int) -> torch.Tensor:
+        """The stored projection of (scale, group), transposed: bf16 [r][M] (M = tokens of that scale)."""
+        buf = torch.empty((M, M), dtype=torch.bfloat16, device="cuda")
+        r = ct.c_int(0)
+        self._check(self.lib.fvar_get_projection(self.ctx, scale_idx, group, buf.data_ptr(), ct.byref(r)))
+        return buf.view(-1)[: r.value * M].view(r.value, M)
 
     def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise=None):
         pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None, SELECT_TOPR, None)

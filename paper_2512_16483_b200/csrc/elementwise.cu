@@ -436,6 +436,64 @@ cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int 
 }
 
 // ------------------------------------------------------------------------------------------------
+// Projection drawn from a seed (Q_ij ~ N(0, 1/r), Sec. 3.3 RP of the paper).  Philox4x32-10 (Salmon et
+// al., SC'11): call t, counter (t, group, scale, 0) under key (seed low, seed high), gives elements
+// 4t .. 4t + 3 of Q^T flattened row-major (element n = j * M + i is Q_ij).  Uniforms u = (x + 0.5) 2^-32,
+// Box-Muller on the word pairs (0, 1) and (2, 3) in fp64, one rounding to bf16.  Each value is written
+// to both halves of the stored [Q^T | Q^T] row (row stride 2 * Mk).
+__device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
+  const uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
+  const uint32_t hi1 = __umulhi(0xCD9E8D57u, c[2]), lo1 = 0xCD9E8D57u * c[2];
+  const uint32_t n0 = hi1 ^ c[1] ^ k0, n2 = hi0 ^ c[3] ^ k1;
+  c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+}
+
+__global__ void __launch_bounds__(256) generate_projection_kernel(bf16 *__restrict__ qt, int M, int Mk, int r,
+                                                                  uint32_t key0, uint32_t key1, uint32_t group,
+                                                                  uint32_t scale) {
+  const long long n_total = static_cast<long long>(M) * r;
+  const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (4 * t >= n_total) return;
+  uint32_t c[4] = {static_cast<uint32_t>(t), group, scale, 0u};
+  uint32_t k0 = key0, k1 = key1;
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    philox_round(c, k0, k1);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  const double sqrt_r = sqrt(static_cast<double>(r));
+  double z[4];
+#pragma unroll
+  for (int a = 0; a < 4; a += 2) {
+    const double u0 = (static_cast<double>(c[a]) + 0.5) * 0x1p-32, u1 = (static_cast<double>(c[a + 1]) + 0.5) * 0x1p-32;
+    const double rad = sqrt(-2.0 * log(u0)), ang = (2.0 * 3.141592653589793) * u1;
+    z[a] = rad * cos(ang);
+    z[a + 1] = rad * sin(ang);
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const long long n = 4 * t + q;
+    if (n < n_total) {
+      const int j = static_cast<int>(n / M), i = static_cast<int>(n - static_cast<long long>(j) * M);
+      const bf16 v = __double2bfloat16(z[q] / sqrt_r);
+      qt[static_cast<long long>(j) * 2 * Mk + i] = v;
+      qt[static_cast<long long>(j) * 2 * Mk + Mk + i] = v;
+    }
+  }
+}
+
+cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned long long seed, int group, int scale,
+                                       cudaStream_t st) {
+  const long long calls = (static_cast<long long>(M) * r + 3) / 4;
+  if (calls <= 0) return cudaSuccess;
+  generate_projection_kernel<<<static_cast<unsigned>((calls + 255) / 256), 256, 0, st>>>(
+      qt, M, Mk, r, static_cast<uint32_t>(seed & 0xFFFFFFFFull), static_cast<uint32_t>(seed >> 32),
+      static_cast<uint32_t>(group), static_cast<uint32_t>(scale));
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Transposed two-term bf16 split of the fp32 rows for the projection GEMM:
 // xt[e][c][m] = hi(x[row(e, m)][c]) and xt[e][c][Mk + m] = lo(...), hi = bf16(x), lo = bf16(x - hi),
 // so that the tensor-core product Q^T (hi + lo) carries ~16 mantissa bits of x.  Mk = M rounded up

@@ -629,6 +629,36 @@ fvar_status fvar_set_projection(fvar_ctx *ctx, int scale_idx, int group, const v
   return FVAR_OK;
 }
 
+fvar_status fvar_generate_projection(fvar_ctx *ctx, int scale_idx, int group, int r, unsigned long long seed) {
+  if (!ctx) return FVAR_EINVAL;
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || group < 0 || group >= ctx->G)
+    return fail(ctx, FVAR_EINVAL, "generate_projection: bad scale / group");
+  const int M = ctx->Mk[scale_idx];
+  if (r <= 0 || r > M) return fail(ctx, FVAR_EINVAL, "generate_projection: need 0 < r <= M");
+  const size_t Mk = align_up(M, 64), slot = static_cast<size_t>(scale_idx) * ctx->G + group;
+  bf16 *dst = ctx->qt_pool + ctx->qt_off[slot];
+  // the padding columns [M, Mk) of both halves stay zero from fvar_init (nothing ever writes them)
+  FV_CUDA(ctx, launch_generate_projection(dst, M, static_cast<int>(Mk), r, seed, group, scale_idx, ctx->st), "generate_projection");
+  ctx->launched();
+  if (!tmap_2d(&ctx->qt_map[slot], dst, Mk + M, r, 2 * Mk, 128)) return fail(ctx, FVAR_ECUDA, "projection tensor map");
+  ctx->qt_r[slot] = r;
+  return FVAR_OK;
+}
+
+fvar_status fvar_get_projection(fvar_ctx *ctx, int scale_idx, int group, void *Qt_out, int *r_host) {
+  if (!ctx) return FVAR_EINVAL;
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || group < 0 || group >= ctx->G || !Qt_out || !r_host)
+    return fail(ctx, FVAR_EINVAL, "get_projection: bad arguments");
+  const size_t slot = static_cast<size_t>(scale_idx) * ctx->G + group;
+  const int r = ctx->qt_r[slot], M = ctx->Mk[scale_idx];
+  if (r <= 0) return fail(ctx, FVAR_ESTATE, "get_projection: no projection stored for this scale and group");
+  const size_t Mk = align_up(M, 64);
+  FV_CUDA(ctx, cudaMemcpy2DAsync(Qt_out, static_cast<size_t>(M) * 2, ctx->qt_pool + ctx->qt_off[slot], 2 * Mk * 2,
+                                 static_cast<size_t>(M) * 2, r, cudaMemcpyDeviceToDevice, ctx->st), "projection copy");
+  *r_host = r;
+  return FVAR_OK;
+}
+
 fvar_status fvar_load_kv(fvar_ctx *ctx, const void *K, const void *V, int L) {
   if (!ctx) return FVAR_EINVAL;
   if (ctx->B <= 0) return fail(ctx, FVAR_ESTATE, "load_kv before set_cond");

@@ -134,6 +134,8 @@ cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int
                                   cudaStream_t st);
 cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st);
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);
+cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned long long seed, int group, int scale,
+                                       cudaStream_t st);
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
 cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,
                            cudaStream_t st);

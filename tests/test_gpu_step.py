@@ -374,3 +374,40 @@ def test_edge_ranks_and_batches(fv, B, cfg):
     assert_out_close(got, ref, what="r = M - 1 / r = 1 after a late scale")
     e0 = 1 if cfg == "null_only" else 0
     assert p.gpu.cache_len(0) == p.oracle.cache_len(0, e0) and p.gpu.cache_len(1) == p.oracle.cache_len(1, e0)
+
+
+@pytest.mark.parametrize("M_side,r", [(16, 128), (13, 85), (16, 255), (10, 1)])
+def test_generated_projection_matches_oracle_bit_for_bit(fv, M_side, r):
+    """Q drawn on the device from a seed (Philox4x32-10 + Box-Muller in fp64, one rounding to bf16)
+    against the oracle's draw: same bits, for row lengths that are and are not multiples of 4 or 64."""
+    shp = si.shape_var_d16(n_blocks=2)
+    k = {10: 7, 13: 8, 16: 9}[M_side]
+    M = M_side * M_side
+    p = Pair(fv, shp, seed=111, B=2)
+    seed = 0x9E3779B97F4A7C15
+    for g in range(2):
+        p.gpu.generate_projection(k, g, r, seed)
+        got = bf16_to_numpy(p.gpu.get_projection(k, g, M))
+        want = orc.generate_projection(seed, k, g, M, r).T
+        assert got.shape == want.shape == (r, M)
+        assert np.array_equal(got, want), "group %d: %d of %d entries differ" % (g, (got != want).sum(), got.size)
+    p.check_ok()
+
+
+def test_step_with_generated_projection(fv):
+    """A late step whose projections both sides draw from the same seed instead of taking them as data."""
+    shp = si.shape_var_d16(n_blocks=2)
+    B, k, M, r = 2, 9, 256, 96
+    p = Pair(fv, shp, seed=112, B=B)
+    p.prefill(k)
+    for g in range(2):
+        p.gpu.generate_projection(k, g, r, 2024 + g)
+        p.oracle.set_projection(k, g, orc.generate_projection(2024 + g, k, g, M, r))
+    toks = si.make_tokens(112, B, M, 1024, "spread")
+    got, ref = _step_both(p, toks, k, mode=fv.LOWRANK_RTR, ranks=[r, r])
+    assert_out_close(got, ref, what="step with generated projection")
+    # a given matrix replaces a generated one and the other way round
+    p.set_projections(k, [r, r])
+    got2, ref2 = _step_both(p, toks, k, mode=fv.LOWRANK_RTR, ranks=[r, r])
+    assert_out_close(got2, ref2, what="step after replacing the projection")
+    assert not np.array_equal(got, got2)
