@@ -4,9 +4,11 @@
 //   warp 0      streams K and V^T tiles of 128 keys through a ring of shared-memory slots (TMA);
 //   warp 1      issues S_t = Q_t K^T and O_t += P_t V on the tensor cores, accumulators in TMEM;
 //   warps 2-5   softmax of tile 0, one query row per thread;   warps 6-9: softmax of tile 1.
-// The two tiles run out of phase: while one warp-group turns S into P (row max, exp2, bf16 P into
-// a swizzled shared tile), the tensor core works for the other tile (P V of block j, then Q K^T
-// of block j+1).  O stays in TMEM for the whole key loop; its rows are rescaled only when the
+// The two tiles run out of phase: while one warp-group turns S into P (row max, exp2, bf16 P
+// written back into the TMEM columns S came from), the tensor core works for the other tile (P V of
+// block j, with P read from TMEM as the A operand, then Q K^T of block j+1).  Keeping P out of shared
+// memory matters: the operand reads of the MMAs alone nearly fill the 128 B/clk of shared-memory
+// bandwidth, and a P tile costs one write and one read on top.  O stays in TMEM for the whole key loop; its rows are rescaled only when the
 // running maximum has grown by more than 2^8 since the last rescale, so the common case costs no
 // TMEM round trip.  Keys at or beyond L are masked.  Every wait is bounded (see ptx.cuh).
 #include <math.h>
@@ -25,12 +27,12 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 template <int D>
 struct AttnCfg {
   static constexpr int kTileBytes = 128 * D * 2;          // a Q tile, a K tile [128 keys][D] or a V^T tile [D][128 keys]
-  static constexpr int kRing = (D == 64) ? 6 : 3;         // K_j, V_j, K_{j+1}, ...
+  static constexpr int kRing = (D == 64) ? 10 : 5;        // K_j, V_j, K_{j+1}, ...
   static constexpr int kQBytes = 2 * kTileBytes;
-  static constexpr int kPTile = kQRows * kKeys * 2;
-  static constexpr int kPBytes = 2 * kPTile;
-  static constexpr int kSmemBytes = kQBytes + kRing * kTileBytes + kPBytes + 1024 + 256;
-  static constexpr int kTmemCols = 512;   // S0 [0,128), S1 [128,256), O0 [256,256+D), O1 [256+D,256+2D)
+  static constexpr int kSmemBytes = kQBytes + kRing * kTileBytes + 1024 + 256;
+  // TMEM: S0 [0,128), S1 [128,256), O0 [256,256+D), O1 [256+D,256+2D).  P (bf16, two keys per 32-bit
+  // column) overwrites columns [0,64) of the S buffer it was computed from.
+  static constexpr int kTmemCols = 512;
   static_assert(kSmemBytes > 116 * 1024, "one CTA per SM (the CTA allocates all of TMEM)");
   static_assert(kSmemBytes + 64 <= 227 * 1024, "shared memory");
   static_assert(256 + 2 * D <= 512, "TMEM columns");
@@ -50,8 +52,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = smem_base;
   const uint32_t ring_smem = q_smem + Cfg::kQBytes;
-  const uint32_t p_smem = ring_smem + NR * Cfg::kTileBytes;
-  const uint32_t bar_base = p_smem + Cfg::kPBytes;
+  const uint32_t bar_base = ring_smem + NR * Cfg::kTileBytes;
   const uint32_t q_full = bar_base;
   auto ring_full = [&](int s) { return bar_base + 8u * (1 + s); };
   auto ring_empty = [&](int s) { return bar_base + 8u * (1 + NR + s); };
@@ -152,13 +153,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         umma_commit(s_full(buf));
       };
-      auto issue_pv = [&](int t, int slot, bool accumulate) {   // O_t (+)= P_t V
-        const uint32_t vs = ring_smem + slot * Cfg::kTileBytes, ps = p_smem + t * Cfg::kPTile;
+      auto issue_pv = [&](int t, int pbuf, int slot, bool accumulate) {   // O_t (+)= P V, P in S buffer `pbuf`
+        const uint32_t vs = ring_smem + slot * Cfg::kTileBytes;
 #pragma unroll
         for (int k = 0; k < kKeys / 16; ++k) {
-          const uint64_t da = smem_desc_sw128(ps + (k / 4) * kAtomBytes) + 2 * (k % 4);
           const uint64_t db = smem_desc_sw128(vs + (k / 4) * (D * 128)) + 2 * (k % 4);
-          umma_bf16(tmem_base + 256 + t * D, da, db, idesc_o, (accumulate || k != 0) ? 1u : 0u);
+          // 16 keys of P = 8 columns of TMEM (two bf16 per column)
+          umma_bf16_tmem_a(tmem_base + 256 + t * D, tmem_base + pbuf * kKeys + 8 * k, db, idesc_o, (accumulate || k != 0) ? 1u : 0u);
         }
         umma_commit(o_full(t));
       };
@@ -183,7 +184,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (!mbar_wait(p_full(0), j & 1u, p.status, &abort_flag)) { ok = false; break; }
           if (!mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
           tc_fence_after();
-          issue_pv(0, vi % NR, j > 0);
+          issue_pv(0, j & 1, vi % NR, j > 0);
           umma_commit(ring_empty(vi % NR));
         }
       } else
@@ -193,7 +194,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (!mbar_wait(p_full(t), j & 1u, p.status, &abort_flag)) { ok = false; break; }
           if (t == 0 && !mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
           tc_fence_after();
-          issue_pv(t, vi % NR, j > 0);
+          issue_pv(t, t, vi % NR, j > 0);
           if (t == ntiles - 1) umma_commit(ring_empty(vi % NR));
           if (j + 1 < nkv) {
             if (t == 0 && !mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
@@ -214,7 +215,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const bool single = (ntiles == 1);               // then S alternates between the two S buffers
       const uint32_t s_base = tmem_base + lane_addr;
       const uint32_t o_addr = tmem_base + 256 + t * D + lane_addr;
-      const uint32_t p_row = p_smem + t * Cfg::kPTile + row_local * 128;
       const float c = p.scale_log2;
       float m_ref = -INFINITY, l_run = 0.f;
       bool ok = true;
@@ -272,30 +272,26 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const float neg_mc = -m_ref * c;
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t pk[16];
+        for (int half = 0; half < 2; ++half) {
+          // keys 64 * half .. 64 * half + 63 of this row, two per word: 32 TMEM columns.  The whole S
+          // row is in registers by now, so overwriting its first columns loses nothing.
+          uint32_t pk[32];
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float p0 = exp2f(fmaf(__uint_as_float(v[cc][i]), c, neg_mc));       // exp2(-inf) = 0 for masked keys
-            const float p1 = exp2f(fmaf(__uint_as_float(v[cc][i + 1]), c, neg_mc));
-            ls[(i >> 1) & 3] += p0 + p1;
-            __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-            pk[i >> 1] = *reinterpret_cast<uint32_t *>(&v2);
-          }
-          // columns cc*32 .. cc*32+31 of this row: four 16-byte chunks of the swizzled tile
-          const uint32_t atom = p_row + (cc >> 1) * kAtomBytes;
+          for (int cc = 2 * half; cc < 2 * half + 2; ++cc) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint32_t chunk = static_cast<uint32_t>((cc & 1) * 4 + q);
-            const uint32_t addr = atom + ((chunk ^ (row_local & 7)) << 4);
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q * 4]), "r"(pk[q * 4 + 1]),
-                         "r"(pk[q * 4 + 2]), "r"(pk[q * 4 + 3])
-                         : "memory");
+            for (int i = 0; i < 32; i += 2) {
+              const float p0 = exp2f(fmaf(__uint_as_float(v[cc][i]), c, neg_mc));       // exp2(-inf) = 0 for masked keys
+              const float p1 = exp2f(fmaf(__uint_as_float(v[cc][i + 1]), c, neg_mc));
+              ls[(i >> 1) & 3] += p0 + p1;
+              __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+              pk[(cc & 1) * 16 + (i >> 1)] = *reinterpret_cast<uint32_t *>(&v2);
+            }
           }
+          tmem_st32(s_addr + half * 32, pk);
         }
         const float l_blk = (ls[0] + ls[1]) + (ls[2] + ls[3]);
         l_run += l_blk;
-        fence_proxy_async_smem();
+        tmem_st_wait();
         tc_fence_before();
         mbar_arrive(p_full(t));
       }
