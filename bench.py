@@ -53,6 +53,23 @@ WORKLOADS = {
 }
 
 
+def resolve_workload(name):
+    """A named workload, or a point of the last-scale sweep on the Infinity-2B shape:
+    `infinity2b_last_r<R>_b<B>` = only the 64 x 64 scale (4096 queries over a cache pre-filled with 6425 rows),
+    batch B, every block group at rank R.  R < 4096 runs the method (null-prompt branch only, RP + RTR);
+    R = 4096 is the unpruned dense path with both CFG branches."""
+    import re
+    if name in WORKLOADS:
+        return WORKLOADS[name]
+    m = re.fullmatch(r"infinity2b_last_r(\d+)_b(\d+)", name)
+    if not m:
+        raise SystemExit("unknown workload %r (named: %s; or infinity2b_last_r<R>_b<B>)" % (name, ", ".join(sorted(WORKLOADS))))
+    R, B = int(m.group(1)), int(m.group(2))
+    if not (1 <= R <= 4096) or B < 1 or (R < 4096 and B % 2):
+        raise SystemExit("need 1 <= R <= 4096 and a batch of whole CFG pairs")
+    return dict(shape="inf2b", B=B, first_late=12, keep=("rank", R), null_only=R < 4096)
+
+
 def scale_plan(wl, shp):
     """Per late scale index: None (skip) or the list of ranks per block group (M = dense)."""
     from paper_2512_16483_b200 import schedule
@@ -61,6 +78,8 @@ def scale_plan(wl, shp):
         keep = wl["keep"]
         if k < wl.get("dense_until", 0):
             plan[k] = [Ms[k]] * shp.n_groups
+        elif isinstance(keep, tuple):
+            plan[k] = [min(keep[1], Ms[k])] * shp.n_groups
         elif keep in ("table", "paper"):
             side = shp.scales[k]
             if keep == "paper" and schedule.INFINITY_ALPHA[schedule.INFINITY_LATE_SCALES.index(side)] == 0.0:
@@ -214,19 +233,21 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="var_d16_late3_b16", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="var_d16_late3_b16",
+                    help="one of %s, or infinity2b_last_r<R>_b<B>" % ", ".join(sorted(WORKLOADS)))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--max-splits", type=int, default=0, help="tuning: largest split-K factor (1, 2, 4); 0 = library default")
     ap.add_argument("--profile-run", action="store_true",
                     help="for runs under ncu: skip the host-buffer leg, the event pass and the CPU baseline")
     args = ap.parse_args()
-    wl = WORKLOADS[args.workload]
+    wl = resolve_workload(args.workload)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     metric = "tokens/s over the late scale steps (output positions delivered per second)"
     config = {"workload": args.workload, "shape": wl["shape"], "batch": wl["B"],
-              "late_scale_sides": list(make_shape(wl["shape"]).scales[wl["first_late"]:]), "keep": wl["keep"],
+              "late_scale_sides": list(make_shape(wl["shape"]).scales[wl["first_late"]:]),
+              "keep": "rank %d" % wl["keep"][1] if isinstance(wl["keep"], tuple) else wl["keep"],
               "cfg": "null_only" if wl["null_only"] else "pair",
               "l2": "inputs_exceed_l2 (the stack's weights, streamed every step, are larger than L2)"}
 
@@ -401,7 +422,7 @@ def main():
     value = whole_job_value(tokens_per_step, args.steps, world, ms_total)
     e2e = whole_job_value(tokens_per_step, args.steps, world, ms_e2e)
     g = classes.get("gemm", {"tflops": 0.0})
-    roofline = {"bound": "tensor", "kernel": "gemm_kernel (every tile width and epilogue the step launches)",
+    roofline = {"bound": "tensor", "kernel": "gemm_kernel + gemm_pair_kernel (every tile width and epilogue the step launches)",
                 "achieved": g["tflops"], "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                 "frac": g["tflops"] / pk["bf16_sustained"], "peak_source": pk["source"] + ", sustained bf16",
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload), "traffic_unit": "bytes per launch (ncu, cold cache)",

@@ -497,26 +497,32 @@ cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned 
 // Transposed two-term bf16 split of the fp32 rows for the projection GEMM:
 // xt[e][c][m] = hi(x[row(e, m)][c]) and xt[e][c][Mk + m] = lo(...), hi = bf16(x), lo = bf16(x - hi),
 // so that the tensor-core product Q^T (hi + lo) carries ~16 mantissa bits of x.  Mk = M rounded up
-// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  64 x 32 tiles
-// through shared memory, two tokens (one bf16x2) per lane on the way out.
+// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  A CTA moves a tile of
+// 64 tokens x 128 channels through shared memory: 512-byte row segments in (one float4 per lane), 128-byte
+// channel rows out (two tokens, one bf16x2, per lane).  C % 4 == 0.
+constexpr int kTrTok = 64, kTrCh = 128;
 __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
                                                              int Mk, bf16 *__restrict__ xt) {
   pdl_wait();
   pdl_launch_dependents();
-  __shared__ float tile[64][33];                 // 64 token rows x 32 channels
-  const int e = blockIdx.z, m0 = blockIdx.x * 64, c0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  __shared__ float tile[kTrTok][kTrCh + 1];      // odd row stride: the column reads below do not conflict
+  const int e = blockIdx.z, m0 = blockIdx.x * kTrTok, c0 = blockIdx.y * kTrCh;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float *src = x + static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb * C;
-  for (int k = ty; k < 64; k += 8) {
-    const int m = m0 + k, c = c0 + tx;
-    tile[k][tx] = (m < M && c < C) ? src[static_cast<long long>(m) * C + c] : 0.f;
+#pragma unroll
+  for (int k = warp; k < kTrTok; k += 8) {
+    const int m = m0 + k, c = c0 + 4 * lane;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (m < M && c < C) v = __ldg(reinterpret_cast<const float4 *>(src + static_cast<long long>(m) * C + c));
+    tile[k][4 * lane] = v.x; tile[k][4 * lane + 1] = v.y; tile[k][4 * lane + 2] = v.z; tile[k][4 * lane + 3] = v.w;
   }
   __syncthreads();
   bf16 *dst = xt + static_cast<long long>(e) * C * 2 * Mk;
-  for (int k = ty; k < 32; k += 8) {             // one channel per warp pass; each lane writes two tokens
-    const int c = c0 + k, m = m0 + 2 * tx;
+#pragma unroll 4
+  for (int k = warp; k < kTrCh; k += 8) {        // one channel per warp pass; each lane writes two tokens
+    const int c = c0 + k, m = m0 + 2 * lane;
     if (c < C) {                                 // m + 1 < Mk always: Mk is a multiple of 64
-      const float v0 = tile[2 * tx][k], v1 = tile[2 * tx + 1][k];
+      const float v0 = tile[2 * lane][k], v1 = tile[2 * lane + 1][k];
       const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
       const float2 hf = __bfloat1622float2(hi);
       const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - hf.x, v1 - hf.y);
@@ -528,7 +534,8 @@ __global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__rest
 
 cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
                                   cudaStream_t st) {
-  dim3 grid(Mk / 64, (C + 31) / 32, E);
+  if (C % 4 != 0) return cudaErrorInvalidValue;
+  dim3 grid(Mk / kTrTok, (C + kTrCh - 1) / kTrCh, E);
   return launch_pdl(transpose_bf16_kernel, dim3(grid), dim3(256), 0, st, x, xmap, M, C, Mk, xt);
 }
 
