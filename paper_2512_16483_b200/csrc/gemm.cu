@@ -386,8 +386,7 @@ static int forced_pair() {
   static int v = -2;
   if (v == -2) {
     const char *e = getenv("FVAR_GEMM_PAIR");
-    v = e ? atoi(e) : -1;
-    if (v != 0 && v != 1) v = -1;
+    v = (e && (e[0] == '0' || e[0] == '1') && e[1] == 0) ? e[0] - '0' : -1;
   }
   return v;
 }

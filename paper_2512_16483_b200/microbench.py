@@ -1,6 +1,7 @@
 """Stand-alone timings of the library's kernels through the C ABI (CUDA events, one GPU).
 
-    python -m paper_2512_16483_b200.microbench gemm        # tile-width sweep: FVAR_GEMM_BLOCK_N=64|128|256 forces a width
+    python -m paper_2512_16483_b200.microbench gemm        # FVAR_GEMM_BLOCK_N=64|128|256 forces a width, FVAR_GEMM_PAIR=0|1 the launch form
+    python -m paper_2512_16483_b200.microbench gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
     python -m paper_2512_16483_b200.microbench attention
     python -m paper_2512_16483_b200.microbench memory      # score, LayerNorm + modulate, restoration fill, selection
 
@@ -30,6 +31,25 @@ def _time(fn, n=20, warm=3):
     return e0.elapsed_time(e1) * 1e3 / n          # microseconds
 
 
+def _gemm_graph_us(lib, R, N, K):
+    ncopy = max(2, min(32, int(300e6 // (N * K * 2))))
+    A = torch.randn(R, K, device="cuda").bfloat16()
+    Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(ncopy)]
+    out = torch.empty(R, N, device="cuda", dtype=torch.float32)
+
+    def call(i):
+        lib.fvar_gemm_bf16(A.data_ptr(), Ws[i % ncopy].data_ptr(), None, R, N, K, out.data_ptr(),
+                           torch.cuda.current_stream().cuda_stream)
+    for i in range(ncopy):
+        call(i)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(ncopy):
+            call(i)
+    return _time(g.replay, n=5, warm=1) / ncopy
+
+
 def gemm():
     lib = fv.load_library()
     bn = os.environ.get("FVAR_GEMM_BLOCK_N", "auto")
@@ -37,24 +57,17 @@ def gemm():
               (16, 2048, 2048), (16, 2048, 8192), (336, 8192, 2048), (4096, 4096, 1024), (8192, 8192, 2048),
               (16384, 4096, 4096)]
     for R, N, K in shapes:
-        ncopy = max(2, min(32, int(300e6 // (N * K * 2))))
-        A = torch.randn(R, K, device="cuda").bfloat16()
-        Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(ncopy)]
-        out = torch.empty(R, N, device="cuda", dtype=torch.float32)
-
-        def call(i):
-            lib.fvar_gemm_bf16(A.data_ptr(), Ws[i % ncopy].data_ptr(), None, R, N, K, out.data_ptr(),
-                               torch.cuda.current_stream().cuda_stream)
-        for i in range(ncopy):
-            call(i)
-        torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for i in range(ncopy):
-                call(i)
-        us = _time(g.replay, n=5, warm=1) / ncopy
+        us = _gemm_graph_us(lib, R, N, K)
         print("BN=%s R=%d N=%d K=%d: %.2f us  %.1f TFLOP/s  weights %.0f GB/s" % (
             bn, R, N, K, us, 2 * R * N * K / us / 1e6, N * K * 2 / us / 1e3))
+
+
+def gemmk():
+    lib = fv.load_library()
+    tag = "PAIR=%s BN=%s" % (os.environ.get("FVAR_GEMM_PAIR", "model"), os.environ.get("FVAR_GEMM_BLOCK_N", "model"))
+    for R, N in [(1024, 3072), (1024, 1024), (4096, 4096)]:
+        res = ["K=%d: %.2f us" % (K, _gemm_graph_us(lib, R, N, K)) for K in (128, 256, 512, 1024, 2048, 4096)]
+        print(tag, "R=%d N=%d |" % (R, N), "  ".join(res), flush=True)
 
 
 def attention():
@@ -104,4 +117,4 @@ def memory():
 
 if __name__ == "__main__":
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
-    {"gemm": gemm, "attention": attention, "memory": memory}[which]()
+    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory}[which]()
