@@ -395,12 +395,13 @@ def main():
     ms_e2e, _ = (ms_total, 0) if args.profile_run else timed(step_host, args.steps, 2)
     assert ctx.poll_status() == fv.OK, "device status word reports an error"
 
-    # per-kernel-class event timing: a separate pass over the same steps, events around every launch
+    # per-kernel-class event timing: a separate pass over the same steps; the library re-captures the step's graph
+    # with event-record nodes around every kernel node, so the kernels are timed inside the graph
     ctx.profile_enable(True)
     prof_steps = 0 if args.profile_run else max(1, min(args.steps, 10))
     for _ in range(prof_steps):
-        # Hold the stream back (a device-side delay of about 10 ms) while the host enqueues the step, so
-        # that the interval between a launch's two events is the kernel, not the host's submission rate.
+        # Hold the stream back (a device-side delay of about 10 ms) while the host captures and enqueues the
+        # step, so that no interval between two events contains host time.
         torch.cuda._sleep(20_000_000)
         step_device()
     classes = {}
@@ -426,7 +427,7 @@ def main():
                 "achieved": g["tflops"], "peak": pk["bf16_sustained"], "unit": "TFLOP/s",
                 "frac": g["tflops"] / pk["bf16_sustained"], "peak_source": pk["source"] + ", sustained bf16",
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload), "traffic_unit": "bytes per launch (ncu, cold cache)",
-                "algorithmic_bytes_per_launch": (g["gbs"] * 1e9 * g["avg_us"] * 1e-6) if "gbs" in g else None, "how": "separate pass of %d steps with CUDA events around every launch, enqueued behind a device-side delay" % prof_steps,
+                "algorithmic_bytes_per_launch": (g["gbs"] * 1e9 * g["avg_us"] * 1e-6) if "gbs" in g else None, "how": "separate pass of %d steps: the step's CUDA graph re-captured with an event-record node before and after every kernel node" % prof_steps,
                 "classes": classes}
     line = {
         "metric": metric, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": warm,

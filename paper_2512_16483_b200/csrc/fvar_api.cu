@@ -164,15 +164,29 @@ struct fvar_ctx {
     }
     return ev_pool[ev_used++];
   }
-  void prof_begin(int kclass, double flops, double bytes) {
+  // While a graph is being captured an event becomes an event-record node of the graph (the "external"
+  // flag), so that the profile pass times the kernels where the timed run executes them: inside the graph,
+  // without the host between launches.  `s`: the stream of the launch (default: where launches go).
+  void prof_record(cudaEvent_t e, cudaStream_t s) {
+    if (launch_st == cap_st && cap_st != nullptr && launch_st != st)
+      cudaEventRecordWithFlags(e, s, cudaEventRecordExternal);
+    else
+      cudaEventRecord(e, s);
+  }
+  void prof_begin(int kclass, double flops, double bytes, cudaStream_t s = nullptr) {
     if (!prof_on) return;
     ProfRec r{kclass, flops, bytes, event(), event()};
-    cudaEventRecord(r.e0, st);
+    prof_record(r.e0, s ? s : launch_st);
     prof.push_back(r);
   }
-  void launched() {
+  void launched(cudaStream_t s = nullptr) {
     launches++;
-    if (prof_on && !prof.empty()) cudaEventRecord(prof.back().e1, st);
+    if (prof_on && !prof.empty()) prof_record(prof.back().e1, s ? s : launch_st);
+  }
+  std::vector<cudaGraphExec_t> prof_execs;   // graphs instantiated by the profile pass (one per step, not cached)
+  void drop_prof_execs() {
+    for (cudaGraphExec_t e : prof_execs) cudaGraphExecDestroy(e);
+    prof_execs.clear();
   }
   const CUtensorMap &wm(int blk, int wid, int bn) const { return wmap[(blk * W_COUNT + wid) * 3 + bn_index(bn)]; }
 };
@@ -504,6 +518,7 @@ fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value) {
 fvar_status fvar_profile_enable(fvar_ctx *ctx, int on) {
   if (!ctx) return FVAR_EINVAL;
   FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  ctx->drop_prof_execs();
   ctx->prof.clear();
   ctx->ev_used = 0;
   ctx->prof_on = on != 0;
@@ -540,6 +555,7 @@ fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long 
 void fvar_destroy(fvar_ctx *ctx) {
   if (!ctx) return;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  ctx->drop_prof_execs();
   ctx->drop_graphs();
   if (ctx->cap_st) cudaStreamDestroy(ctx->cap_st);
   if (ctx->cap_st2) cudaStreamDestroy(ctx->cap_st2);
@@ -775,23 +791,23 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         side = ctx->cap_st2;
       }
       if (pol->forced_indices) {
-        ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * E * (M + 2.0 * r));
+        ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * E * (M + 2.0 * r), side);
         FV_CUDA(ctx, launch_copy_indices(pol->forced_indices + static_cast<size_t>(g) * E * r_max, E, M, r, r_max, idx_g,
                                          inv_g, ctx->status, side), "copy_indices");
-        ctx->launched();
+        ctx->launched(side);
       } else {
-        ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M);
+        ctx->prof_begin(FVAR_KCLASS_SCORE, 2.0 * E * M * C, 4.0 * E * M * C + 4.0 * E * M, side);
         FV_CUDA(ctx, launch_row_scores(X_in, bmap, E, M, C,
                                        sampled ? pol->sample_noise + static_cast<size_t>(g) * E * M : nullptr, ctx->scores, side), "row_scores");
-        ctx->launched();
-        ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r));
+        ctx->launched(side);
+        ctx->prof_begin(FVAR_KCLASS_SELECT, 0.0, 4.0 * E * (2.0 * M + r), side);
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, side), "select_topr");
-        ctx->launched();
+        ctx->launched(side);
       }
       // restoration fill: rows outside the index set, from the upsampled cache of the previous scale
-      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M);
+      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M, side);
       FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, side), "rtr_fill");
-      ctx->launched();
+      ctx->launched(side);
       if (forked) FV_CUDA(ctx, cudaEventRecord(ctx->ev_join, side), "join record");
       const int Mk = static_cast<int>(align_up(M, 64));
       ctx->prof_begin(FVAR_KCLASS_TRANSPOSE, 0.0, 4.0 * E * M * C + 4.0 * E * C * Mk);
@@ -902,7 +918,29 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   return FVAR_OK;
   };
 
-  if (ctx->use_graphs && !ctx->prof_on && !pol->forced_indices) {
+  if (ctx->use_graphs && ctx->prof_on && !pol->forced_indices) {
+    // Profile pass: the same capture, instantiated afresh for this step so that every launch has event nodes of
+    // its own; the executable graph lives until the profile is switched off or read out.
+    const long long l0 = ctx->launches;
+    FV_CUDA(ctx, cudaStreamBeginCapture(ctx->cap_st, cudaStreamCaptureModeThreadLocal), "begin capture");
+    st = ctx->launch_st = ctx->cap_st;
+    s = body();
+    st = ctx->launch_st = ctx->st;
+    cudaGraph_t graph = nullptr;
+    cudaError_t ce = cudaStreamEndCapture(ctx->cap_st, &graph);
+    if (s != FVAR_OK) {
+      if (graph) cudaGraphDestroy(graph);
+      return s;
+    }
+    if (ce != cudaSuccess) return cuda_fail(ctx, ce, "end capture");
+    (void)l0;
+    cudaGraphExec_t exec = nullptr;
+    ce = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ce != cudaSuccess) return cuda_fail(ctx, ce, "graph instantiate");
+    ctx->prof_execs.push_back(exec);
+    FV_CUDA(ctx, cudaGraphLaunch(exec, st), "graph launch");
+  } else if (ctx->use_graphs && !ctx->prof_on && !pol->forced_indices) {
     std::string key;
     auto put = [&](long long v) { key.append(reinterpret_cast<const char *>(&v), sizeof(v)); };
     put(scale_idx); put(B); put(E); put(prev_slot); put(cur_slot); put(ctx->cache_scale);

@@ -411,3 +411,38 @@ def test_step_with_generated_projection(fv):
     got2, ref2 = _step_both(p, toks, k, mode=fv.LOWRANK_RTR, ranks=[r, r])
     assert_out_close(got2, ref2, what="step after replacing the projection")
     assert not np.array_equal(got, got2)
+
+
+def test_profile_pass_times_every_launch_and_changes_nothing(fv):
+    """With per-launch event timing switched on (the step's graph re-captured with event nodes) a step gives
+    the same bits as the timed path, every launch is accounted for in exactly one kernel class, and every
+    interval is positive."""
+    shp = si.shape_var_d16(n_blocks=2)
+    B, k, M, r = 2, 9, 256, 96
+    p = Pair(fv, shp, seed=113, B=B)
+    p.prefill(k)
+    p.set_projections(k, [r, r])
+    toks = to_bf16_cuda(si.make_tokens(113, B, M, 1024, "spread"))
+    p.gpu.restore_loaded()
+    first = p.gpu.scale_step(toks, k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r]).clone()
+    p.gpu.profile_enable(True)
+    n0 = p.gpu.launch_count()
+    for _ in range(2):
+        p.gpu.restore_loaded()
+        again = p.gpu.scale_step(toks, k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r])
+        assert torch.equal(first, again)
+    launched = p.gpu.launch_count() - n0
+    total = 0
+    for i, name in enumerate(fv.KCLASSES):
+        ms, n, fl, by = p.gpu.profile_read(i)
+        total += n
+        if n:
+            assert ms > 0.0, name
+            assert all(t > 0.0 for t in p.gpu.profile_dump(i)), name
+    assert total == launched > 0
+    gemm_ms, gemm_n, gemm_fl, _ = p.gpu.profile_read(fv.KCLASSES.index("gemm"))
+    assert gemm_n == 2 * 2 * 5 and gemm_fl > 0          # per step: 2 groups x (projection + 4 block GEMMs)
+    p.gpu.profile_enable(False)
+    p.gpu.restore_loaded()
+    assert torch.equal(first, p.gpu.scale_step(toks, k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r]))
+    p.check_ok()
