@@ -15,6 +15,8 @@ What the paper fixes and this file follows:
   * random projection  F_r = Q^T F,  Q in R^{M x r}, Q_ij ~ N(0, 1/r)
                                                           (Sec. 3.3 RP; Algorithm 1)
     Q is either given as data or drawn from a seed (Philox4x32-10 + Box-Muller, below)
+  * between two steps: R_k = Q(F_k^o), F_k = F_{k-1} + Up(R_k, (h_K, w_K)), next input Down(F_k, (h_{k+1}, w_{k+1}))
+                                                          (Algorithm 1; Eq. "var_upf", Eq. "var_downf")
   * cached output upsampled, F^{o,cache}_{k-1} = Up(F^o_{k-1})   (Eq. "upcache")
   * restoration F^o_k := {F^o_r rows at I} U {cache rows elsewhere} (Eq. "redefine")
   * CFG = 0 in the fidelity-refinement stage = null-prompt branch only
@@ -217,6 +219,47 @@ def upsample_bilinear(F: np.ndarray, hw_in, hw_out) -> np.ndarray:
             bot = (1.0 - fx) * G[y1, x0] + fx * G[y1, x1]
             out[y, x] = (1.0 - fy) * top + fy * bot
     return out.reshape(h1 * w1, C)
+
+
+# --------------------------------------------------------------------------- between two scale steps
+# Algorithm 1 ("Vanilla VAR" lines, the same in both stages), Eq. "var_upf" and Eq. "var_downf":
+#   R_k = Q(F_k^o);  F_k = F_{k-1} + Up(R_k, (h_K, w_K));  next input = Down(F_k, (h_{k+1}, w_{k+1})).
+# The paper leaves Q, Up and Down abstract (Q "typically includes a codebook Z in R^{V x d}"); here
+# Q is the nearest codeword in Euclidean distance (ties: lowest code), Up is upsample_bilinear above and
+# Down averages the source cells each target cell covers ("area" resampling).
+
+def nearest_codeword(F_o: np.ndarray, Z: np.ndarray, dtype=np.float32) -> np.ndarray:
+    """argmin_v ||F_o[i] - Z[v]||^2 for every row i, as argmax_v (F_o[i] . Z[v] - ||Z[v]||^2 / 2); the
+    score that decides is taken in `dtype` (fp32: the precision the kernel decides in).  int32 [rows]."""
+    F64, Z64 = np.asarray(F_o, dtype=np.float64), np.asarray(Z, dtype=np.float64)
+    score = (F64 @ Z64.T).astype(dtype) - (0.5 * (Z64 * Z64).sum(axis=1)).astype(dtype)[None, :]
+    return np.argmax(score, axis=1).astype(np.int32)          # first maximum = lowest code on ties
+
+
+def downsample_area(F: np.ndarray, hw_in, hw_out) -> np.ndarray:
+    """Down(.) on a row-major (h, w) grid, per channel: target cell (y, x) is the mean of the source cells
+    [floor(y h_in / h_out), ceil((y + 1) h_in / h_out)) x [floor(x w_in / w_out), ceil((x + 1) w_in / w_out)).
+    F is [h_in*w_in][C]; returns [h_out*w_out][C].  Equal sizes give the identity."""
+    (h0, w0), (h1, w1) = hw_in, hw_out
+    G = np.asarray(F, dtype=np.float64).reshape(h0, w0, -1)
+    out = np.empty((h1, w1, G.shape[2]), dtype=np.float64)
+    for y in range(h1):
+        ya, yb = (y * h0) // h1, -((-(y + 1) * h0) // h1)
+        for x in range(w1):
+            xa, xb = (x * w0) // w1, -((-(x + 1) * w0) // w1)
+            out[y, x] = G[ya:yb, xa:xb].mean(axis=(0, 1))
+    return out.reshape(h1 * w1, -1)
+
+
+def scale_transition(F_prev: np.ndarray, F_o: np.ndarray, Z: np.ndarray, hw_k, hw_K, hw_next):
+    """One transition for one batch element.  F_prev [h_K*w_K][C] (F_{k-1}; zeros before the first
+    scale), F_o [h_k*w_k][C] (the step's output), Z [V][C].  Returns (codes int32 [h_k*w_k], F_k
+    [h_K*w_K][C], next tokens [h_next*w_next][C] or None when hw_next is None)."""
+    codes = nearest_codeword(F_o, Z)
+    R = np.asarray(Z, dtype=np.float64)[codes]
+    F_k = np.asarray(F_prev, dtype=np.float64) + upsample_bilinear(R, hw_k, hw_K)
+    nxt = downsample_area(F_k, hw_K, hw_next) if hw_next is not None else None
+    return codes, F_k, nxt
 
 
 def rtr_restore(F_r_out: np.ndarray, idx: np.ndarray, cache_up: np.ndarray) -> np.ndarray:

@@ -551,3 +551,67 @@ def test_generated_projection_layout_and_distribution():
     assert np.array_equal(Q, orc.generate_projection(seed, k, g, M, r))
     assert not np.array_equal(Q, orc.generate_projection(seed, k, g + 1, M, r))
     assert not np.array_equal(Q, orc.generate_projection(seed + 1, k, g, M, r))
+
+
+# ----------------------------------------------------------------------------- between two scale steps
+
+def test_nearest_codeword_is_the_euclidean_argmin():
+    rng = np.random.default_rng(21)
+    Z = rng.standard_normal((37, 16))
+    X = rng.standard_normal((50, 16))
+    got = orc.nearest_codeword(X, Z, dtype=np.float64)
+    want = np.array([min(range(37), key=lambda v: (float(((x - Z[v]) ** 2).sum()), v)) for x in X])
+    assert np.array_equal(got, want)
+    assert np.array_equal(got, torch.cdist(torch.from_numpy(X), torch.from_numpy(Z)).argmin(dim=1).numpy())
+    # a codeword maps to itself; duplicates resolve to the lowest code
+    Z2 = np.concatenate([Z, Z[:5]])
+    assert np.array_equal(orc.nearest_codeword(Z2, Z2, dtype=np.float64)[-5:], np.arange(5))
+    assert np.array_equal(orc.nearest_codeword(Z, Z, dtype=np.float64), np.arange(37))
+
+
+@pytest.mark.parametrize("hw_in,hw_out", [((16, 16), (13, 13)), ((64, 64), (48, 48)), ((6, 10), (4, 3)), ((8, 8), (8, 8)),
+                                          ((16, 16), (1, 1)), ((5, 7), (2, 7))])
+def test_downsample_area_matches_library_and_exact_cases(hw_in, hw_out):
+    rng = np.random.default_rng(22)
+    C = 5
+    Fm = rng.standard_normal((hw_in[0] * hw_in[1], C))
+    got = orc.downsample_area(Fm, hw_in, hw_out)
+    t = torch.from_numpy(Fm.reshape(hw_in[0], hw_in[1], C)).permute(2, 0, 1)[None]
+    ref = F.interpolate(t, size=hw_out, mode="area")[0].permute(1, 2, 0).reshape(-1, C).numpy()
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+    const = orc.downsample_area(np.full_like(Fm, 3.25), hw_in, hw_out)
+    np.testing.assert_allclose(const, 3.25, atol=1e-13)
+    if hw_in == hw_out:
+        assert np.array_equal(got, Fm)
+    if hw_out == (1, 1):
+        np.testing.assert_allclose(got[0], Fm.mean(axis=0), atol=1e-12)
+
+
+def test_scale_transition_telescopes_to_the_sum_of_upsampled_residuals():
+    """Eq. "var_upf": after k transitions F_k = sum_i Up(R_i, (h_K, w_K)); the next input is Down of it
+    (Eq. "var_downf"); at the last scale Up is the identity and there is no next input."""
+    rng = np.random.default_rng(23)
+    C, V = 8, 20
+    sides = [1, 2, 3, 5, 8]
+    Z = rng.standard_normal((V, C))
+    hwK = (sides[-1], sides[-1])
+    Fk = np.zeros((hwK[0] * hwK[1], C))
+    total = np.zeros_like(Fk)
+    for k, sd in enumerate(sides):
+        Fo = rng.standard_normal((sd * sd, C))
+        nxt_hw = (sides[k + 1], sides[k + 1]) if k + 1 < len(sides) else None
+        codes, Fk, nxt = orc.scale_transition(Fk, Fo, Z, (sd, sd), hwK, nxt_hw)
+        assert codes.dtype == np.int32 and codes.shape == (sd * sd,)
+        total += orc.upsample_bilinear(Z[codes], (sd, sd), hwK)
+        np.testing.assert_allclose(Fk, total, atol=1e-12)
+        if nxt_hw is None:
+            assert nxt is None
+            np.testing.assert_allclose(Fk - prev, Z[codes], atol=1e-12)         # Up at equal size is the identity
+        else:
+            np.testing.assert_allclose(nxt, orc.downsample_area(total, hwK, nxt_hw), atol=1e-12)
+        prev = Fk.copy()
+    # an output that is exactly a codeword everywhere adds that codeword everywhere (constant maps stay constant)
+    codes, F1, nxt = orc.scale_transition(np.zeros((64, C)), np.tile(Z[7], (9, 1)), Z, (3, 3), (8, 8), (5, 5))
+    assert (codes == 7).all()
+    np.testing.assert_allclose(F1, np.tile(Z[7], (64, 1)), atol=1e-12)
+    np.testing.assert_allclose(nxt, np.tile(Z[7], (25, 1)), atol=1e-12)
