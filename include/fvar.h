@@ -127,6 +127,28 @@ fvar_status fvar_generate_projection(fvar_ctx *ctx, int scale_idx, int group, in
  * FVAR_ESTATE if none is stored. */
 fvar_status fvar_get_projection(fvar_ctx *ctx, int scale_idx, int group, void *Qt_out, int *r_host);
 
+/* Codebook Z of the quantizer Q (Algorithm 1: "the quantizer Q, which typically includes a codebook
+ * Z in R^{V x d}"): Z dev bf16 [V][C], 16-byte aligned, 1 <= V <= 65536, d = C (the block width).  The
+ * library keeps the pointer (the caller keeps the memory alive) and computes |Z_v|^2 / 2 into its workspace.
+ * FVAR_EUNSUPPORTED for a larger codebook. */
+fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V);
+
+/* The transition between two scale steps (Algorithm 1, the three lines after the blocks in both stages;
+ * Eq. "var_upf", Eq. "var_downf"):
+ *     R_k = Q(F_k^o);   F_k = F_{k-1} + Up(R_k, (h_K, w_K));   next input = Down(F_k, (h_{k+1}, w_{k+1})).
+ * The paper leaves Q, Up and Down abstract; here Q takes the nearest codeword of every token in Euclidean
+ * distance (arg-max of F_k^o Z^T - |Z_v|^2 / 2, decided on fp32 scores, lowest code on ties), Up is the
+ * library's bilinear upsampling (as in the restoration fill) and Down averages the cells of the last
+ * scale's grid that each target cell covers ("area" resampling).  F_0 = 0: scale 0 overwrites the map.
+ * fo dev bf16 [B][M_k][C] (what fvar_scale_step returned for scale_idx, B = its B_eff), 16-byte aligned;
+ * codes dev int32 [B][M_k] or NULL; next_tokens dev bf16 [B][M_{k+1}][C], NULL at the last scale (and
+ * only there).  Scales must come in order from 0 with one B (FVAR_ESTATE otherwise).  Asynchronous on the
+ * context's stream; allocates nothing. */
+fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens);
+
+/* Copies the accumulated map F_k of the last transition, fp32 [B][h_K * w_K][C], to F_out (device). */
+fvar_status fvar_get_feature(fvar_ctx *ctx, float *F_out);
+
 /* One scale step (Algorithm 1: the dense loop body, or the fidelity-refinement loop body RP -> blocks
  * -> RTR).  tokens dev bf16 [B][M][C] with M = h_k * w_k; out dev bf16 [B_eff][M][C], B_eff = B
  * (pair) or B/2 (null-only).  Stages this scale's K/V rows at the cache tail; they become visible

@@ -73,6 +73,9 @@ def load_library() -> ct.CDLL:
         "fvar_set_cond": (i, [vp, i, vp, vp]),
         "fvar_set_projection": (i, [vp, i, i, vp, i]),
         "fvar_generate_projection": (i, [vp, i, i, i, ct.c_ulonglong]),
+        "fvar_set_codebook": (i, [vp, vp, i]),
+        "fvar_scale_transition": (i, [vp, vp, i, i, vp, vp]),
+        "fvar_get_feature": (i, [vp, vp]),
         "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
         "fvar_scale_step": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_scale_step_host": (i, [vp, vp, i, P(_Policy), vp]),
@@ -110,7 +113,7 @@ def load_library() -> ct.CDLL:
 
 
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_generate_projection",
-            "fvar_get_projection", "fvar_scale_step",
+            "fvar_get_projection", "fvar_set_codebook", "fvar_scale_transition", "fvar_get_feature", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
@@ -303,6 +306,27 @@ class Fvar:
         r = ct.c_int(0)
         self._check(self.lib.fvar_get_projection(self.ctx, scale_idx, group, buf.data_ptr(), ct.byref(r)))
         return buf.view(-1)[: r.value * M].view(r.value, M)
+
+    def set_codebook(self, Z: torch.Tensor):
+        """Z bf16 [V][C]: the quantizer's codebook (kept by reference)."""
+        _dev(Z, torch.bfloat16)
+        self._codebook = Z
+        self._check(self.lib.fvar_set_codebook(self.ctx, Z.data_ptr(), Z.shape[0]))
+
+    def scale_transition(self, fo: torch.Tensor, scale_idx: int, next_M: Optional[int]):
+        """fo bf16 [B][M_k][C] -> (codes int32 [B][M_k], next tokens bf16 [B][next_M][C] or None at the last scale)."""
+        _dev(fo, torch.bfloat16)
+        B, M, C = fo.shape
+        codes = torch.empty((B, M), dtype=torch.int32, device=fo.device)
+        nxt = torch.empty((B, next_M, C), dtype=torch.bfloat16, device=fo.device) if next_M else None
+        self._check(self.lib.fvar_scale_transition(self.ctx, fo.data_ptr(), scale_idx, B, codes.data_ptr(), _ptr(nxt)))
+        return codes, nxt
+
+    def get_feature(self, B: int, M_last: int, C: int) -> torch.Tensor:
+        """The accumulated feature map F_k: fp32 [B][M_last][C]."""
+        out = torch.empty((B, M_last, C), dtype=torch.float32, device="cuda")
+        self._check(self.lib.fvar_get_feature(self.ctx, out.data_ptr()))
+        return out
 
     def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise=None):
         pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None, SELECT_TOPR, None)

@@ -82,6 +82,7 @@ static inline int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); 
 static const int kBNs[3] = {64, 128, 256};
 constexpr size_t kSplitScratchBytes = 64u << 20;   // split-K partial tiles
 constexpr size_t kSplitCounters = 4096;            // one arrival counter per tile
+constexpr int kMaxCodebook = 65536;                // largest codebook fvar_set_codebook takes
 
 enum WeightId { W_QKV = 0, W_O, W_FC1, W_FC2, W_ADA, W_CQ, W_CKV, W_CO, W_COUNT };
 
@@ -112,6 +113,15 @@ struct fvar_ctx {
   unsigned *status;
   bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *xt, *qt_pool;
   float *ada, *gcache, *x0, *xs, *scores, *split_partial;
+  // transition between scale steps: codebook (caller's memory), half-norms, packed arg-max words, codes and
+  // the accumulated feature map F_k at the last scale's resolution
+  const bf16 *codebook;
+  int codebook_V;
+  float *tr_hn, *tr_F;
+  unsigned long long *tr_best;
+  int *tr_codes;
+  int tr_scale;                        // last scale accumulated into tr_F (-1: none)
+  int tr_B;
   int *idx, *inv, *split_counters;
   std::vector<size_t> qt_off;          // [scale][group] offset (elements) into qt_pool
   std::vector<int> qt_r;               // [scale][group] rank of the stored projection (0: none)
@@ -195,6 +205,7 @@ namespace {
 
 struct Layout {
   size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
+  size_t tr_hn, tr_best, tr_codes, tr_F;
   std::vector<size_t> qt_off;
 };
 
@@ -258,6 +269,11 @@ Layout make_layout(const fvar_cfg *c) {
     }
   }
   take(pool * 2);
+  const size_t M_last = static_cast<size_t>(c->scale_hw[2 * (c->n_scales - 1)]) * c->scale_hw[2 * (c->n_scales - 1) + 1];
+  L.tr_hn = take(static_cast<size_t>(kMaxCodebook) * 4);
+  L.tr_best = take(B * Mmax * 8);
+  L.tr_codes = take(B * Mmax * 4);
+  L.tr_F = take(B * M_last * C * 4);
   L.total = off;
   return L;
 }
@@ -388,6 +404,9 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->xt = reinterpret_cast<bf16 *>(at(L.xt)); c->scores = reinterpret_cast<float *>(at(L.scores));
   c->idx = reinterpret_cast<int *>(at(L.idx)); c->inv = reinterpret_cast<int *>(at(L.inv));
   c->qt_pool = reinterpret_cast<bf16 *>(at(L.qt_pool));
+  c->tr_hn = reinterpret_cast<float *>(at(L.tr_hn)); c->tr_F = reinterpret_cast<float *>(at(L.tr_F));
+  c->tr_best = reinterpret_cast<unsigned long long *>(at(L.tr_best)); c->tr_codes = reinterpret_cast<int *>(at(L.tr_codes));
+  c->codebook = nullptr; c->codebook_V = 0; c->tr_scale = -1; c->tr_B = 0;
   c->qt_off = L.qt_off;
   c->qt_r.assign(L.qt_off.size(), 0);
   c->qt_map.resize(L.qt_off.size());
@@ -672,6 +691,81 @@ fvar_status fvar_get_projection(fvar_ctx *ctx, int scale_idx, int group, void *Q
   FV_CUDA(ctx, cudaMemcpy2DAsync(Qt_out, static_cast<size_t>(M) * 2, ctx->qt_pool + ctx->qt_off[slot], 2 * Mk * 2,
                                  static_cast<size_t>(M) * 2, r, cudaMemcpyDeviceToDevice, ctx->st), "projection copy");
   *r_host = r;
+  return FVAR_OK;
+}
+
+fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!Z || V <= 0) return fail(ctx, FVAR_EINVAL, "set_codebook: NULL codebook or V <= 0");
+  if (V > kMaxCodebook) return fail(ctx, FVAR_EUNSUPPORTED, "set_codebook: more than 65536 codewords");
+  if (reinterpret_cast<uintptr_t>(Z) & 15) return fail(ctx, FVAR_EINVAL, "set_codebook: codebook must be 16-byte aligned");
+  FV_CUDA(ctx, launch_half_norms(static_cast<const bf16 *>(Z), V, ctx->C, ctx->tr_hn, ctx->st), "half_norms");
+  ctx->launched();
+  ctx->codebook = static_cast<const bf16 *>(Z);
+  ctx->codebook_V = V;
+  ctx->tr_scale = -1;
+  return FVAR_OK;
+}
+
+fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!ctx->codebook) return fail(ctx, FVAR_ESTATE, "scale_transition before set_codebook");
+  const int nS = ctx->cfg.n_scales;
+  if (!fo || scale_idx < 0 || scale_idx >= nS || B <= 0 || B > ctx->Bmax)
+    return fail(ctx, FVAR_EINVAL, "scale_transition: bad arguments");
+  if (scale_idx == nS - 1 ? next_tokens != nullptr : next_tokens == nullptr)
+    return fail(ctx, FVAR_EINVAL, "scale_transition: next_tokens must be given for every scale but the last, where it must be NULL");
+  if (scale_idx > 0 && (ctx->tr_scale != scale_idx - 1 || ctx->tr_B != B))
+    return fail(ctx, FVAR_ESTATE, "scale_transition: scales must be accumulated in order, 0 first, with one batch size");
+  const int C = ctx->C, V = ctx->codebook_V, M = ctx->Mk[scale_idx], R = B * M;
+  const int hk = ctx->hw[2 * scale_idx], wk = ctx->hw[2 * scale_idx + 1];
+  const int hK = ctx->hw[2 * (nS - 1)], wK = ctx->hw[2 * (nS - 1) + 1];
+  cudaStream_t st = ctx->st;
+
+  // R_k = Q(F_k^o): scores F_k^o Z^T - |Z|^2 / 2 on the tensor cores, arg-max in the epilogue
+  const GemmPlan plan = gemm_plan(R, 1, V, C, ctx->num_sms, ctx->max_clusters, 1, 0);
+  CUtensorMap ta, tw;
+  if (!tmap_2d(&ta, fo, C, R, C, 128) || !tmap_2d(&tw, ctx->codebook, C, V, C, plan.pair ? plan.block_n / 2 : plan.block_n))
+    return fail(ctx, FVAR_EINVAL, "scale_transition: fo must be 16-byte aligned");
+  FV_CUDA(ctx, cudaMemsetAsync(ctx->tr_best, 0, static_cast<size_t>(R) * 8, st), "arg-max words clear");
+  GemmArgs g = gemm_args(R, V, C);
+  g.col_sub = ctx->tr_hn;
+  g.best = ctx->tr_best;
+  g.status = ctx->status;
+  ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * R * V * C, 2.0 * (static_cast<double>(V) * C + static_cast<double>(R) * C) + 8.0 * R);
+  if (plan.pair)
+    FV_CUDA(ctx, launch_gemm_pair(EPI_ARGMAX, plan.block_n, ta, tw, g, st), "codeword search");
+  else
+    FV_CUDA(ctx, launch_gemm(EPI_ARGMAX, plan.block_n, ta, tw, g, ctx->num_sms, st), "codeword search");
+  ctx->launched();
+  ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 12.0 * R);
+  FV_CUDA(ctx, launch_unpack_codes(ctx->tr_best, R, V, ctx->tr_codes, ctx->status, st), "unpack codes");
+  ctx->launched();
+  if (codes) FV_CUDA(ctx, cudaMemcpyAsync(codes, ctx->tr_codes, static_cast<size_t>(R) * 4, cudaMemcpyDeviceToDevice, st), "codes copy");
+
+  // F_k = F_{k-1} + Up(R_k, (h_K, w_K))
+  ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, (scale_idx == 0 ? 4.0 : 8.0) * B * hK * wK * C + 2.0 * R * C);
+  FV_CUDA(ctx, launch_up_accumulate(ctx->codebook, ctx->tr_codes, B, hk, wk, hK, wK, C, scale_idx == 0, ctx->tr_F, st), "up_accumulate");
+  ctx->launched();
+  // next input = Down(F_k, (h_{k+1}, w_{k+1}))
+  if (next_tokens) {
+    const int hn = ctx->hw[2 * (scale_idx + 1)], wn = ctx->hw[2 * (scale_idx + 1) + 1];
+    ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * B * hK * wK * C + 2.0 * B * hn * wn * C);
+    FV_CUDA(ctx, launch_down_area(ctx->tr_F, B, hK, wK, hn, wn, C, static_cast<bf16 *>(next_tokens), st), "down_area");
+    ctx->launched();
+  }
+  ctx->tr_scale = scale_idx;
+  ctx->tr_B = B;
+  return FVAR_OK;
+}
+
+fvar_status fvar_get_feature(fvar_ctx *ctx, float *F_out) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!F_out) return fail(ctx, FVAR_EINVAL, "get_feature: NULL output");
+  if (ctx->tr_scale < 0) return fail(ctx, FVAR_ESTATE, "get_feature: no scale accumulated yet");
+  const int nS = ctx->cfg.n_scales;
+  const size_t n = static_cast<size_t>(ctx->tr_B) * ctx->hw[2 * (nS - 1)] * ctx->hw[2 * (nS - 1) + 1] * ctx->C;
+  FV_CUDA(ctx, cudaMemcpyAsync(F_out, ctx->tr_F, n * 4, cudaMemcpyDeviceToDevice, ctx->st), "feature copy");
   return FVAR_OK;
 }
 

@@ -442,6 +442,7 @@ static cudaError_t set_attr_bn() {
   if (e == cudaSuccess) e = set_attr<BN, EPI_GELU_BF16>();
   if (e == cudaSuccess) e = set_attr<BN, EPI_QKV>();
   if (e == cudaSuccess) e = set_attr<BN, EPI_RESID>();
+  if (e == cudaSuccess) e = set_attr<BN, EPI_ARGMAX>();
   return e;
 }
 
@@ -474,6 +475,7 @@ static cudaError_t launch_bn(int epi, const CUtensorMap &tmA, const CUtensorMap 
     case EPI_GELU_BF16: return launch_one<BN, EPI_GELU_BF16>(tmA, tmW, a, num_sms, st);
     case EPI_QKV: return launch_one<BN, EPI_QKV>(tmA, tmW, a, num_sms, st);
     case EPI_RESID: return launch_one<BN, EPI_RESID>(tmA, tmW, a, num_sms, st);
+    case EPI_ARGMAX: return launch_one<BN, EPI_ARGMAX>(tmA, tmW, a, num_sms, st);
   }
   return cudaErrorInvalidValue;
 }

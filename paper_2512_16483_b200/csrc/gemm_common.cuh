@@ -1,6 +1,7 @@
 // Epilogue code shared by the tensor-core GEMM kernels: bias, tanh-GELU, gate + residual, the
 // QKV / KV-cache split and warp-wide row-segment stores through a shared-memory staging tile.
 #pragma once
+#include <math.h>
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -120,6 +121,28 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t
       for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_f(v[i]);
     }
     warp_store_bf16(stage, lane, v, valid ? p.out_bf16 + grow * p.ld_out + col0 : nullptr);
+  } else if constexpr (EPI == EPI_ARGMAX) {
+    if (valid) {
+      float best_v = -INFINITY;
+      int best_c = -1;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int c = col0 + i;
+        if (c < p.N) {
+          float sc = v[i] - __ldg(p.col_sub + c);
+          if (sc != sc) sc = -INFINITY;         // NaN never wins
+          if (sc > best_v || best_c < 0) {      // strict: the lowest column wins a tie
+            best_v = sc;
+            best_c = c;
+          }
+        }
+      }
+      if (best_c >= 0) {
+        const unsigned u = __float_as_uint(best_v);
+        const unsigned key = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // unsigned order = float order
+        atomicMax(p.best + grow, (static_cast<unsigned long long>(key) << 32) | (0xFFFFFFFFu - static_cast<unsigned>(best_c)));
+      }
+    }
   } else if constexpr (EPI == EPI_QKV) {
     const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
     const int b = e * p.bmul + p.boff;

@@ -277,6 +277,7 @@ static cudaError_t pair_prepare_bn() {
   if (e == cudaSuccess) e = pair_prepare_one<BN, EPI_GELU_BF16>();
   if (e == cudaSuccess) e = pair_prepare_one<BN, EPI_QKV>();
   if (e == cudaSuccess) e = pair_prepare_one<BN, EPI_RESID>();
+  if (e == cudaSuccess) e = pair_prepare_one<BN, EPI_ARGMAX>();
   return e;
 }
 
@@ -327,6 +328,7 @@ static cudaError_t pair_launch_bn(int epi, const CUtensorMap &tmA, const CUtenso
     case EPI_GELU_BF16: return pair_launch_one<BN, EPI_GELU_BF16>(tmA, tmW, a, st);
     case EPI_QKV: return pair_launch_one<BN, EPI_QKV>(tmA, tmW, a, st);
     case EPI_RESID: return pair_launch_one<BN, EPI_RESID>(tmA, tmW, a, st);
+    case EPI_ARGMAX: return pair_launch_one<BN, EPI_ARGMAX>(tmA, tmW, a, st);
   }
   return cudaErrorInvalidValue;
 }

@@ -16,7 +16,7 @@ struct RowMap {
   int bmul, boff, rpb;
 };
 
-enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU_BF16 = 2, EPI_QKV = 3, EPI_RESID = 4 };
+enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU_BF16 = 2, EPI_QKV = 3, EPI_RESID = 4, EPI_ARGMAX = 5 };
 
 struct GemmArgs {
   int R, N, K;            // out[R][N] = A[R][K] * W[N][K]^T, per batch
@@ -40,6 +40,11 @@ struct GemmArgs {
   // EPI_QKV: virtual column = col + col_base; [0,C) -> q, [C,2C) -> K cache, [2C,3C) -> transposed V cache
   bf16 *kc, *vt;
   int C, H, D, L_cap, L_prev, col_base;
+  // EPI_ARGMAX: per row, the column with the largest (acc - col_sub[col]), lowest column on ties, kept as one
+  // 64-bit word per row: ordered score bits << 32 | ~column (so that an unsigned max picks it); best must be
+  // zero before the launch
+  const float *col_sub;
+  unsigned long long *best;
   // split-K (splits > 1): fp32 partial tiles [tile][split][128][BN] and one arrival counter per tile
   int splits;
   float *partial;
@@ -136,6 +141,13 @@ cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);
 cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned long long seed, int group, int scale,
                                        cudaStream_t st);
+// Between two scale steps: codeword half-norms, the packed argmax words, Up-accumulate and area Down.
+cudaError_t launch_half_norms(const bf16 *Z, int V, int C, float *hn, cudaStream_t st);
+cudaError_t launch_unpack_codes(const unsigned long long *best, long long n, int V, int *codes, unsigned *status,
+                                cudaStream_t st);
+cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0, int w0, int h1, int w1, int C,
+                                 bool overwrite, float *F, cudaStream_t st);
+cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st);
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
 cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,
                            cudaStream_t st);

@@ -181,3 +181,17 @@ def make_sample_noise(seed: int, scale_idx: int, G: int, B_eff: int, M: int) -> 
     """Exp(1) variates [G][B_eff][M] (fp32) for the sampled row selection; one draw per (scale, group, element, row)."""
     rng = np.random.default_rng([seed, 8, scale_idx])
     return rng.standard_exponential(size=(G, B_eff, M)).astype(np.float32) + np.float32(1e-30)
+
+
+def make_codebook(seed: int, V: int, C: int) -> np.ndarray:
+    """Quantizer codebook Z [V][C], entries N(0, 1), bf16-rounded (stands in for a trained codebook)."""
+    return normal_bf16(np.random.default_rng([seed, 9]), (V, C))
+
+
+def make_step_outputs(seed: int, scale_idx: int, B: int, M: int, Z: np.ndarray, noise: float) -> np.ndarray:
+    """Stand-in block outputs F_k^o [B][M][C] for the transition between steps: a randomly chosen codeword per
+    token plus N(0, noise^2), bf16-rounded.  Small noise keeps every token's nearest codeword well separated;
+    noise >= 1 gives generic rows with near ties."""
+    rng = np.random.default_rng([seed, 10, scale_idx])
+    pick = rng.integers(0, Z.shape[0], size=(B, M))
+    return round_to_bf16(Z[pick] + noise * rng.standard_normal((B, M, Z.shape[1]), dtype=np.float32))
