@@ -262,6 +262,14 @@ def scale_transition(F_prev: np.ndarray, F_o: np.ndarray, Z: np.ndarray, hw_k, h
     return codes, F_k, nxt
 
 
+def cfg_combine(F_prompt: np.ndarray, F_null: np.ndarray, s: float) -> np.ndarray:
+    """Classifier-free guidance on the two branches of a CFG pair: F_null + s (F_prompt - F_null).  s = 0 is
+    the null-prompt branch alone, which is what "setting the CFG to 0" in the fidelity-refinement stage means
+    (Sec. 3.3: "equivalent to conditioning only on the null text prompt")."""
+    a, b = np.asarray(F_prompt, dtype=np.float64), np.asarray(F_null, dtype=np.float64)
+    return b + s * (a - b)
+
+
 def rtr_restore(F_r_out: np.ndarray, idx: np.ndarray, cache_up: np.ndarray) -> np.ndarray:
     """Eq. "redefine": row idx[j] takes row j of the block output, every other row
     takes the upsampled cached row."""

@@ -615,3 +615,12 @@ def test_scale_transition_telescopes_to_the_sum_of_upsampled_residuals():
     assert (codes == 7).all()
     np.testing.assert_allclose(F1, np.tile(Z[7], (64, 1)), atol=1e-12)
     np.testing.assert_allclose(nxt, np.tile(Z[7], (25, 1)), atol=1e-12)
+
+
+def test_cfg_combine_end_points_and_linearity():
+    rng = np.random.default_rng(24)
+    a, b = rng.standard_normal((7, 5)), rng.standard_normal((7, 5))
+    assert np.array_equal(orc.cfg_combine(a, b, 0.0), b)                 # CFG = 0: the null-prompt branch alone
+    np.testing.assert_allclose(orc.cfg_combine(a, b, 1.0), a, atol=1e-15)
+    np.testing.assert_allclose(orc.cfg_combine(a, b, 3.0), 3.0 * a - 2.0 * b, atol=1e-14)
+    np.testing.assert_allclose(orc.cfg_combine(a, a, 7.5), a, atol=1e-14)  # equal branches: guidance changes nothing
