@@ -50,7 +50,15 @@ WORKLOADS = {
     "infinity2b_gen13_vanilla_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=13, keep=1.0, null_only=False),
     "infinity2b_gen13_fastervar_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=10, keep="paper", null_only=True),
     "infinity2b_gen13_fastervar_late3_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=10, keep="table", null_only=True),
+    # The same two generations as a closed autoregressive loop: every step's tokens come from the previous step
+    # through the library's transition (CFG combination of the two branches, nearest codeword of a seeded random
+    # codebook of 8192 entries, Up-accumulate at 64 x 64, area Down), starting from one seeded start token.  With the
+    # schedule of Sec. 4.1 the loop ends after scale 40: the accumulated map is already at the final resolution.
+    "infinity2b_loop13_vanilla_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=13, keep=1.0, null_only=False, loop=True),
+    "infinity2b_loop13_fastervar_b2": dict(shape="inf2b", B=2, first_late=0, dense_until=10, keep="paper", null_only=True, loop=True),
 }
+LOOP_CODEBOOK = 8192
+LOOP_GUIDANCE = 3.0
 
 
 def resolve_workload(name):
@@ -350,6 +358,31 @@ def main():
     outs_host = {k: torch.empty((E_at[k], Ms[k], shp.width), dtype=torch.bfloat16).pin_memory() for k in late_scales}
     tokens_per_step = sum(E_at[k] * Ms[k] for k in late_scales)     # a skipped scale still delivers its positions
     rewind = ctx.reset if k0 == 0 else ctx.restore_loaded
+    loop = bool(wl.get("loop"))
+    if loop:
+        codebook = randn_bf16((LOOP_CODEBOOK, shp.width))
+        ctx.set_codebook(codebook)
+        tokens_per_step = (B // 2) * sum(Ms)                        # one image per CFG pair, every scale's positions
+        start_host = toks[0].cpu().pin_memory()
+        feat_host = torch.empty((B // 2, Ms[-1], shp.width), dtype=torch.float32).pin_memory()
+
+    def step_loop(host=False):
+        """Closed loop: step -> (CFG combination) -> transition -> the next step's tokens, for both branches."""
+        rewind()
+        tok = start_host.cuda(non_blocking=True) if host else toks[0]
+        run = [k for k in late_scales if modes[k][0] != fv.SKIP]
+        for i, k in enumerate(run):
+            mode, ranks = modes[k]
+            out = ctx.scale_step(tok, k, mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks, out=outs[k])
+            ctx.kv_append(k)
+            fo = out if null_at[k] else fv.fvar_cfg_combine(out, LOOP_GUIDANCE)
+            more = i + 1 < len(run)
+            _, nxt = ctx.scale_transition(fo, k, Ms[k + 1] if more else None)
+            if more:
+                tok = nxt.repeat_interleave(2, dim=0)               # both branches of a pair see the same tokens
+        if host:
+            feat_host.copy_(ctx.get_feature(B // 2, Ms[-1], shp.width), non_blocking=True)
+            torch.cuda.synchronize()
 
     def step_device():
         rewind()
@@ -390,9 +423,10 @@ def main():
 
     warm = max(args.warmup, 3)
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    ms_total, launches = timed(step_device, args.steps, warm)
+    dev_fn, host_fn = (step_loop, lambda: step_loop(True)) if loop else (step_device, step_host)
+    ms_total, launches = timed(dev_fn, args.steps, warm)
     clocks = sampler.stop() if sampler else None
-    ms_e2e, _ = (ms_total, 0) if args.profile_run else timed(step_host, args.steps, 2)
+    ms_e2e, _ = (ms_total, 0) if args.profile_run else timed(host_fn, args.steps, 2)
     assert ctx.poll_status() == fv.OK, "device status word reports an error"
 
     # per-kernel-class event timing: a separate pass over the same steps; the library re-captures the step's graph
@@ -403,7 +437,7 @@ def main():
         # Hold the stream back (a device-side delay of about 10 ms) while the host captures and enqueues the
         # step, so that no interval between two events contains host time.
         torch.cuda._sleep(20_000_000)
-        step_device()
+        dev_fn()
     classes = {}
     for i, name in enumerate(fv.KCLASSES):
         ms, n, fl, by = ctx.profile_read(i)
@@ -435,8 +469,10 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e, "unit": "tokens/s",
-                "h2d_bytes_per_step": sum(B * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP),
-                "d2h_bytes_per_step": sum(E_at[k] * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP)},
+                "h2d_bytes_per_step": B * Ms[0] * shp.width * 2 if loop else
+                sum(B * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP),
+                "d2h_bytes_per_step": (B // 2) * Ms[-1] * shp.width * 4 if loop else
+                sum(E_at[k] * Ms[k] * shp.width * 2 for k in late_scales if modes[k][0] != fv.SKIP)},
         "roofline": roofline,
     }
     if world == 1 and not args.no_cpu_baseline and not args.profile_run and "dense_until" not in wl:

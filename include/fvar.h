@@ -141,10 +141,19 @@ fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V);
  * library's bilinear upsampling (as in the restoration fill) and Down averages the cells of the last
  * scale's grid that each target cell covers ("area" resampling).  F_0 = 0: scale 0 overwrites the map.
  * fo dev bf16 [B][M_k][C] (what fvar_scale_step returned for scale_idx, B = its B_eff), 16-byte aligned;
- * codes dev int32 [B][M_k] or NULL; next_tokens dev bf16 [B][M_{k+1}][C], NULL at the last scale (and
- * only there).  Scales must come in order from 0 with one B (FVAR_ESTATE otherwise).  Asynchronous on the
+ * codes dev int32 [B][M_k] or NULL; next_tokens dev bf16 [B][M_{k+1}][C], or NULL when no further step follows
+ * (always at the last scale; also when the remaining steps are skipped, Sec. 4.1: F_k, already at the final
+ * resolution, is then the output).  Scales must come in order from 0 with one B (FVAR_ESTATE otherwise).  Asynchronous on the
  * context's stream; allocates nothing. */
 fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens);
+
+/* Classifier-free guidance on the outputs of a step that ran both branches: out[p] = null + guidance *
+ * (prompt - null) for the CFG pair p = elements (2p, 2p + 1) = (prompt, null prompt) of `pair`.  The paper
+ * only says that VAR "adopts classifier-free guidance to combine text prompts with null text prompts" and
+ * that setting it to 0 leaves the null-prompt branch alone (Sec. 3.2, Sec. 3.3); applying it to the block
+ * outputs is this library's reading.  pair dev bf16 [B][per_elem], B even, per_elem % 8 == 0; out dev bf16
+ * [B / 2][per_elem]; both 16-byte aligned. */
+fvar_status fvar_cfg_combine(const void *pair, int B, long long per_elem, float guidance, void *out, void *stream);
 
 /* Copies the accumulated map F_k of the last transition, fp32 [B][h_K * w_K][C], to F_out (device). */
 fvar_status fvar_get_feature(fvar_ctx *ctx, float *F_out);

@@ -76,6 +76,7 @@ def load_library() -> ct.CDLL:
         "fvar_set_codebook": (i, [vp, vp, i]),
         "fvar_scale_transition": (i, [vp, vp, i, i, vp, vp]),
         "fvar_get_feature": (i, [vp, vp]),
+        "fvar_cfg_combine": (i, [vp, i, ll, f, vp, vp]),
         "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
         "fvar_scale_step": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_scale_step_host": (i, [vp, vp, i, P(_Policy), vp]),
@@ -118,7 +119,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
+            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
 
 def _stream() -> int:
@@ -192,6 +193,16 @@ def fvar_gemm_bf16_form(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.T
     out = torch.empty((R, N), dtype=torch.float32, device=A.device)
     _check_kernel(load_library().fvar_gemm_bf16_form(A.data_ptr(), W.data_ptr(), _ptr(bias), R, N, K, form, block_n,
                                                      out.data_ptr(), _stream()))
+    return out
+
+
+def fvar_cfg_combine(pair: torch.Tensor, guidance: float) -> torch.Tensor:
+    """pair bf16 [B][...] with elements (2p, 2p + 1) = (prompt, null) -> bf16 [B / 2][...] = null + guidance (prompt - null)."""
+    _dev(pair, torch.bfloat16)
+    B = pair.shape[0]
+    per = pair[0].numel()
+    out = torch.empty((B // 2,) + tuple(pair.shape[1:]), dtype=torch.bfloat16, device=pair.device)
+    _check_kernel(load_library().fvar_cfg_combine(pair.data_ptr(), B, per, float(guidance), out.data_ptr(), _stream()))
     return out
 
 

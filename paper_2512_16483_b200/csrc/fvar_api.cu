@@ -713,8 +713,8 @@ fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, 
   const int nS = ctx->cfg.n_scales;
   if (!fo || scale_idx < 0 || scale_idx >= nS || B <= 0 || B > ctx->Bmax)
     return fail(ctx, FVAR_EINVAL, "scale_transition: bad arguments");
-  if (scale_idx == nS - 1 ? next_tokens != nullptr : next_tokens == nullptr)
-    return fail(ctx, FVAR_EINVAL, "scale_transition: next_tokens must be given for every scale but the last, where it must be NULL");
+  if (scale_idx == nS - 1 && next_tokens != nullptr)
+    return fail(ctx, FVAR_EINVAL, "scale_transition: there is no next input after the last scale (next_tokens must be NULL)");
   if (scale_idx > 0 && (ctx->tr_scale != scale_idx - 1 || ctx->tr_B != B))
     return fail(ctx, FVAR_ESTATE, "scale_transition: scales must be accumulated in order, 0 first, with one batch size");
   const int C = ctx->C, V = ctx->codebook_V, M = ctx->Mk[scale_idx], R = B * M;
@@ -1240,6 +1240,15 @@ fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B,
              kernel_status_ptr(), 1, nullptr, nullptr};
   if (!a.status) return kfail(FVAR_ECUDA, "attention: status word");
   FK_CUDA(launch_attention(tq, tk, tv, a, static_cast<cudaStream_t>(stream)), "attention");
+  return FVAR_OK;
+}
+
+fvar_status fvar_cfg_combine(const void *pair, int B, long long per_elem, float guidance, void *out, void *stream) {
+  if (!pair || !out || B <= 0 || (B & 1) || per_elem <= 0 || per_elem % 8 || (reinterpret_cast<uintptr_t>(pair) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 15))
+    return kfail(FVAR_EINVAL, "cfg_combine: bad arguments");
+  FK_CUDA(launch_cfg_combine(static_cast<const bf16 *>(pair), B / 2, per_elem, guidance, static_cast<bf16 *>(out),
+                             static_cast<cudaStream_t>(stream)), "cfg_combine");
   return FVAR_OK;
 }
 

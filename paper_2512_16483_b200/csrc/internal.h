@@ -147,6 +147,7 @@ cudaError_t launch_unpack_codes(const unsigned long long *best, long long n, int
                                 cudaStream_t st);
 cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0, int w0, int h1, int w1, int C,
                                  bool overwrite, float *F, cudaStream_t st);
+cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st);
 cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st);
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
 cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,

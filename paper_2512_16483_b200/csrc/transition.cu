@@ -155,4 +155,34 @@ cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int 
                     tokens);
 }
 
+// Classifier-free guidance on CFG pairs: out[p] = null + s (prompt - null) with (prompt, null) = elements
+// (2p, 2p + 1); fp32 arithmetic on bf16 inputs, one rounding.  Eight elements per thread.
+__global__ void __launch_bounds__(256) cfg_combine_kernel(const bf16 *__restrict__ pair, long long n8_per_elem, long long total8,
+                                                          float s, bf16 *__restrict__ out) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= total8) return;
+  const long long pidx = i / n8_per_elem, off = i - pidx * n8_per_elem;
+  const uint4 ua = __ldg(reinterpret_cast<const uint4 *>(pair) + (2 * pidx) * n8_per_elem + off);
+  const uint4 ub = __ldg(reinterpret_cast<const uint4 *>(pair) + (2 * pidx + 1) * n8_per_elem + off);
+  const __nv_bfloat162 *ha = reinterpret_cast<const __nv_bfloat162 *>(&ua), *hb = reinterpret_cast<const __nv_bfloat162 *>(&ub);
+  uint32_t w[4];
+#pragma unroll
+  for (int t = 0; t < 4; ++t) {
+    const float2 a = __bfloat1622float2(ha[t]), b = __bfloat1622float2(hb[t]);
+    const __nv_bfloat162 o = __floats2bfloat162_rn(fmaf(s, a.x - b.x, b.x), fmaf(s, a.y - b.y, b.y));
+    w[t] = *reinterpret_cast<const uint32_t *>(&o);
+  }
+  reinterpret_cast<uint4 *>(out)[i] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st) {
+  if (per_elem % 8 != 0) return cudaErrorInvalidValue;
+  const long long total8 = static_cast<long long>(pairs) * (per_elem / 8);
+  if (total8 <= 0) return cudaSuccess;
+  return launch_pdl(cfg_combine_kernel, dim3(static_cast<unsigned>((total8 + 255) / 256)), dim3(256), 0, st, pair, per_elem / 8,
+                    total8, s, out);
+}
+
 }  // namespace fvar

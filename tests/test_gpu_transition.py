@@ -105,10 +105,23 @@ def test_transition_state_and_argument_errors(fv):
     fo1 = to_bf16_cuda(si.make_step_outputs(306, 1, 2, Ms[1], Z, 0.05))
     with pytest.raises(fv.FvarError):
         g.scale_transition(fo1, 1, Ms[2])                        # scale 1 before scale 0
-    with pytest.raises(fv.FvarError):
-        g.scale_transition(fo0, 0, None)                         # next tokens missing before the last scale
-    g.scale_transition(fo0, 0, Ms[1])
+    codes_a, none = g.scale_transition(fo0, 0, None)             # allowed: the caller stops here (remaining steps skipped)
+    assert none is None
+    codes_b, _ = g.scale_transition(fo0, 0, Ms[1])               # scale 0 starts a new accumulation
+    assert torch.equal(codes_a, codes_b)
     g.scale_transition(fo1, 1, Ms[2])
     with pytest.raises(fv.FvarError):
         g.scale_transition(fo1[:1].contiguous(), 2, Ms[3] if len(shp.hw()) > 3 else None)   # batch changed midway
     assert g.poll_status() == fv.OK
+
+
+@pytest.mark.parametrize("guidance", [0.0, 1.0, 3.0])
+def test_cfg_combine(fv, guidance):
+    rng = np.random.default_rng(31)
+    x = si.normal_bf16(rng, (6, 100, 128))
+    got = bf16_to_numpy(fv.fvar_cfg_combine(to_bf16_cuda(x), guidance))
+    ref = np.stack([orc.cfg_combine(x[2 * p], x[2 * p + 1], guidance) for p in range(3)])
+    # fp32 arithmetic on bf16 inputs, one rounding to bf16
+    np.testing.assert_allclose(got, ref, rtol=2 ** -8, atol=1e-6)
+    if guidance == 0.0:
+        assert np.array_equal(got, x[1::2])                      # CFG = 0: the null-prompt branch, bit for bit
