@@ -116,40 +116,57 @@ cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0,
 
 // tokens[b][q][:] = mean of F over the source cells target cell q = (y, x) of the (h1, w1) grid covers:
 // rows [floor(y h0 / h1), ceil((y + 1) h0 / h1)), columns likewise ("area" resampling); bf16 out.
-// One warp per (target cell, 128-channel slab): lanes over channels, the window walked row by row.
+// One warp per target cell: the lanes walk the channels four float4 groups at a time (so that several
+// loads per lane are in flight), the window cell by cell inside.  C % 4 == 0.
 __global__ void __launch_bounds__(256) down_area_kernel(const float *__restrict__ F, int B, int h0, int w0, int h1, int w1,
                                                         int C, bf16 *__restrict__ tokens) {
   pdl_wait();
   pdl_launch_dependents();
-  const int slabs = (C + 127) / 128, M1 = h1 * w1;
-  const long long gw = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
-  if (gw >= static_cast<long long>(B) * M1 * slabs) return;
-  const int slab = static_cast<int>(gw % slabs);
-  const long long cell = gw / slabs;
+  const int M1 = h1 * w1, lane = threadIdx.x & 31;
+  const long long cell = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (cell >= static_cast<long long>(B) * M1) return;
   const int b = static_cast<int>(cell / M1), q = static_cast<int>(cell - static_cast<long long>(b) * M1);
   const int y = q / w1, x = q - y * w1;
   const int ya = (y * h0) / h1, yb = ((y + 1) * h0 + h1 - 1) / h1;
   const int xa = (x * w0) / w1, xb = ((x + 1) * w0 + w1 - 1) / w1;
-  const int c = slab * 128 + 4 * (threadIdx.x & 31);
-  if (c >= C) return;
-  const float *src = F + static_cast<long long>(b) * h0 * w0 * C + c;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int yy = ya; yy < yb; ++yy)
-    for (int xx = xa; xx < xb; ++xx) {
-      const float4 v = __ldg(reinterpret_cast<const float4 *>(src + (static_cast<long long>(yy) * w0 + xx) * C));
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    }
   const float inv = 1.0f / static_cast<float>((yb - ya) * (xb - xa));
-  const __nv_bfloat162 o0 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), o1 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-  uint2 pk;
-  pk.x = *reinterpret_cast<const uint32_t *>(&o0);
-  pk.y = *reinterpret_cast<const uint32_t *>(&o1);
-  *reinterpret_cast<uint2 *>(tokens + (static_cast<long long>(b) * M1 + q) * C + c) = pk;
+  const float4 *src = reinterpret_cast<const float4 *>(F + static_cast<long long>(b) * h0 * w0 * C);
+  uint2 *dst = reinterpret_cast<uint2 *>(tokens + (static_cast<long long>(b) * M1 + q) * C);
+  const int ngroups = C / 4, row4 = C / 4;
+  for (int g0 = lane; g0 < ngroups; g0 += 128) {
+    float4 acc[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int yy = ya; yy < yb; ++yy)
+      for (int xx = xa; xx < xb; ++xx) {
+        const float4 *cellp = src + (static_cast<long long>(yy) * w0 + xx) * row4;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int g = g0 + 32 * u;
+          if (g < ngroups) {
+            const float4 v = __ldg(cellp + g);
+            acc[u].x += v.x; acc[u].y += v.y; acc[u].z += v.z; acc[u].w += v.w;
+          }
+        }
+      }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int g = g0 + 32 * u;
+      if (g < ngroups) {
+        const __nv_bfloat162 o0 = __floats2bfloat162_rn(acc[u].x * inv, acc[u].y * inv);
+        const __nv_bfloat162 o1 = __floats2bfloat162_rn(acc[u].z * inv, acc[u].w * inv);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t *>(&o0);
+        pk.y = *reinterpret_cast<const uint32_t *>(&o1);
+        dst[g] = pk;
+      }
+    }
+  }
 }
 
 cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st) {
   if (C % 4 != 0) return cudaErrorInvalidValue;
-  const long long warps = static_cast<long long>(B) * h1 * w1 * ((C + 127) / 128);
+  const long long warps = static_cast<long long>(B) * h1 * w1;
   if (warps <= 0) return cudaSuccess;
   return launch_pdl(down_area_kernel, dim3(static_cast<unsigned>((warps + 7) / 8)), dim3(256), 0, st, F, B, h0, w0, h1, w1, C,
                     tokens);

@@ -4,6 +4,7 @@
     python -m paper_2512_16483_b200.microbench gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
     python -m paper_2512_16483_b200.microbench attention
     python -m paper_2512_16483_b200.microbench memory      # score, LayerNorm + modulate, restoration fill, selection
+    python -m paper_2512_16483_b200.microbench transition  # between two scale steps: codeword search, Up-accumulate, Down
 
 GEMM calls rotate over several weight copies (more than L2 holds) and are captured in one CUDA graph so
 that host launch cost does not enter the time.
@@ -115,6 +116,38 @@ def memory():
         print("select_topr  B=%d M=%d r=%d: %.1f us (includes ~10 us of host call overhead)" % (B, M, M // 4, us))
 
 
+def transition():
+    """Transitions of an Infinity-2B-shaped schedule tail (32 x 32, 48 x 48, 64 x 64 tokens; accumulation at
+    64 x 64; C = 2048, 8192 codewords) for 8 elements, timed per kernel by the library's profile pass."""
+    C, V, B = 2048, 8192, 8
+    hw = [(32, 32), (48, 48), (64, 64)]
+    Ms = [h * w_ for h, w_ in hw]
+    dims = {"w_qkv": (3 * C, C), "b_qkv": (3 * C,), "w_o": (C, C), "b_o": (C,), "w_fc1": (4 * C, C), "b_fc1": (4 * C,),
+            "w_fc2": (C, 4 * C), "b_fc2": (C,), "w_ada": (6 * C, C), "b_ada": (6 * C,)}
+    w = [{n: torch.zeros(shape, dtype=torch.bfloat16, device="cuda") for n, shape in dims.items()}]
+    ctx = fv.Fvar(w, blocks_per_group=1, n_heads=16, head_dim=128, ffn_dim=4 * C, scale_hw=hw, max_batch=B)
+    ctx.set_codebook(torch.randn(V, C, device="cuda").bfloat16())
+    fo = [torch.randn(B, m, C, device="cuda").bfloat16() for m in Ms]
+
+    def chain():
+        ctx.scale_transition(fo[0], 0, Ms[1])
+        ctx.scale_transition(fo[1], 1, Ms[2])
+    chain()
+    ctx.profile_enable(True)
+    for _ in range(5):
+        chain()
+    gemm_t = ctx.profile_dump(fv.KCLASSES.index("gemm"))          # per pass: search of scale 0, of scale 1
+    up_t = ctx.profile_dump(fv.KCLASSES.index("rtr_fill"))        # per pass: Up of scale 0 (write), of scale 1 (accumulate)
+    cv_t = ctx.profile_dump(fv.KCLASSES.index("convert"))         # per pass: unpack, Down 64->48, unpack, Down 64->64
+    t_g, t_u, t_d = 1e3 * min(gemm_t[1::2]), 1e3 * min(up_t[1::2]), 1e3 * min(cv_t[1::4])
+    print("codeword search  R=%d V=%d K=%d: %.1f us  %.0f TFLOP/s" % (B * Ms[1], V, C, t_g, 2.0 * B * Ms[1] * V * C / t_g / 1e6))
+    print("up_accumulate    B=%d 48x48 -> 64x64 C=%d: %.1f us  %.0f GB/s (fp32 map read and written once)" % (
+        B, C, t_u, 8.0 * B * Ms[2] * C / t_u / 1e3))
+    print("down_area        B=%d 64x64 -> 48x48 C=%d: %.1f us  %.0f GB/s (map read once, bf16 tokens written once)" % (
+        B, C, t_d, (4.0 * B * Ms[2] * C + 2.0 * B * Ms[1] * C) / t_d / 1e3))
+    ctx.profile_enable(False)
+
+
 if __name__ == "__main__":
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
-    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory}[which]()
+    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition}[which]()
