@@ -399,8 +399,9 @@ def main():
             mode, ranks = modes[k]
             if mode == fv.SKIP:
                 continue
-            ctx.scale_step_host(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks)
+            ctx.scale_step_host_async(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks)
             ctx.kv_append(k)
+        ctx.host_sync()                         # every result of the step is in host memory before the step counts
 
     def barrier():
         if dist is not None:

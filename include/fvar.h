@@ -173,6 +173,20 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
 fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int scale_idx,
                                  const fvar_keep_policy *policy, void *out_host);
 
+/* The same with the copies taken off the step's stream: the upload runs on a stream of its own, the step on
+ * the context's stream once its tokens have arrived, the download on a third stream once the step has
+ * finished, through two staging slots each way inside the workspace.  Consecutive calls therefore overlap:
+ * the tokens of call n + 1 go up and the result of call n - 1 comes down while step n computes.  Returns as
+ * soon as everything is enqueued.  tokens_host must stay valid and unchanged, and out_host must not be read,
+ * until fvar_host_sync returns; both should be pinned (pageable memory makes the copies synchronous).
+ * The paper has no counterpart (it times whole generations on one GPU); this is the library's end-to-end
+ * entry point. */
+fvar_status fvar_scale_step_host_async(fvar_ctx *ctx, const void *tokens_host, int scale_idx,
+                                       const fvar_keep_policy *policy, void *out_host);
+
+/* Waits for every upload, step and download enqueued so far (host-blocking). */
+fvar_status fvar_host_sync(fvar_ctx *ctx);
+
 /* Commit the rows staged by the last step of `scale_idx` (O(1), host only).  FVAR_ESTATE if that
  * scale was not the last one stepped or was already appended. */
 fvar_status fvar_kv_append(fvar_ctx *ctx, int scale_idx);

@@ -80,6 +80,8 @@ def load_library() -> ct.CDLL:
         "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
         "fvar_scale_step": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_scale_step_host": (i, [vp, vp, i, P(_Policy), vp]),
+        "fvar_scale_step_host_async": (i, [vp, vp, i, vp, vp]),
+        "fvar_host_sync": (i, [vp]),
         "fvar_kv_append": (i, [vp, i]),
         "fvar_get_indices": (i, [vp, i, vp, P(i)]),
         "fvar_get_group_output": (i, [vp, i, vp]),
@@ -115,7 +117,7 @@ def load_library() -> ct.CDLL:
 
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_generate_projection",
             "fvar_get_projection", "fvar_set_codebook", "fvar_scale_transition", "fvar_get_feature", "fvar_scale_step",
-            "fvar_scale_step_host", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
+            "fvar_scale_step_host", "fvar_scale_step_host_async", "fvar_host_sync", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
@@ -380,6 +382,18 @@ class Fvar:
         self._check(self.lib.fvar_scale_step_host(self.ctx, tokens_host.data_ptr(), scale_idx, ct.byref(pol),
                                                   out_host.data_ptr()))
         return out_host
+
+    def scale_step_host_async(self, tokens_host: torch.Tensor, scale_idx: int, out_host: torch.Tensor, *, mode: int = DENSE,
+                              cfg_mode: int = CFG_PAIR, keep_ratio: float = 1.0, rank_per_group=None):
+        """Pipelined host entry point: enqueues upload, step and download and returns; host_sync() waits for them."""
+        assert not tokens_host.is_cuda and not out_host.is_cuda
+        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, None)
+        self._check(self.lib.fvar_scale_step_host_async(self.ctx, tokens_host.data_ptr(), scale_idx, ct.byref(pol),
+                                                        out_host.data_ptr()))
+        return out_host
+
+    def host_sync(self):
+        self._check(self.lib.fvar_host_sync(self.ctx))
 
     def kv_append(self, scale_idx: int):
         self._check(self.lib.fvar_kv_append(self.ctx, scale_idx))

@@ -122,6 +122,12 @@ struct fvar_ctx {
   int *tr_codes;
   int tr_scale;                        // last scale accumulated into tr_F (-1: none)
   int tr_B;
+  // pipelined host entry point: two staging slots each way, one stream per copy direction
+  bf16 *hin[2], *hout[2];
+  cudaStream_t h2d_st, d2h_st;
+  cudaEvent_t ev_in[2], ev_cmp[2], ev_out[2];
+  long long host_calls;
+  bool host_pipe_ok;
   int *idx, *inv, *split_counters;
   std::vector<size_t> qt_off;          // [scale][group] offset (elements) into qt_pool
   std::vector<int> qt_r;               // [scale][group] rank of the stored projection (0: none)
@@ -206,6 +212,7 @@ namespace {
 struct Layout {
   size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
   size_t tr_hn, tr_best, tr_codes, tr_F;
+  size_t hin[2], hout[2];
   std::vector<size_t> qt_off;
 };
 
@@ -274,6 +281,10 @@ Layout make_layout(const fvar_cfg *c) {
   L.tr_best = take(B * Mmax * 8);
   L.tr_codes = take(B * Mmax * 4);
   L.tr_F = take(B * M_last * C * 4);
+  for (int s2 = 0; s2 < 2; ++s2) {
+    L.hin[s2] = take(B * Mmax * C * 2);
+    L.hout[s2] = take(B * Mmax * C * 2);
+  }
   L.total = off;
   return L;
 }
@@ -407,6 +418,13 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->tr_hn = reinterpret_cast<float *>(at(L.tr_hn)); c->tr_F = reinterpret_cast<float *>(at(L.tr_F));
   c->tr_best = reinterpret_cast<unsigned long long *>(at(L.tr_best)); c->tr_codes = reinterpret_cast<int *>(at(L.tr_codes));
   c->codebook = nullptr; c->codebook_V = 0; c->tr_scale = -1; c->tr_B = 0;
+  for (int s2 = 0; s2 < 2; ++s2) {
+    c->hin[s2] = reinterpret_cast<bf16 *>(at(L.hin[s2]));
+    c->hout[s2] = reinterpret_cast<bf16 *>(at(L.hout[s2]));
+    c->ev_in[s2] = c->ev_cmp[s2] = c->ev_out[s2] = nullptr;
+  }
+  c->h2d_st = c->d2h_st = nullptr;
+  c->host_calls = 0;
   c->qt_off = L.qt_off;
   c->qt_r.assign(L.qt_off.size(), 0);
   c->qt_map.resize(L.qt_off.size());
@@ -484,6 +502,12 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+  c->host_pipe_ok = cudaStreamCreateWithFlags(&c->h2d_st, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&c->d2h_st, cudaStreamNonBlocking) == cudaSuccess;
+  for (int s2 = 0; s2 < 2 && c->host_pipe_ok; ++s2)
+    c->host_pipe_ok = cudaEventCreateWithFlags(&c->ev_in[s2], cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&c->ev_cmp[s2], cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&c->ev_out[s2], cudaEventDisableTiming) == cudaSuccess;
   if (gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   c->max_clusters = gemm_pair_max_clusters();
@@ -576,6 +600,13 @@ void fvar_destroy(fvar_ctx *ctx) {
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
   ctx->drop_prof_execs();
   ctx->drop_graphs();
+  if (ctx->h2d_st) cudaStreamDestroy(ctx->h2d_st);
+  if (ctx->d2h_st) cudaStreamDestroy(ctx->d2h_st);
+  for (int s2 = 0; s2 < 2; ++s2) {
+    if (ctx->ev_in[s2]) cudaEventDestroy(ctx->ev_in[s2]);
+    if (ctx->ev_cmp[s2]) cudaEventDestroy(ctx->ev_cmp[s2]);
+    if (ctx->ev_out[s2]) cudaEventDestroy(ctx->ev_out[s2]);
+  }
   if (ctx->cap_st) cudaStreamDestroy(ctx->cap_st);
   if (ctx->cap_st2) cudaStreamDestroy(ctx->cap_st2);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -1105,6 +1136,44 @@ fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int sca
   if (s != FVAR_OK) return s;
   FV_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->a, static_cast<size_t>(E) * M * ctx->C * 2, cudaMemcpyDeviceToHost, ctx->st), "out D2H");
   FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  return FVAR_OK;
+}
+
+fvar_status fvar_scale_step_host_async(fvar_ctx *ctx, const void *tokens_host, int scale_idx, const fvar_keep_policy *pol,
+                                       void *out_host) {
+  if (!ctx) return FVAR_EINVAL;
+  if (!pol) return fail(ctx, FVAR_EINVAL, "scale_step_host_async: policy is NULL");
+  if (pol->mode == FVAR_SKIP) return FVAR_OK;
+  if (!tokens_host || !out_host) return fail(ctx, FVAR_EINVAL, "scale_step_host_async: NULL tokens / out");
+  if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || ctx->B <= 0) return fail(ctx, FVAR_EINVAL, "scale_step_host_async: bad scale_idx or no cond");
+  if (!ctx->host_pipe_ok) return fail(ctx, FVAR_ECUDA, "scale_step_host_async: copy streams unavailable");
+  const size_t M = ctx->Mk[scale_idx], in_bytes = static_cast<size_t>(ctx->B) * M * ctx->C * 2;
+  const int E = pol->cfg_mode == FVAR_CFG_NULL_ONLY ? ctx->B / 2 : ctx->B;
+  const int s = static_cast<int>(ctx->host_calls & 1);
+  const bool reuse = ctx->host_calls >= 2;     // the slot was used two calls ago
+  // host -> device on the upload stream, once the step that last read this slot has finished
+  if (reuse) FV_CUDA(ctx, cudaStreamWaitEvent(ctx->h2d_st, ctx->ev_cmp[s], 0), "upload wait");
+  FV_CUDA(ctx, cudaMemcpyAsync(ctx->hin[s], tokens_host, in_bytes, cudaMemcpyHostToDevice, ctx->h2d_st), "tokens H2D");
+  FV_CUDA(ctx, cudaEventRecord(ctx->ev_in[s], ctx->h2d_st), "upload record");
+  // the step on the caller's stream, once its tokens are there and the slot's previous result has left
+  FV_CUDA(ctx, cudaStreamWaitEvent(ctx->st, ctx->ev_in[s], 0), "step wait");
+  if (reuse) FV_CUDA(ctx, cudaStreamWaitEvent(ctx->st, ctx->ev_out[s], 0), "step wait");
+  fvar_status rc = fvar_scale_step(ctx, ctx->hin[s], scale_idx, pol, ctx->hout[s]);
+  if (rc != FVAR_OK) return rc;
+  FV_CUDA(ctx, cudaEventRecord(ctx->ev_cmp[s], ctx->st), "step record");
+  // device -> host on the download stream
+  FV_CUDA(ctx, cudaStreamWaitEvent(ctx->d2h_st, ctx->ev_cmp[s], 0), "download wait");
+  FV_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->hout[s], static_cast<size_t>(E) * M * ctx->C * 2, cudaMemcpyDeviceToHost, ctx->d2h_st), "out D2H");
+  FV_CUDA(ctx, cudaEventRecord(ctx->ev_out[s], ctx->d2h_st), "download record");
+  ctx->host_calls++;
+  return FVAR_OK;
+}
+
+fvar_status fvar_host_sync(fvar_ctx *ctx) {
+  if (!ctx) return FVAR_EINVAL;
+  if (ctx->h2d_st) FV_CUDA(ctx, cudaStreamSynchronize(ctx->h2d_st), "upload synchronize");
+  FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+  if (ctx->d2h_st) FV_CUDA(ctx, cudaStreamSynchronize(ctx->d2h_st), "download synchronize");
   return FVAR_OK;
 }
 

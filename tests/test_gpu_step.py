@@ -446,3 +446,37 @@ def test_profile_pass_times_every_launch_and_changes_nothing(fv):
     p.gpu.restore_loaded()
     assert torch.equal(first, p.gpu.scale_step(toks, k, mode=fv.LOWRANK_RTR, rank_per_group=[r, r]))
     p.check_ok()
+
+
+def test_pipelined_host_entry_point_matches_the_synchronous_one(fv):
+    """Three late scales through fvar_scale_step_host_async (uploads, steps and downloads on three streams, two
+    staging slots each way; more calls than slots) give the same bits as the synchronous host entry point."""
+    shp = si.shape_var_d16(n_blocks=2)
+    B = 4
+    Ms = shp.tokens_per_scale()
+    results = {}
+    for variant in ("sync", "async"):
+        p = Pair(fv, shp, seed=114, B=B)
+        p.prefill(7)
+        outs = []
+        for rep in range(2):                                       # 6 calls: every staging slot is reused twice
+            p.gpu.restore_loaded()
+            for k in (7, 8, 9):
+                r = Ms[k] // 2
+                p.set_projections(k, [r, r])
+                toks = to_bf16_cuda(si.make_tokens(114, B, Ms[k], 1024, "spread")).cpu().pin_memory()
+                out = torch.empty((B // 2, Ms[k], 1024), dtype=torch.bfloat16).pin_memory()
+                kw = dict(mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY, rank_per_group=[r, r])
+                if variant == "sync":
+                    p.gpu.scale_step_host(toks, k, out, **kw)
+                else:
+                    p.gpu.scale_step_host_async(toks, k, out, **kw)
+                p.gpu.kv_append(k)
+                outs.append((toks, out))
+        if variant == "async":
+            p.gpu.host_sync()
+        p.check_ok()
+        results[variant] = [o.clone() for _, o in outs]
+    for a, b in zip(results["sync"], results["async"]):
+        assert torch.equal(a, b)
+    assert float(results["async"][-1].float().abs().sum()) > 0
