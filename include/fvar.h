@@ -284,6 +284,13 @@ fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, c
 fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out,
                            void *stream);
 
+/* The same product with the second operand given transposed: Wt dev bf16 [K][N] row-major (ldw = N, N % 8 == 0),
+ * out = A Wt + bias.  The tensor core then reads W as an MN-major operand; nothing is transposed in memory.
+ * block_n in {0 (picked), 64, 128, 256}; single-CTA tiles.  Used by the random projection F_r = Q^T F (Sec. 3.3 RP),
+ * whose second operand, the token rows, is stored [M][C]. */
+fvar_status fvar_gemm_bf16_wt(const void *A, const void *Wt, const void *bias, int R, int N, int K, int block_n,
+                              float *out, void *stream);
+
 /* The same product with the launch form given instead of picked: form FVAR_GEMM_AUTO (the library's
  * cost model, as fvar_gemm_bf16), FVAR_GEMM_SINGLE (one CTA per 128 x block_n tile, block_n in
  * {64, 128, 256}) or FVAR_GEMM_PAIR (two CTAs on neighbouring SMs share one 256 x block_n tile through

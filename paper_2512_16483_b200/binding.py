@@ -104,6 +104,7 @@ def load_library() -> ct.CDLL:
         "fvar_ln_modulate": (i, [vp, i, i, i, vp, vp, ll, f, vp, vp]),
         "fvar_gemm_bf16": (i, [vp, vp, vp, i, i, i, vp, vp]),
         "fvar_gemm_bf16_form": (i, [vp, vp, vp, i, i, i, i, i, vp, vp]),
+        "fvar_gemm_bf16_wt": (i, [vp, vp, vp, i, i, i, i, vp, vp]),
         "fvar_attention": (i, [vp, vp, vp, i, i, i, i, i, i, vp, vp]),
         "fvar_rtr_fill": (i, [vp, i, i, i, i, i, i, vp, vp, vp]),
         "fvar_select_rows_static": (i, [vp, i, i, i, i, vp, vp, vp]),
@@ -121,7 +122,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
+            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_gemm_bf16_wt", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
 
 
 def _stream() -> int:
@@ -195,6 +196,16 @@ def fvar_gemm_bf16_form(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.T
     out = torch.empty((R, N), dtype=torch.float32, device=A.device)
     _check_kernel(load_library().fvar_gemm_bf16_form(A.data_ptr(), W.data_ptr(), _ptr(bias), R, N, K, form, block_n,
                                                      out.data_ptr(), _stream()))
+    return out
+
+
+def fvar_gemm_bf16_wt(A: torch.Tensor, Wt: torch.Tensor, bias: Optional[torch.Tensor] = None, block_n: int = 0) -> torch.Tensor:
+    """A bf16 [R][K], Wt bf16 [K][N] (the second operand transposed, row-major) -> fp32 [R][N] = A Wt + bias."""
+    _dev(A, torch.bfloat16), _dev(Wt, torch.bfloat16)
+    R, K = A.shape
+    N = Wt.shape[1]
+    out = torch.empty((R, N), dtype=torch.float32, device=A.device)
+    _check_kernel(load_library().fvar_gemm_bf16_wt(A.data_ptr(), Wt.data_ptr(), _ptr(bias), R, N, K, block_n, out.data_ptr(), _stream()))
     return out
 
 

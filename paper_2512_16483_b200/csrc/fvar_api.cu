@@ -1291,6 +1291,27 @@ fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, 
   return FVAR_OK;
 }
 
+fvar_status fvar_gemm_bf16_wt(const void *A, const void *Wt, const void *bias, int R, int N, int K, int block_n, float *out,
+                              void *stream) {
+  if (!A || !Wt || !out || R <= 0 || N <= 0 || K <= 0 || K % 8 || N % 8) return kfail(FVAR_EINVAL, "gemm_wt: bad arguments");
+  int dev = 0, sms = 0;
+  FK_CUDA(cudaGetDevice(&dev), "get device");
+  FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
+  int bn = block_n ? block_n : gemm_pick_block_n((R + 127) / 128, N, K, sms);
+  if (bn != 64 && bn != 128 && bn != 256) return kfail(FVAR_EINVAL, "gemm_wt: block_n must be 64, 128 or 256");
+  CUtensorMap ta, tw;
+  if (!tmap_2d(&ta, A, K, R, K, 128) || !tmap_2d(&tw, Wt, N, K, N, 64)) return kfail(FVAR_EINVAL, "gemm_wt: operands must be 16-byte aligned");
+  GemmArgs g = gemm_args(R, N, K);
+  g.bias = static_cast<const bf16 *>(bias);
+  g.out_f32 = out;
+  g.ld_out = N;
+  g.w_mn_major = 1;
+  g.status = kernel_status_ptr();
+  if (!g.status) return kfail(FVAR_ECUDA, "gemm_wt: status word");
+  FK_CUDA(launch_gemm(EPI_F32, bn, ta, tw, g, sms, static_cast<cudaStream_t>(stream)), "gemm_wt");
+  return FVAR_OK;
+}
+
 fvar_status fvar_gemm_bf16(const void *A, const void *W, const void *bias, int R, int N, int K, float *out, void *stream) {
   return fvar_gemm_bf16_form(A, W, bias, R, N, K, FVAR_GEMM_AUTO, 0, out, stream);
 }

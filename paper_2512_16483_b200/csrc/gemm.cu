@@ -111,7 +111,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int e = tile / tiles_per_batch, rem = tile - e * tiles_per_batch;
         const int n_idx = rem / tiles_m, m_idx = rem - n_idx * tiles_m;
         const int row_a = e * p.a_batch_rows + m_idx * kBlockM;
-        const int row_w = e * p.b_batch_rows + n_idx * BN;
+        const int row_w = p.w_mn_major ? e * p.b_batch_rows : e * p.b_batch_rows + n_idx * BN;
         const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
 #ifdef FVAR_TRACE
@@ -127,7 +127,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           for (int ka = 0; ka < kKAtoms; ++ka) {
             const int kx = (kb * kKAtoms + ka) * kBlockK;      // fully out-of-range atoms are zero-filled
             tma_load_2d(sa + ka * Cfg::kAtomBytesA, &tmA, full_bar(stage), kx, row_a);
-            tma_load_2d(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB, &tmW, full_bar(stage), kx, row_w);
+            if (!p.w_mn_major) {
+              tma_load_2d(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB, &tmW, full_bar(stage), kx, row_w);
+            } else {
+              // 64-column blocks of W^T, each a run of K rows: block j of the stage holds kKAtoms x 64 rows of 128 bytes
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_2d(sa + Cfg::kStageBytesA + (j * kKAtoms + ka) * 8192, &tmW, full_bar(stage), n_idx * BN + j * 64, row_w + kx);
+            }
           }
           armed |= 1u << stage;
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
@@ -155,7 +162,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // The whole warp walks the loop (so that stage counters, addresses and descriptors are
       // warp-uniform values); one elected lane issues the MMAs and the commits.
       const bool leader = elect_one();
-      constexpr uint32_t idesc = umma_idesc_bf16(kBlockM, BN);
+      const uint32_t idesc = umma_idesc_bf16(kBlockM, BN) | (p.w_mn_major ? (1u << 16) : 0u);   // bit 16: B is MN-major
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -185,15 +192,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int ka = 0; ka < kKAtoms; ++ka) {
             da[ka] = smem_desc_sw128(sa + ka * Cfg::kAtomBytesA);
-            db[ka] = smem_desc_sw128(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB);
+            db[ka] = p.w_mn_major ? smem_desc_sw128_mn(sa + Cfg::kStageBytesA + ka * 8192, kKAtoms * 8192)
+                                  : smem_desc_sw128(sa + Cfg::kStageBytesA + ka * Cfg::kAtomBytesB);
           }
+          const uint32_t kstep_b = p.w_mn_major ? (2048u >> 4) : 2u;      // descriptor advance per 16 of K
           const uint32_t acc_first = (kb > kb0) ? 1u : 0u;
           if (leader) {
 #pragma unroll
           for (int ka = 0; ka < kKAtoms; ++ka) {
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)
-              umma_bf16(d_tmem, da[ka] + 2 * k, db[ka] + 2 * k, idesc, (ka != 0 || k != 0) ? 1u : acc_first);
+              umma_bf16(d_tmem, da[ka] + 2 * k, db[ka] + kstep_b * k, idesc, (ka != 0 || k != 0) ? 1u : acc_first);
           }
           umma_commit(empty_bar(stage));
           }

@@ -45,6 +45,9 @@ struct GemmArgs {
   // zero before the launch
   const float *col_sub;
   unsigned long long *best;
+  // W given MN-major: the tensor map describes W^T, a row-major [K][N] matrix (64-column boxes of 64 K rows), with
+  // batch e at row offset e * b_batch_rows along K.  Single-CTA kernel only.
+  int w_mn_major;
   // split-K (splits > 1): fp32 partial tiles [tile][split][128][BN] and one arrival counter per tile
   int splits;
   float *partial;

@@ -258,6 +258,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
+// The same for an MN-major tile: rows are K indices, each 128 bytes = 64 consecutive M/N elements, eight rows
+// per 1024-byte swizzle group (what a TMA box of 64 columns x k rows of a row-major [K][N] matrix writes).  Stride
+// field = distance between 8-row K groups (1024 B); leading field = distance between 64-element blocks along M/N.
+// Advancing along K by 16 rows adds 2048 bytes to the start.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr, uint32_t block_stride_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((block_stride_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
 // Instruction descriptor, kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9 and
 // 10-12 = 1), both K-major (bits 15, 16 = 0), N/8 in bits 17-22, M/16 in bits 24-28.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {

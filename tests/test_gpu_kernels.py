@@ -125,6 +125,21 @@ def test_gemm_bf16_every_form(fv, R, N, K, form, block_n):
     np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
 
 
+@pytest.mark.parametrize("R,N,K", [(128, 64, 64), (300, 200, 136), (1000, 1024, 512), (130, 1920, 344), (64, 2048, 8192)])
+@pytest.mark.parametrize("block_n", [0, 64, 128, 256])
+def test_gemm_bf16_second_operand_transposed(fv, R, N, K, block_n):
+    """out = A Wt with Wt stored [K][N]: the tensor core reads it as an MN-major operand (no transpose in memory)."""
+    rng = np.random.default_rng(R + N + K)
+    A = si.normal_bf16(rng, (R, K))
+    Wt = si.normal_bf16(rng, (K, N), 0.05)
+    b = si.normal_bf16(rng, (N,))
+    got = fv.fvar_gemm_bf16_wt(to_bf16_cuda(A), to_bf16_cuda(Wt), to_bf16_cuda(b), block_n).cpu().numpy()
+    _poll(fv)
+    ref = A.astype(np.float64) @ Wt.astype(np.float64) + b.astype(np.float64)
+    tol = 1e-5 * (np.abs(A).astype(np.float64) @ np.abs(Wt).astype(np.float64)).max() + 1e-6
+    np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
+
+
 def test_gemm_form_rejects_what_the_problem_does_not_allow(fv):
     A = to_bf16_cuda(np.zeros((128, 64), np.float32))
     W = to_bf16_cuda(np.zeros((128, 64), np.float32))
