@@ -393,7 +393,7 @@ cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int
 // One warp per output row; rows inside the index set are skipped.
 __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__ prev, float *__restrict__ out, int E,
                                                        int bmul, int boff, int h0, int w0, int h1, int w1, int C,
-                                                       const int *__restrict__ inv) {
+                                                       const int *__restrict__ inv, bf16 *__restrict__ xsplit, int mk) {
   pdl_wait();
   pdl_launch_dependents();
   const int M1 = h1 * w1;
@@ -414,6 +414,8 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
   const float4 *p10 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y1) * w0 + x0) * C);
   const float4 *p11 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y1) * w0 + x1) * C);
   float4 *dst = reinterpret_cast<float4 *>(out + (static_cast<long long>(b) * M1 + i) * C);
+  uint2 *hi_dst = xsplit ? reinterpret_cast<uint2 *>(xsplit + (static_cast<long long>(e) * 2 * mk + i) * C) : nullptr;
+  const long long lo_off = static_cast<long long>(mk) * C / 4;      // in 4-element groups
   const float w00 = (1.f - fy) * (1.f - fx), w01 = (1.f - fy) * fx, w10 = fy * (1.f - fx), w11 = fy * fx;
 #pragma unroll 4
   for (int c = threadIdx.x & 31; c < C / 4; c += 32) {
@@ -424,15 +426,22 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
     o.z = w00 * a.z + w01 * bq.z + w10 * cq.z + w11 * d.z;
     o.w = w00 * a.w + w01 * bq.w + w10 * cq.w + w11 * d.w;
     __stcs(dst + c, o);                          // written once, read by a later kernel: stream it
+    if (hi_dst != nullptr) {
+      const __nv_bfloat162 h0 = __floats2bfloat162_rn(o.x, o.y), h1 = __floats2bfloat162_rn(o.z, o.w);
+      const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+      const __nv_bfloat162 l0 = __floats2bfloat162_rn(o.x - f0.x, o.y - f0.y), l1 = __floats2bfloat162_rn(o.z - f1.x, o.w - f1.y);
+      hi_dst[c] = make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
+      hi_dst[lo_off + c] = make_uint2(*reinterpret_cast<const uint32_t *>(&l0), *reinterpret_cast<const uint32_t *>(&l1));
+    }
   }
 }
 
 cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1, int w1,
-                            int C, const int *inv, cudaStream_t st) {
+                            int C, const int *inv, bf16 *xsplit, int mk, cudaStream_t st) {
   const long long warps = static_cast<long long>(E) * h1 * w1;
   if (warps <= 0) return cudaSuccess;
   return launch_pdl(rtr_fill_kernel, dim3(static_cast<unsigned>((warps + 7) / 8)), dim3(256), 0, st, prev, out, E, bmul, boff, h0, w0, h1, w1, C,
-                                                                         inv);
+                                                                         inv, xsplit, mk);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -494,58 +503,21 @@ cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Transposed two-term bf16 split of the fp32 rows for the projection GEMM:
-// xt[e][c][m] = hi(x[row(e, m)][c]) and xt[e][c][Mk + m] = lo(...), hi = bf16(x), lo = bf16(x - hi),
-// so that the tensor-core product Q^T (hi + lo) carries ~16 mantissa bits of x.  Mk = M rounded up
-// to 64; columns [M, Mk) of both halves are written as zeros.  Row stride 2 * Mk.  A CTA moves a tile of
-// 64 tokens x 128 channels through shared memory: 512-byte row segments in (one float4 per lane), 128-byte
-// channel rows out (two tokens, one bf16x2, per lane).  C % 4 == 0.
-constexpr int kTrTok = 64, kTrCh = 128;
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C,
-                                                             int Mk, bf16 *__restrict__ xt) {
-  pdl_wait();
-  pdl_launch_dependents();
-  __shared__ float tile[kTrTok][kTrCh + 1];      // odd row stride: the column reads below do not conflict
-  const int e = blockIdx.z, m0 = blockIdx.x * kTrTok, c0 = blockIdx.y * kTrCh;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const float *src = x + static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb * C;
-#pragma unroll
-  for (int k = warp; k < kTrTok; k += 8) {
-    const int m = m0 + k, c = c0 + 4 * lane;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (m < M && c < C) v = __ldg(reinterpret_cast<const float4 *>(src + static_cast<long long>(m) * C + c));
-    tile[k][4 * lane] = v.x; tile[k][4 * lane + 1] = v.y; tile[k][4 * lane + 2] = v.z; tile[k][4 * lane + 3] = v.w;
-  }
-  __syncthreads();
-  bf16 *dst = xt + static_cast<long long>(e) * C * 2 * Mk;
-#pragma unroll 4
-  for (int k = warp; k < kTrCh; k += 8) {        // one channel per warp pass; each lane writes two tokens
-    const int c = c0 + k, m = m0 + 2 * lane;
-    if (c < C) {                                 // m + 1 < Mk always: Mk is a multiple of 64
-      const float v0 = tile[2 * lane][k], v1 = tile[2 * lane + 1][k];
-      const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
-      const float2 hf = __bfloat1622float2(hi);
-      const __nv_bfloat162 lo = __floats2bfloat162_rn(v0 - hf.x, v1 - hf.y);
-      *reinterpret_cast<__nv_bfloat162 *>(dst + static_cast<long long>(c) * 2 * Mk + m) = hi;
-      *reinterpret_cast<__nv_bfloat162 *>(dst + static_cast<long long>(c) * 2 * Mk + Mk + m) = lo;
-    }
-  }
-}
-
-cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
-                                  cudaStream_t st) {
-  if (C % 4 != 0) return cudaErrorInvalidValue;
-  dim3 grid(Mk / kTrTok, (C + kTrCh - 1) / kTrCh, E);
-  return launch_pdl(transpose_bf16_kernel, dim3(grid), dim3(256), 0, st, x, xmap, M, C, Mk, xt);
-}
-
-// ------------------------------------------------------------------------------------------------
-__global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__restrict__ x, long long n8) {
+__global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__restrict__ x, long long n8, long long per8,
+                                     bf16 *__restrict__ xsplit, long long half8, int bmul, int boff) {
   pdl_wait();
   pdl_launch_dependents();
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n8) return;
   const uint4 u = __ldg(reinterpret_cast<const uint4 *>(tok) + i);
+  if (xsplit != nullptr) {                       // hi = the token itself, lo = 0, for the elements that are computed
+    const long long b = i / per8, off = i - b * per8;
+    if (b >= boff && (b - boff) % bmul == 0) {
+      uint4 *dst = reinterpret_cast<uint4 *>(xsplit) + ((b - boff) / bmul) * 2 * half8 + off;
+      dst[0] = u;
+      dst[half8] = make_uint4(0u, 0u, 0u, 0u);
+    }
+  }
   const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
   const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]), c = __bfloat1622float2(h[2]),
                d = __bfloat1622float2(h[3]);
@@ -553,10 +525,12 @@ __global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__rest
   reinterpret_cast<float4 *>(x)[2 * i + 1] = make_float4(c.x, c.y, d.x, d.y);
 }
 
-cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st) {
-  const long long n8 = static_cast<long long>(B) * per_elem / 8;
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, int M, int C, bf16 *xsplit, int mk, int bmul, int boff,
+                                 cudaStream_t st) {
+  const long long per8 = static_cast<long long>(M) * C / 8, n8 = static_cast<long long>(B) * per8;
   if (n8 <= 0) return cudaSuccess;
-  return launch_pdl(tokens_to_f32_kernel, dim3(static_cast<unsigned>((n8 + 255) / 256)), dim3(256), 0, st, tok, x, n8);
+  return launch_pdl(tokens_to_f32_kernel, dim3(static_cast<unsigned>((n8 + 255) / 256)), dim3(256), 0, st, tok, x, n8, per8, xsplit,
+                    static_cast<long long>(mk) * C / 8, bmul, boff);
 }
 
 __global__ void out_to_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C, bf16 *__restrict__ out) {

@@ -111,7 +111,8 @@ struct fvar_ctx {
   uint8_t *ws;
   size_t ws_bytes;
   unsigned *status;
-  bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *xt, *qt_pool;
+  bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *qt_pool;
+  bf16 *xsplit[2];                     // hi / lo bf16 split of a group's input rows, [E][2][Mk][C]; groups alternate
   float *ada, *gcache, *x0, *xs, *scores, *split_partial;
   // transition between scale steps: codebook (caller's memory), half-norms, packed arg-max words, codes and
   // the accumulated feature map F_k at the last scale's resolution
@@ -132,7 +133,7 @@ struct fvar_ctx {
   std::vector<size_t> qt_off;          // [scale][group] offset (elements) into qt_pool
   std::vector<int> qt_r;               // [scale][group] rank of the stored projection (0: none)
   std::vector<CUtensorMap> qt_map;     // [scale][group]
-  std::vector<CUtensorMap> xt_map;     // [scale][3]
+  std::vector<CUtensorMap> xsplit_map; // [scale][2 buffers]: rows = elements x (hi rows, lo rows), 64 x 64 boxes
   std::vector<CUtensorMap> kmap, vmap, ckmap, cvmap;   // per block
   // GEMM A operands: one map per box height (16, 32, 64, 128 rows); q_map feeds the attention kernel
   struct ActMaps { CUtensorMap m[4]; };
@@ -210,7 +211,7 @@ struct fvar_ctx {
 namespace {
 
 struct Layout {
-  size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xt, scores, idx, inv, qt_pool, total;
+  size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xsplit[2], scores, idx, inv, qt_pool, total;
   size_t tr_hn, tr_best, tr_codes, tr_F;
   size_t hin[2], hout[2];
   std::vector<size_t> qt_off;
@@ -261,7 +262,8 @@ Layout make_layout(const fvar_cfg *c) {
   L.q = take(B * Mmax * C * 2);
   L.a = take(B * Mmax * C * 2);
   L.hbuf = take(B * Mmax * F * 2);
-  L.xt = take(B * C * 2 * Mk * 2);
+  L.xsplit[0] = take(B * 2 * Mk * C * 2);
+  L.xsplit[1] = take(B * 2 * Mk * C * 2);
   L.scores = take(B * Mmax * 4);
   L.idx = take(G * B * Mmax * 4);
   L.inv = take(G * B * Mmax * 4);
@@ -412,7 +414,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->x0 = reinterpret_cast<float *>(at(L.x0)); c->xs = reinterpret_cast<float *>(at(L.xs));
   c->y = reinterpret_cast<bf16 *>(at(L.y)); c->q = reinterpret_cast<bf16 *>(at(L.q));
   c->a = reinterpret_cast<bf16 *>(at(L.a)); c->hbuf = reinterpret_cast<bf16 *>(at(L.hbuf));
-  c->xt = reinterpret_cast<bf16 *>(at(L.xt)); c->scores = reinterpret_cast<float *>(at(L.scores));
+  c->xsplit[0] = reinterpret_cast<bf16 *>(at(L.xsplit[0])); c->xsplit[1] = reinterpret_cast<bf16 *>(at(L.xsplit[1]));
+  c->scores = reinterpret_cast<float *>(at(L.scores));
   c->idx = reinterpret_cast<int *>(at(L.idx)); c->inv = reinterpret_cast<int *>(at(L.inv));
   c->qt_pool = reinterpret_cast<bf16 *>(at(L.qt_pool));
   c->tr_hn = reinterpret_cast<float *>(at(L.tr_hn)); c->tr_F = reinterpret_cast<float *>(at(L.tr_F));
@@ -470,11 +473,10 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
          tmap_2d(&c->h_map.m[t], c->hbuf, F, act_rows, F, box) && tmap_2d(&c->silu_map.m[t], c->silu_c, C, c->Bmax, C, box);
   }
   ok = ok && tmap_2d(&c->q_map, c->q, C, act_rows, C, 128);
-  c->xt_map.resize(static_cast<size_t>(cfg->n_scales) * 3);
+  c->xsplit_map.resize(static_cast<size_t>(cfg->n_scales) * 2);
   for (int k = 0; k < cfg->n_scales && ok; ++k)
-    for (int t = 0; t < 3 && ok; ++t)
-      ok = tmap_2d(&c->xt_map[k * 3 + t], c->xt, align_up(c->Mk[k], 64) + c->Mk[k], static_cast<size_t>(c->Bmax) * C,
-                   2 * align_up(c->Mk[k], 64), kBNs[t]);
+    for (int t = 0; t < 2 && ok; ++t)
+      ok = tmap_2d(&c->xsplit_map[k * 2 + t], c->xsplit[t], C, static_cast<size_t>(c->Bmax) * 2 * align_up(c->Mk[k], 64), C, 64);
   c->kmap.resize(nb); c->vmap.resize(nb); c->ckmap.resize(nb); c->cvmap.resize(nb);
   const int BH = c->Bmax * c->H, D = c->D;
   for (int b = 0; b < nb && ok; ++b) {
@@ -885,7 +887,10 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   cudaStream_t st = ctx->st;
 
   ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * B * M * C);
-  FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, B, static_cast<long long>(M) * C, st), "tokens_to_f32");
+  const int Mk = static_cast<int>(align_up(M, 64));
+  // the projection of a late group reads its input rows as a hi / lo bf16 split, written by whoever produces them
+  FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, B, M, C, rank[0] < M ? ctx->xsplit[0] : nullptr, Mk,
+                                    bmul, boff, st), "tokens_to_f32");
   ctx->launched();
   const float *X_in = ctx->x0;
   const RowMap bmap{bmul, boff, M};              // buffers indexed by the caller's batch element
@@ -903,6 +908,8 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
     int *idx_g = ctx->idx + static_cast<size_t>(g) * ctx->Bmax * ctx->Mmax;
     int *inv_g = ctx->inv + static_cast<size_t>(g) * ctx->Bmax * ctx->Mmax;
     const RowMap smap{1, 0, r};                  // the compact work stream of this group
+    // the next group's projection, if it has one, reads this group's output as a hi / lo bf16 split
+    bf16 *next_split = (g + 1 < G && rank[g + 1] < M) ? ctx->xsplit[(g + 1) & 1] : nullptr;
 
     // While a graph is being captured, the index selection and the restoration fill of a late group
     // go to a second stream: they depend only on the group's input and on the previous scale's
@@ -931,26 +938,23 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       }
       // restoration fill: rows outside the index set, from the upsampled cache of the previous scale
       ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M, side);
-      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, side), "rtr_fill");
+      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, next_split, Mk, side), "rtr_fill");
       ctx->launched(side);
       if (forked) FV_CUDA(ctx, cudaEventRecord(ctx->ev_join, side), "join record");
-      const int Mk = static_cast<int>(align_up(M, 64));
-      ctx->prof_begin(FVAR_KCLASS_TRANSPOSE, 0.0, 4.0 * E * M * C + 4.0 * E * C * Mk);
-      FV_CUDA(ctx, launch_transpose_bf16(X_in, bmap, E, M, C, Mk, ctx->xt, st), "transpose");
-      ctx->launched();
-      // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e; the reduction
-      // runs over the hi and lo halves of X
+      // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e.  The reduction runs over the hi
+      // and lo bf16 parts of X ([Qt | Qt] against [hi ; lo]); X's rows are read in place as an MN-major operand.
       GemmArgs ga = gemm_args(r, C, Mk + M);
       ga.nbatch = E;
       ga.a_batch_rows = 0;
-      ga.b_batch_rows = C;
+      ga.b_batch_rows = 2 * Mk;
+      ga.w_mn_major = 1;
       ga.out_f32 = ctx->xs;
       ga.ld_out = C;
       ga.status = ctx->status;
       const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, Mk + M, ctx->num_sms);
-      ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + static_cast<double>(E) * M * C) + 4.0 * E * r * C);
+      ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + 2.0 * E * M * C) + 4.0 * E * r * C);
       FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
-                               ctx->xt_map[scale_idx * 3 + bn_index(bn)], ga, ctx->num_sms, st), "projection gemm");
+                               ctx->xsplit_map[scale_idx * 2 + (g & 1)], ga, ctx->num_sms, st), "projection gemm");
       ctx->launched();
     }
 
@@ -1030,6 +1034,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
           if (forked) FV_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0), "join wait");
           ga.out_f32 = gout; ga.omap = bmap;
           ga.scatter = late ? idx_g : nullptr;
+          ga.xsplit = next_split; ga.xsplit_mk = Mk;
         } else {
           ga.out_f32 = ctx->xs; ga.omap = smap;
         }
@@ -1346,7 +1351,7 @@ fvar_status fvar_rtr_fill(const float *prev, int B, int h0, int w0, int h1, int 
                           void *stream) {
   if (!prev || !out || B <= 0 || h0 <= 0 || w0 <= 0 || h1 <= 0 || w1 <= 0 || C <= 0 || C % 4)
     return kfail(FVAR_EINVAL, "rtr_fill: bad arguments");
-  FK_CUDA(launch_rtr_fill(prev, out, B, 1, 0, h0, w0, h1, w1, C, inv, static_cast<cudaStream_t>(stream)), "rtr_fill");
+  FK_CUDA(launch_rtr_fill(prev, out, B, 1, 0, h0, w0, h1, w1, C, inv, nullptr, 0, static_cast<cudaStream_t>(stream)), "rtr_fill");
   return FVAR_OK;
 }
 

@@ -180,6 +180,19 @@ __device__ __forceinline__ void epilogue_chunk(const GemmArgs &p, const uint32_t
       }
     }
     warp_store_f32(stage, lane, v, dst);
+    if (p.xsplit != nullptr) {                   // uniform across the grid
+      bf16 *hi = nullptr;
+      if (valid) {
+        const int e = row / p.rows_per_batch, j = row - e * p.rows_per_batch;
+        const int jo = p.scatter ? __ldg(p.scatter + static_cast<long long>(e) * p.rows_per_batch + j) : j;
+        hi = p.xsplit + (static_cast<long long>(e) * 2 * p.xsplit_mk + jo) * p.ld_out + col0;
+      }
+      float lo[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) lo[i] = v[i] - __bfloat162float(__float2bfloat16_rn(v[i]));
+      warp_store_bf16(stage, lane, v, hi);
+      warp_store_bf16(stage, lane, lo, hi ? hi + static_cast<long long>(p.xsplit_mk) * p.ld_out : nullptr);
+    }
   }
 }
 

@@ -37,6 +37,10 @@ struct GemmArgs {
   const float *gate;      // vector of caller batch element b at gate + b * gate_stride, or nullptr (gate = 1)
   long long gate_stride;
   const int *scatter;     // [E][rows_per_batch] or nullptr
+  // EPI_RESID, optional: the result also goes out as its two-term bf16 split for the next group's projection,
+  // xsplit[e][half][row j'][col] with half 0 = hi = bf16(x), half 1 = lo = bf16(x - hi); xsplit_mk rows per half
+  bf16 *xsplit;
+  int xsplit_mk;
   // EPI_QKV: virtual column = col + col_base; [0,C) -> q, [C,2C) -> K cache, [2C,3C) -> transposed V cache
   bf16 *kc, *vt;
   int C, H, D, L_cap, L_prev, col_base;
@@ -136,11 +140,13 @@ cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_f
 cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int C, const float *shift,
                                const float *scale, long long vec_stride, int bmul, int boff,
                                const bf16 *gamma, float eps, bf16 *y, cudaStream_t st);
+// xsplit (optional): the filled rows also go out as their two-term bf16 split, [E][2][mk][C] (see GemmArgs::xsplit).
 cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1,
-                            int w1, int C, const int *inv, cudaStream_t st);
-cudaError_t launch_transpose_bf16(const float *x, RowMap xmap, int E, int M, int C, int Mk, bf16 *xt,
-                                  cudaStream_t st);
-cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, long long per_elem, cudaStream_t st);
+                            int w1, int C, const int *inv, bf16 *xsplit, int mk, cudaStream_t st);
+// xsplit (optional): the rows of the computed elements b = e * bmul + boff also go out as hi = token, lo = 0 in the
+// [E][2][mk][C] split layout (tokens are bf16 already).
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, int M, int C, bf16 *xsplit, int mk, int bmul, int boff,
+                                 cudaStream_t st);
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);
 cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned long long seed, int group, int scale,
                                        cudaStream_t st);
