@@ -125,3 +125,26 @@ def test_cfg_combine(fv, guidance):
     np.testing.assert_allclose(got, ref, rtol=2 ** -8, atol=1e-6)
     if guidance == 0.0:
         assert np.array_equal(got, x[1::2])                      # CFG = 0: the null-prompt branch, bit for bit
+
+
+def test_transition_at_the_infinity_shape(fv):
+    """The last two scales of the Infinity-2B-shaped schedule (48 x 48 and 64 x 64 tokens, C = 2048) with the 8192
+    codewords the closed-loop benchmark uses: every code, the whole accumulated map and the next tokens."""
+    shp = si.ModelShape(n_blocks=1, blocks_per_group=1, width=2048, n_heads=16, head_dim=128, ffn_dim=2048,
+                        scales=(48, 64))
+    B, V = 1, 8192
+    g = _ctx(fv, shp, B, seed=307)
+    C, Ms, hw = shp.width, shp.tokens_per_scale(), shp.hw()
+    Z = si.make_codebook(308, V, C)
+    g.set_codebook(to_bf16_cuda(Z))
+    F_ref = np.zeros((Ms[-1], C))
+    for k in range(2):
+        fo = si.make_step_outputs(309, k, B, Ms[k], Z, 0.05)
+        codes, nxt = g.scale_transition(to_bf16_cuda(fo), k, None if k == 1 else Ms[1])
+        assert g.poll_status() == fv.OK
+        c_ref, F_ref, n_ref = orc.scale_transition(F_ref, fo[0], Z, hw[k], hw[-1], None if k == 1 else hw[1])
+        assert np.array_equal(codes[0].cpu().numpy(), c_ref)
+        got_F = g.get_feature(B, Ms[-1], C)[0].cpu().numpy().astype(np.float64)
+        np.testing.assert_allclose(got_F, F_ref, rtol=0, atol=2e-5 * (k + 1) * np.abs(Z).max())
+        if k == 0:
+            np.testing.assert_allclose(bf16_to_numpy(nxt[0]), n_ref, rtol=2 ** -8, atol=1e-5 * np.abs(Z).max())
