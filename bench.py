@@ -171,9 +171,9 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------- the oracle leg
 
 def oracle_leg(wl, steps, warmup):
-    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  VAR shapes: 2 of the CFG
-    pairs, every block, every late scale.  Infinity shape: the one CFG pair, the first block group of the 8,
-    every non-skipped late scale, extrapolated x 8 groups.  Returns (tokens/s, seconds per step,
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload.  VAR shapes: up to 8 of the
+    CFG pairs (d16) or 2 (d30), every block, every late scale.  Infinity shape: the one CFG pair, the first block
+    group of the 8, every non-skipped late scale, extrapolated x 8 groups.  Returns (tokens/s, seconds per step,
     description, threads)."""
     from oracle import fvar_oracle as orc
     try:
@@ -189,7 +189,7 @@ def oracle_leg(wl, steps, warmup):
     big = wl["shape"] == "inf2b"
     groups = 1 if big else full.n_groups
     shp.n_blocks = groups * shp.blocks_per_group
-    B = 2 if big else 4
+    B = 2 if big else (min(wl["B"], 16) if wl["shape"] == "d16" else 4)      # bounded sample: 10-15 s of CPU work
     Ms = shp.tokens_per_scale()
     k0 = wl["first_late"]
     weights = si.make_weights(SEED, shp)
