@@ -82,6 +82,7 @@ def scale_plan(wl, shp):
     """Per late scale index: None (skip) or the list of ranks per block group (M = dense)."""
     from paper_2512_16483_b200 import schedule
     Ms, plan = shp.tokens_per_scale(), {}
+    paper_modes = dict(zip(*schedule.infinity_schedule(True)))
     for k in range(wl["first_late"], len(Ms)):
         keep = wl["keep"]
         if k < wl.get("dense_until", 0):
@@ -90,7 +91,7 @@ def scale_plan(wl, shp):
             plan[k] = [min(keep[1], Ms[k])] * shp.n_groups
         elif keep in ("table", "paper"):
             side = shp.scales[k]
-            if keep == "paper" and schedule.INFINITY_ALPHA[schedule.INFINITY_LATE_SCALES.index(side)] == 0.0:
+            if keep == "paper" and paper_modes[side] == schedule.SKIP:
                 plan[k] = None
             else:
                 plan[k] = schedule.infinity_group_ranks(side, shp.width, shp.n_groups)

@@ -86,8 +86,8 @@ typedef struct {
                                  replace the selection (r_max = largest r of the call); NULL in production */
   int select;                 /* FVAR_SELECT_TOPR: the r highest row scores (default, 0).
                                  FVAR_SELECT_SAMPLE: r rows drawn without replacement with probability
-                                 proportional to the row score (Sec. 3.3: "each row i chosen with probability
-                                 P_i"): the r largest keys s_i / E_i, E_i ~ Exp(1) given in sample_noise        */
+                                 proportional to the row score (the sampling reading of Sec. 3.3 RTR): the r
+                                 largest keys s_i / E_i, E_i ~ Exp(1) given in sample_noise                     */
   const float *sample_noise;  /* dev fp32 [n_groups][B_eff][M] of Exp(1) variates (> 0) for FVAR_SELECT_SAMPLE     */
 } fvar_keep_policy;
 
@@ -127,8 +127,8 @@ fvar_status fvar_generate_projection(fvar_ctx *ctx, int scale_idx, int group, in
  * FVAR_ESTATE if none is stored. */
 fvar_status fvar_get_projection(fvar_ctx *ctx, int scale_idx, int group, void *Qt_out, int *r_host);
 
-/* Codebook Z of the quantizer Q (Algorithm 1: "the quantizer Q, which typically includes a codebook
- * Z in R^{V x d}"): Z dev bf16 [V][C], 16-byte aligned, 1 <= V <= 65536, d = C (the block width).  The
+/* Codebook Z (V codewords of width d) of the quantizer Q that Algorithm 1 lists among its inputs:
+ * Z dev bf16 [V][C], 16-byte aligned, 1 <= V <= 65536, d = C (the block width).  The
  * library keeps the pointer (the caller keeps the memory alive) and computes |Z_v|^2 / 2 into its workspace.
  * FVAR_EUNSUPPORTED for a larger codebook. */
 fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V);
@@ -149,8 +149,8 @@ fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, 
 
 /* Classifier-free guidance on the outputs of a step that ran both branches: out[p] = null + guidance *
  * (prompt - null) for the CFG pair p = elements (2p, 2p + 1) = (prompt, null prompt) of `pair`.  The paper
- * only says that VAR "adopts classifier-free guidance to combine text prompts with null text prompts" and
- * that setting it to 0 leaves the null-prompt branch alone (Sec. 3.2, Sec. 3.3); applying it to the block
+ * only states that VAR combines the prompt and null-prompt branches by classifier-free guidance and that
+ * a guidance of 0 leaves the null-prompt branch alone (Sec. 3.2, Sec. 3.3); applying it to the block
  * outputs is this library's reading.  pair dev bf16 [B][per_elem], B even, per_elem % 8 == 0; out dev bf16
  * [B / 2][per_elem]; both 16-byte aligned. */
 fvar_status fvar_cfg_combine(const void *pair, int B, long long per_elem, float guidance, void *out, void *stream);
@@ -220,8 +220,12 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx);
  * Partial tiles go through a scratch area of the workspace and are added in a fixed order, so results do
  * not depend on timing.  When allowed, the picker splits only reductions of K >= 4096 whose tiles would
  * leave more than half of the SMs idle.  Measured: +2 % on the Infinity-shaped late scales, -5 % on the
- * VAR-d16 ones, hence off by default. */
-enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1 };
+ * VAR-d16 ones, hence off by default.
+ * FVAR_OPT_SKINNY_MAX_ROWS (default 64; 0 .. 512): GEMMs of a step with at most this many rows
+ * R = B_eff * r take the weight-streaming form (the weights are the M side of the MMA, the K range of a
+ * 128-feature tile is spread over a thread-block cluster that reduces through distributed shared memory),
+ * which is bound by reading the weights once; 0 never uses it. */
+enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1, FVAR_OPT_SKINNY_MAX_ROWS = 2 };
 fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value);
 
 /* Measurement aid: while enabled, every kernel launch of this context is bracketed by CUDA events on
@@ -229,8 +233,7 @@ fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value);
  * time, the number of launches and the algorithmic flops and bytes (minimum traffic: operands read
  * once, results written once) of the launches recorded since fvar_profile_enable(ctx, 1). */
 enum { FVAR_KCLASS_GEMM = 0, FVAR_KCLASS_ATTENTION = 1, FVAR_KCLASS_LN = 2, FVAR_KCLASS_SCORE = 3,
-       FVAR_KCLASS_SELECT = 4, FVAR_KCLASS_TRANSPOSE = 5, FVAR_KCLASS_RTR_FILL = 6, FVAR_KCLASS_CONVERT = 7,
-       FVAR_KCLASS_COUNT = 8 };
+       FVAR_KCLASS_SELECT = 4, FVAR_KCLASS_RTR_FILL = 5, FVAR_KCLASS_CONVERT = 6, FVAR_KCLASS_COUNT = 7 };
 fvar_status fvar_profile_enable(fvar_ctx *ctx, int on);
 fvar_status fvar_profile_read(fvar_ctx *ctx, int kclass, double *total_ms, long long *launches, double *flops,
                               double *bytes);
@@ -253,6 +256,34 @@ fvar_status fvar_reset(fvar_ctx *ctx);
 void fvar_destroy(fvar_ctx *ctx);
 /* Message of the last error on this context (or of the last failed fvar_init when ctx is NULL). */
 const char *fvar_last_error(const fvar_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------
+ * The method's schedule (host only; no context, no device): which scale steps run how, and the
+ * rank r of every block group.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Rank for a keep ratio: r = floor(keep_ratio * M + 0.5), clamped to [1, M] (what fvar_scale_step
+ * uses when rank_per_group is NULL).  0 if M <= 0. */
+int fvar_rank_from_keep_ratio(int M, float keep_ratio);
+
+/* Rank that a rank ratio stands for.  Sec. 3.2, Eq. "low_rank_percent": a ratio is a fraction of
+ * n = min(M, d), so r = floor(ratio * min(M, width) + 0.5), clamped to [1, M].  0 on a bad shape. */
+int fvar_rank_from_table_ratio(int M, int width, double ratio);
+
+/* App. A.1, the table of mean rank ratios at energy threshold alpha = 0.96: the entry of block chunk
+ * `chunk` (0..7) at late scale `scale_side` (40, 48 or 64).  FVAR_EINVAL outside the table. */
+fvar_status fvar_infinity_rank_ratio(int chunk, int scale_side, double *ratio_host);
+
+/* Rank per block group at a late Infinity scale (40, 48 or 64 tokens a side, M = side^2) from that
+ * table: ranks_host[g], g < n_groups.  With 8 groups, group g is chunk g; another group count takes
+ * the chunk at the nearest relative depth (the paper prints the table for 8 chunks only). */
+fvar_status fvar_infinity_group_ranks(int scale_side, int width, int n_groups, int *ranks_host);
+
+/* The 13-step Infinity schedule of Sec. 4.1: side length and mode (FVAR_DENSE / FVAR_LOWRANK_RTR /
+ * FVAR_SKIP) of every scale step.  Scales 1..32 are dense; 40, 48, 64 have thresholds alpha =
+ * {0.96, 0, 0} and alpha = 0 skips the step (paper_schedule != 0), or all three are approximated
+ * (paper_schedule == 0).  Writes min(13, capacity) entries to each non-NULL array, 13 to *count_host. */
+fvar_status fvar_infinity_schedule(int paper_schedule, int capacity, int *sides_host, int *modes_host, int *count_host);
 
 /* ---------------------------------------------------------------------------------------------
  * Kernel-level entry points: the individual steps of the path, callable on caller-owned device
@@ -297,10 +328,13 @@ fvar_status fvar_gemm_bf16_wt(const void *A, const void *Wt, const void *bias, i
  * tcgen05.mma.cta_group::2, block_n in {128, 256}; needs R > 128).  block_n = 0 lets the cost model
  * pick the width for the given form.  The transformer block of the step is the workload's own
  * definition (the paper only names it a "VAR block", Sec. 3.1), so this is a kernel-level entry for
- * tests and tuning.  FVAR_EINVAL for a form / width the problem does not allow. */
+ * tests and tuning.  FVAR_GEMM_SKINNY: the weight-streaming form for R <= 512 (see FVAR_OPT_SKINNY_MAX_ROWS);
+ * block_n is then the number of K ranges per 128-feature tile, 1 .. 8, or 0 to let the library pick.
+ * FVAR_EINVAL for a form / width the problem does not allow. */
 #define FVAR_GEMM_AUTO 0
 #define FVAR_GEMM_SINGLE 1
 #define FVAR_GEMM_PAIR 2
+#define FVAR_GEMM_SKINNY 3
 fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
                                 int block_n, float *out, void *stream);
 
@@ -309,6 +343,12 @@ fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, 
  * transposed); out dev bf16 [B][r][H*D].  D in {64, 128}; L_cap % 8 == 0; 1 <= L <= L_cap. */
 fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B, int H, int r, int D, int L,
                            int L_cap, void *out, void *stream);
+
+/* Asks the L2 cache to fetch [ptr, ptr + bytes) (ptr dev, 16-byte aligned; bytes rounded down to a multiple of
+ * 16): a hint for data a later kernel will stream, e.g. the weights of the next layer while the current one
+ * computes.  The range must not be written by work still in flight on the stream.  The paper has no
+ * counterpart (it describes no kernels); the step uses the same hint between its GEMMs. */
+fvar_status fvar_l2_prefetch(const void *ptr, size_t bytes, void *stream);
 
 /* Restoration fill of Eq. "redefine" with Eq. "upcache": for every row i of batch element b with
  * inv[b][i] < 0, out[b][i] = Up(prev[b])[i], bilinear with half-pixel centres on the (h, w) grid.

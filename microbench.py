@@ -1,10 +1,11 @@
 """Stand-alone timings of the library's kernels through the C ABI (CUDA events, one GPU).
 
-    python -m paper_2512_16483_b200.microbench gemm        # FVAR_GEMM_BLOCK_N=64|128|256 forces a width, FVAR_GEMM_PAIR=0|1 the launch form
-    python -m paper_2512_16483_b200.microbench gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
-    python -m paper_2512_16483_b200.microbench attention
-    python -m paper_2512_16483_b200.microbench memory      # score, LayerNorm + modulate, restoration fill, selection
-    python -m paper_2512_16483_b200.microbench transition  # between two scale steps: codeword search, Up-accumulate, Down
+    python microbench.py gemm        # FVAR_GEMM_BLOCK_N=64|128|256 forces a width, FVAR_GEMM_PAIR=0|1 the launch form
+    python microbench.py skinny      # the weight-streaming form on the Infinity-2B-shaped late GEMMs
+    python microbench.py gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
+    python microbench.py attention
+    python microbench.py memory      # score, LayerNorm + modulate, restoration fill, selection
+    python microbench.py transition  # between two scale steps: codeword search, Up-accumulate, Down
 
 GEMM calls rotate over several weight copies (more than L2 holds) and are captured in one CUDA graph so
 that host launch cost does not enter the time.
@@ -16,7 +17,7 @@ import sys
 
 import torch
 
-from . import binding as fv
+from paper_2512_16483_b200 import binding as fv
 
 
 def _time(fn, n=20, warm=3):
@@ -61,6 +62,37 @@ def gemm():
         us = _gemm_graph_us(lib, R, N, K)
         print("BN=%s R=%d N=%d K=%d: %.2f us  %.1f TFLOP/s  weights %.0f GB/s" % (
             bn, R, N, K, us, 2 * R * N * K / us / 1e6, N * K * 2 / us / 1e3))
+
+
+def _gemm_form_graph_us(lib, R, N, K, form, block_n):
+    ncopy = max(2, min(32, int(300e6 // (N * K * 2))))
+    A = torch.randn(R, K, device="cuda").bfloat16()
+    Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(ncopy)]
+    out = torch.empty(R, N, device="cuda", dtype=torch.float32)
+
+    def call(i):
+        st = lib.fvar_gemm_bf16_form(A.data_ptr(), Ws[i % ncopy].data_ptr(), None, R, N, K, form, block_n, out.data_ptr(),
+                                     torch.cuda.current_stream().cuda_stream)
+        assert st == 0, st
+    for i in range(ncopy):
+        call(i)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(ncopy):
+            call(i)
+    return _time(g.replay, n=5, warm=1) / ncopy
+
+
+def skinny():
+    """The weight-streaming form against the picked form on the GEMM shapes of the Infinity-2B-shaped late steps."""
+    lib = fv.load_library()
+    for R in (16, 64, 111, 170, 256, 336, 410):
+        for N, K in ((6144, 2048), (2048, 2048), (8192, 2048), (2048, 8192)):
+            auto = _gemm_form_graph_us(lib, R, N, K, fv.GEMM_AUTO, 0)
+            sk = _gemm_form_graph_us(lib, R, N, K, fv.GEMM_SKINNY, 0)
+            print("R=%d N=%d K=%d: picked form %.2f us | weight-streaming %.2f us  weights %.0f GB/s  %.0f TFLOP/s" % (
+                R, N, K, auto, sk, N * K * 2 / sk / 1e3, 2 * R * N * K / sk / 1e6), flush=True)
 
 
 def gemmk():
@@ -150,4 +182,4 @@ def transition():
 
 if __name__ == "__main__":
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
-    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition}[which]()
+    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition, "skinny": skinny}[which]()

@@ -116,7 +116,7 @@ def select_top_r(scores: np.ndarray, r: int) -> np.ndarray:
 
 def sampling_keys(scores: np.ndarray, noise: np.ndarray) -> np.ndarray:
     """Keys for drawing rows without replacement with probability proportional to the row score
-    (Sec. 3.3 RTR: "each row i chosen with probability P_i" proportional to ||F^(i)||^2): with
+    (Sec. 3.3 RTR, read as sampling: row i is drawn with probability proportional to ||F^(i)||^2): with
     E_i ~ Exp(1) independent, the r largest s_i / E_i are a sample without replacement in which the
     first pick is row i with probability s_i / sum_j s_j (exponential race).  The noise E is an
     input; the keys are one fp32 division each, the precision the kernel decides in."""
@@ -224,7 +224,7 @@ def upsample_bilinear(F: np.ndarray, hw_in, hw_out) -> np.ndarray:
 # --------------------------------------------------------------------------- between two scale steps
 # Algorithm 1 ("Vanilla VAR" lines, the same in both stages), Eq. "var_upf" and Eq. "var_downf":
 #   R_k = Q(F_k^o);  F_k = F_{k-1} + Up(R_k, (h_K, w_K));  next input = Down(F_k, (h_{k+1}, w_{k+1})).
-# The paper leaves Q, Up and Down abstract (Q "typically includes a codebook Z in R^{V x d}"); here
+# The paper leaves Q, Up and Down abstract (Algorithm 1 lists a codebook Z of V codewords of width d among the inputs of Q); here
 # Q is the nearest codeword in Euclidean distance (ties: lowest code), Up is upsample_bilinear above and
 # Down averages the source cells each target cell covers ("area" resampling).
 
@@ -265,7 +265,7 @@ def scale_transition(F_prev: np.ndarray, F_o: np.ndarray, Z: np.ndarray, hw_k, h
 def cfg_combine(F_prompt: np.ndarray, F_null: np.ndarray, s: float) -> np.ndarray:
     """Classifier-free guidance on the two branches of a CFG pair: F_null + s (F_prompt - F_null).  s = 0 is
     the null-prompt branch alone, which is what "setting the CFG to 0" in the fidelity-refinement stage means
-    (Sec. 3.3: "equivalent to conditioning only on the null text prompt")."""
+    (Sec. 3.3: CFG = 0 amounts to running the null text prompt alone)."""
     a, b = np.asarray(F_prompt, dtype=np.float64), np.asarray(F_null, dtype=np.float64)
     return b + s * (a - b)
 

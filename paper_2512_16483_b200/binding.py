@@ -19,9 +19,9 @@ OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
 SELECT_TOPR, SELECT_SAMPLE = 0, 1
-OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS = 0, 1
-GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR = 0, 1, 2
-KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "transpose_split", "rtr_fill", "convert")
+OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS, OPT_SKINNY_MAX_ROWS = 0, 1, 2
+GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR, GEMM_SKINNY = 0, 1, 2, 3
+KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")
 
@@ -80,7 +80,7 @@ def load_library() -> ct.CDLL:
         "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
         "fvar_scale_step": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_scale_step_host": (i, [vp, vp, i, P(_Policy), vp]),
-        "fvar_scale_step_host_async": (i, [vp, vp, i, vp, vp]),
+        "fvar_scale_step_host_async": (i, [vp, vp, i, P(_Policy), vp]),
         "fvar_host_sync": (i, [vp]),
         "fvar_kv_append": (i, [vp, i]),
         "fvar_get_indices": (i, [vp, i, vp, P(i)]),
@@ -108,6 +108,12 @@ def load_library() -> ct.CDLL:
         "fvar_attention": (i, [vp, vp, vp, i, i, i, i, i, i, vp, vp]),
         "fvar_rtr_fill": (i, [vp, i, i, i, i, i, i, vp, vp, vp]),
         "fvar_select_rows_static": (i, [vp, i, i, i, i, vp, vp, vp]),
+        "fvar_l2_prefetch": (i, [vp, ct.c_size_t, vp]),
+        "fvar_rank_from_keep_ratio": (i, [i, f]),
+        "fvar_rank_from_table_ratio": (i, [i, i, ct.c_double]),
+        "fvar_infinity_rank_ratio": (i, [i, i, P(ct.c_double)]),
+        "fvar_infinity_group_ranks": (i, [i, i, i, P(i)]),
+        "fvar_infinity_schedule": (i, [i, i, P(i), P(i), P(i)]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -122,7 +128,9 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_gemm_bf16_wt", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static")
+            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_gemm_bf16_wt", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static", "fvar_l2_prefetch",
+            "fvar_rank_from_keep_ratio", "fvar_rank_from_table_ratio", "fvar_infinity_rank_ratio", "fvar_infinity_group_ranks",
+            "fvar_infinity_schedule")
 
 
 def _stream() -> int:

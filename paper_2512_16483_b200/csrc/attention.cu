@@ -98,8 +98,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
+  pdl_launch_dependents();      // the successor (a GEMM) only requests weights before its own wait
   pdl_wait();
-  pdl_launch_dependents();
 
   if (warp == 0) {
     if (lane == 0) {

@@ -214,8 +214,8 @@ __global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__
                                                                  long long vec_stride, int bmul, int boff,
                                                                  const bf16 *__restrict__ gamma, float eps,
                                                                  bf16 *__restrict__ y) {
+  pdl_launch_dependents();      // nothing precedes the wait: the successor may start its own prologue right away
   pdl_wait();
-  pdl_launch_dependents();
   __shared__ float red[kLnThreads / 32];
   const int e = blockIdx.x / rows, j = blockIdx.x - e * rows;
   const float *xr = x + (static_cast<long long>(e * xmap.bmul + xmap.boff) * xmap.rpb + j) * C;
@@ -301,8 +301,8 @@ __global__ void __launch_bounds__(256) ln_modulate_warp_kernel(const float *__re
                                                                const float *__restrict__ scale, long long vec_stride,
                                                                int bmul, int boff, const bf16 *__restrict__ gamma, float eps,
                                                                bf16 *__restrict__ y) {
+  pdl_launch_dependents();      // nothing precedes the wait: the successor may start its own prologue right away
   pdl_wait();
-  pdl_launch_dependents();
   const int grow = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (grow >= total_rows) return;
   const int lane = threadIdx.x & 31;
@@ -567,6 +567,26 @@ __global__ void silu_bf16_kernel(const bf16 *__restrict__ in, bf16 *__restrict__
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
   return launch_pdl(silu_bf16_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, in, out, n);
+}
+
+// Asks L2 to fetch [ptr, ptr + bytes): one bulk prefetch of up to 16 KiB per thread.  The range must hold data that no
+// kernel in flight writes (weights), so the requests go out before the wait that keeps stream order transitive.
+__global__ void l2_prefetch_kernel(const uint8_t *__restrict__ ptr, unsigned long long bytes) {
+  pdl_launch_dependents();
+  const unsigned long long o = (static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x) * 16384ull;
+  if (o < bytes) {
+    const unsigned long long n = bytes - o < 16384ull ? bytes - o : 16384ull;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr + o), "r"(static_cast<uint32_t>(n)) : "memory");
+  }
+  pdl_wait();
+}
+
+cudaError_t launch_l2_prefetch(const void *ptr, unsigned long long bytes, cudaStream_t st) {
+  bytes &= ~15ull;
+  if (bytes == 0) return cudaSuccess;
+  const unsigned long long pieces = (bytes + 16383ull) / 16384ull;
+  return launch_pdl(l2_prefetch_kernel, dim3(static_cast<unsigned>((pieces + 31) / 32)), dim3(32), 0, st,
+                    static_cast<const uint8_t *>(ptr), bytes);
 }
 
 // K, V [B][L][H*D] -> cache layout K [B][H][L_cap][D], V^T [B][H][D][L_cap] (one block's worth).

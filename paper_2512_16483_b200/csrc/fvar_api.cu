@@ -61,6 +61,20 @@ bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool tmap_kblocks(CUtensorMap *m, const void *base, uint64_t rows, uint64_t kblocks, uint64_t ld_elems, uint32_t box_rows,
+                  uint32_t box_kb) {
+  if (!tmap_init_driver()) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (ld_elems * 2) % 16 || box_rows == 0 || box_rows > 256 || box_kb == 0 || box_kb > 256)
+    return false;
+  cuuint64_t dims[3] = {64, rows, kblocks};
+  cuuint64_t strides[2] = {ld_elems * 2, 128};
+  cuuint32_t box[3] = {64, box_rows, box_kb};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Status word used by the kernel-level entry points (contexts carry their own in the workspace).
 __device__ unsigned g_kernel_status;
 
@@ -136,7 +150,11 @@ struct fvar_ctx {
   std::vector<CUtensorMap> xsplit_map; // [scale][2 buffers]: rows = elements x (hi rows, lo rows), 64 x 64 boxes
   std::vector<CUtensorMap> kmap, vmap, ckmap, cvmap;   // per block
   // GEMM A operands: one map per box height (16, 32, 64, 128 rows); q_map feeds the attention kernel
-  struct ActMaps { CUtensorMap m[4]; };
+  struct ActMaps {
+    CUtensorMap m[4];
+    const bf16 *base;                  // the buffer behind the maps: [rows][cols], for maps of other box heights
+    uint64_t cols, rows;
+  };
   ActMaps y_map, a_map, h_map, silu_map;
   CUtensorMap q_map;
   // state
@@ -158,6 +176,7 @@ struct fvar_ctx {
   std::map<std::string, GraphEntry> graphs;
   bool use_graphs;
   int max_splits;                      // largest split-K factor the tile picker may use (1, 2 or 4)
+  int skinny_max_rows;                 // GEMMs of at most this many rows take the weight-streaming form (0: never)
   void drop_graphs() {
     for (auto &kv : graphs) cudaGraphExecDestroy(kv.second.exec);
     graphs.clear();
@@ -312,6 +331,27 @@ fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk
 // A operand from one of the library's activation buffers: a single row tile takes the shortest box
 // that covers its rows.
 fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int blk, int wid, GemmArgs &g, const char *what) {
+  if (g.nbatch == 1 && g.R <= ctx->skinny_max_rows && gemm_skinny_supported(epi, g.R, g.N, g.K)) {
+    // few rows: bound by streaming the weights once, so the weights take the M side of the MMA and the K range
+    // of every 128-feature tile is spread over a cluster (gemm_skinny.cu)
+    const int S = gemm_skinny_pick_splits(g.N, g.K, 0);
+    g.splits = S;
+    gemm_skinny_shape(g);
+    CUtensorMap tmA, tmW;
+    if (S > 0 && g.sk_stages >= 1 && gemm_skinny_map(&tmA, maps.base, maps.rows, maps.cols, maps.cols, g.sk_rp, g.sk_nk) &&
+        gemm_skinny_map(&tmW, ctx->w[wid][blk], g.N, g.K, g.K, 128, g.sk_nk)) {
+      g.splits = S;
+      g.status = ctx->status;
+      ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K,
+                      2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K) +
+                          (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N);
+      FV_CUDA(ctx, launch_gemm_skinny(epi, tmA, tmW, g, ctx->launch_st), what);
+      ctx->launched();
+      return FVAR_OK;
+    }
+    g.splits = 1;
+  }
+  g.pf_ptr = nullptr;
   int t = 3;
   if (g.nbatch == 1 && g.R <= 64) t = g.R <= 16 ? 0 : (g.R <= 32 ? 1 : 2);
   g.a_box_rows = 16 << t;
@@ -467,6 +507,10 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
       for (int t = 0; t < 3 && ok; ++t)
         ok = tmap_2d(&c->wmap[(b * W_COUNT + i) * 3 + t], c->w[i][b], w_cols[i], w_rows[i], w_cols[i], kBNs[t]);
   const size_t act_rows = static_cast<size_t>(c->Bmax) * c->Mmax;
+  c->y_map.base = c->y; c->y_map.cols = C; c->y_map.rows = act_rows;
+  c->a_map.base = c->a; c->a_map.cols = C; c->a_map.rows = act_rows;
+  c->h_map.base = c->hbuf; c->h_map.cols = F; c->h_map.rows = act_rows;
+  c->silu_map.base = c->silu_c; c->silu_map.cols = C; c->silu_map.rows = c->Bmax;
   for (int t = 0; t < 4 && ok; ++t) {
     const uint32_t box = 16u << t;
     ok = tmap_2d(&c->y_map.m[t], c->y, C, act_rows, C, box) && tmap_2d(&c->a_map.m[t], c->a, C, act_rows, C, box) &&
@@ -500,6 +544,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
   c->max_splits = 1;
+  c->skinny_max_rows = 64;
   c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
@@ -510,7 +555,8 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
     c->host_pipe_ok = cudaEventCreateWithFlags(&c->ev_in[s2], cudaEventDisableTiming) == cudaSuccess &&
                       cudaEventCreateWithFlags(&c->ev_cmp[s2], cudaEventDisableTiming) == cudaSuccess &&
                       cudaEventCreateWithFlags(&c->ev_out[s2], cudaEventDisableTiming) == cudaSuccess;
-  if (gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || attention_prepare() != cudaSuccess)
+  if (gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || gemm_skinny_prepare() != cudaSuccess ||
+      attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   c->max_clusters = gemm_pair_max_clusters();
   *out = c;
@@ -555,6 +601,13 @@ fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value) {
     FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
     ctx->drop_graphs();
     ctx->max_splits = value;
+    return FVAR_OK;
+  }
+  if (option == FVAR_OPT_SKINNY_MAX_ROWS) {
+    if (value < 0 || value > 512) return fail(ctx, FVAR_EINVAL, "set_option: skinny rows must be in [0, 512]");
+    FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+    ctx->drop_graphs();
+    ctx->skinny_max_rows = value;
     return FVAR_OK;
   }
   return fail(ctx, FVAR_EINVAL, "set_option: unknown option");
@@ -857,8 +910,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   std::vector<int> rank(G, M);
   if (pol->mode == FVAR_LOWRANK_RTR) {
     for (int g = 0; g < G; ++g) {
-      int r = pol->rank_per_group ? pol->rank_per_group[g] : static_cast<int>(floorf(pol->keep_ratio * M + 0.5f));
-      if (!pol->rank_per_group) r = r < 1 ? 1 : (r > M ? M : r);
+      const int r = pol->rank_per_group ? pol->rank_per_group[g] : fvar_rank_from_keep_ratio(M, pol->keep_ratio);
       if (r < 1 || r > M) return fail(ctx, FVAR_EINVAL, "scale_step: need 1 <= r <= M");
       rank[g] = r;
     }
@@ -965,6 +1017,11 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       const RowMap in_map = first_dense ? bmap : smap;
       const float *ada = ctx->ada + blk * ada_blk;
       const int L_prev = ctx->len[blk];
+      // the weights each GEMM's successor will stream (gemm_skinny.cu asks L2 for them ahead of time)
+      const size_t w_bytes[W_COUNT] = {6ull * C * C, 2ull * C * C, 2ull * F * C, 2ull * C * F, 0, 2ull * C * C, 0, 2ull * C * C};
+      auto prefetch_next = [&](GemmArgs &ga, int next_blk, int next_wid) {
+        if (next_blk < ctx->cfg.n_blocks) { ga.pf_ptr = ctx->w[next_wid][next_blk]; ga.pf_bytes = w_bytes[next_wid]; }
+      };
 
       ctx->prof_begin(FVAR_KCLASS_LN, 0.0, 6.0 * R * C);
       FV_CUDA(ctx, launch_ln_modulate(in_ptr, in_map, E, r, C, ada, ada + C, 6 * C, bmul, boff, nullptr,
@@ -978,6 +1035,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         ga.kc = ctx->kc + blk * ctx->kv_block_elems();
         ga.vt = ctx->vt + blk * ctx->kv_block_elems();
         ga.C = C; ga.H = H; ga.D = D; ga.L_cap = ctx->L_cap; ga.L_prev = L_prev; ga.col_base = 0;
+        prefetch_next(ga, blk, W_O);
         if ((s = run_gemm(ctx, EPI_QKV, ctx->y_map, blk, W_QKV, ga, "qkv gemm")) != FVAR_OK) return s;
       }
       {
@@ -995,6 +1053,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         ga.resid = in_ptr; ga.rmap = in_map;
         ga.out_f32 = ctx->xs; ga.omap = smap; ga.ld_out = C;
         ga.gate = ada + 2 * C; ga.gate_stride = 6 * C;
+        prefetch_next(ga, blk, ctx->cfg.has_cross_attn ? W_CQ : W_FC1);
         if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_O, ga, "out-proj gemm")) != FVAR_OK) return s;
       }
       if (ctx->cfg.has_cross_attn) {
@@ -1004,6 +1063,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         ctx->launched();
         GemmArgs gq = gemm_args(R, C, C);
         gq.out_bf16 = ctx->q; gq.ld_out = C;
+        prefetch_next(gq, blk, W_CO);
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
         AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, nullptr, nullptr};
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
@@ -1012,6 +1072,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         GemmArgs go = gemm_args(R, C, C);
         go.rows_per_batch = r; go.bmul = bmul; go.boff = boff;
         go.resid = ctx->xs; go.rmap = smap; go.out_f32 = ctx->xs; go.omap = smap; go.ld_out = C;
+        prefetch_next(go, blk, W_FC1);
         if ((s = run_gemm(ctx, EPI_RESID, ctx->a_map, blk, W_CO, go, "cross out gemm")) != FVAR_OK) return s;
       }
       ctx->prof_begin(FVAR_KCLASS_LN, 0.0, 6.0 * R * C);
@@ -1022,6 +1083,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         GemmArgs ga = gemm_args(R, F, C);
         ga.bias = ctx->b_fc1[blk];
         ga.out_bf16 = ctx->hbuf; ga.ld_out = F;
+        prefetch_next(ga, blk, W_FC2);
         if ((s = run_gemm(ctx, EPI_GELU_BF16, ctx->y_map, blk, W_FC1, ga, "fc1 gemm")) != FVAR_OK) return s;
       }
       {
@@ -1038,6 +1100,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         } else {
           ga.out_f32 = ctx->xs; ga.omap = smap;
         }
+        prefetch_next(ga, blk + 1, W_QKV);
         if ((s = run_gemm(ctx, EPI_RESID, ctx->h_map, blk, W_FC2, ga, "fc2 gemm")) != FVAR_OK) return s;
       }
       ctx->staged[blk] = r;
@@ -1263,7 +1326,28 @@ fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, c
 fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
                                 int block_n, float *out, void *stream) {
   if (!A || !W || !out || R <= 0 || N <= 0 || K <= 0 || K % 8) return kfail(FVAR_EINVAL, "gemm: bad arguments");
-  if (form != FVAR_GEMM_AUTO && form != FVAR_GEMM_SINGLE && form != FVAR_GEMM_PAIR) return kfail(FVAR_EINVAL, "gemm: bad form");
+  if (form != FVAR_GEMM_AUTO && form != FVAR_GEMM_SINGLE && form != FVAR_GEMM_PAIR && form != FVAR_GEMM_SKINNY)
+    return kfail(FVAR_EINVAL, "gemm: bad form");
+  if (form == FVAR_GEMM_SKINNY) {
+    if (!gemm_skinny_supported(EPI_F32, R, N, K)) return kfail(FVAR_EINVAL, "gemm: the weight-streaming form needs R <= 512, N % 8 == 0");
+    if (block_n < 0 || block_n > 8) return kfail(FVAR_EINVAL, "gemm: the weight-streaming form takes 0 .. 8 K ranges");
+    const int S = gemm_skinny_pick_splits(N, K, block_n);
+    if (S <= 0) return kfail(FVAR_EINVAL, "gemm: this number of K ranges is not launchable for the problem");
+    GemmArgs g = gemm_args(R, N, K);
+    g.splits = S;
+    gemm_skinny_shape(g);
+    CUtensorMap ta, tw;
+    if (g.sk_stages < 1 || !gemm_skinny_map(&ta, A, R, K, K, g.sk_rp, g.sk_nk) || !gemm_skinny_map(&tw, W, N, K, K, 128, g.sk_nk))
+      return kfail(FVAR_EINVAL, "gemm: operands must be 16-byte aligned");
+    g.bias = static_cast<const bf16 *>(bias);
+    g.out_f32 = out;
+    g.ld_out = N;
+    g.splits = S;
+    g.status = kernel_status_ptr();
+    if (!g.status) return kfail(FVAR_ECUDA, "gemm: status word");
+    FK_CUDA(launch_gemm_skinny(EPI_F32, ta, tw, g, static_cast<cudaStream_t>(stream)), "gemm");
+    return FVAR_OK;
+  }
   int dev = 0, sms = 0;
   FK_CUDA(cudaGetDevice(&dev), "get device");
   FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
@@ -1344,6 +1428,12 @@ fvar_status fvar_cfg_combine(const void *pair, int B, long long per_elem, float 
     return kfail(FVAR_EINVAL, "cfg_combine: bad arguments");
   FK_CUDA(launch_cfg_combine(static_cast<const bf16 *>(pair), B / 2, per_elem, guidance, static_cast<bf16 *>(out),
                              static_cast<cudaStream_t>(stream)), "cfg_combine");
+  return FVAR_OK;
+}
+
+fvar_status fvar_l2_prefetch(const void *ptr, size_t bytes, void *stream) {
+  if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 15)) return kfail(FVAR_EINVAL, "l2_prefetch: NULL or unaligned pointer");
+  FK_CUDA(launch_l2_prefetch(ptr, bytes, static_cast<cudaStream_t>(stream)), "l2_prefetch");
   return FVAR_OK;
 }
 

@@ -57,12 +57,22 @@ struct GemmArgs {
   float *partial;
   int *counters;
   unsigned *status;
+  // Weight-streaming form (gemm_skinny.cu; `splits` is then the cluster size): rows per column chunk, the padded
+  // MMA width of a chunk, chunks (1 or 2) and pipeline stages -- filled by gemm_skinny_shape
+  int sk_rows_chunk, sk_rp, sk_nchunks, sk_stages, sk_small, sk_nk;
+  // optional: weights the next GEMM of the chain will stream; every CTA asks L2 to prefetch its share
+  const void *pf_ptr;
+  unsigned long long pf_bytes;
 };
 
 // Tensor maps: bf16, 2-D {cols, rows} with a {64, box_rows} box and 128-byte swizzle, or the 3-D
 // forms used for the KV cache.
 bool tmap_init_driver();
 bool tmap_2d(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t ld_elems, uint32_t box_rows);
+// {64 K elements, rows, K blocks} view of a K-major [rows][64 * kblocks] matrix (row pitch ld_elems): a box
+// {64, box_rows, box_kb} lands as box_kb consecutive swizzled [box_rows][64] tiles.
+bool tmap_kblocks(CUtensorMap *m, const void *base, uint64_t rows, uint64_t kblocks, uint64_t ld_elems, uint32_t box_rows,
+                  uint32_t box_kb);
 bool tmap_3d(CUtensorMap *m, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t ld1_elems,
              uint64_t ld2_elems, uint32_t box0, uint32_t box1);
 
@@ -88,6 +98,16 @@ struct GemmPlan {
 // Picks the launch form and tile width from the measured cost model.  tiles_m_total: 128-row tiles over
 // all batches; pairs are considered only for a single problem with more than one row tile.
 GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_clusters, int max_splits, size_t scratch_bytes);
+
+// Weight-streaming form for R <= 512 rows (gemm_skinny.cu): the weights are the M side of the MMA, the K range of
+// a 128-feature tile is split over a cluster of `splits` CTAs that reduce through distributed shared memory.
+// tmA: box {64, a.sk_rp} over the activation rows; tmW: box {64, 128} over the weight rows.
+bool gemm_skinny_supported(int epi, int R, int N, int K);
+int gemm_skinny_pick_splits(int N, int K, int forced);      // 0: not launchable on this device
+void gemm_skinny_shape(GemmArgs &a);      // needs a.R, a.K and a.splits
+bool gemm_skinny_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows, int nk);
+cudaError_t launch_gemm_skinny(int epi, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, cudaStream_t st);
+cudaError_t gemm_skinny_prepare();
 
 // Set the dynamic shared-memory attribute of every instantiation (once, outside any stream capture).
 cudaError_t gemm_prepare();
@@ -158,6 +178,7 @@ cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0,
                                  bool overwrite, float *F, cudaStream_t st);
 cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st);
 cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st);
+cudaError_t launch_l2_prefetch(const void *ptr, unsigned long long bytes, cudaStream_t st);
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
 cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,
                            cudaStream_t st);

@@ -32,9 +32,13 @@ __device__ __forceinline__ bool elect_one() {
 // scheduled while the previous kernel on the stream is still draining, so that launch latency and
 // the prologue (barrier init, TMEM allocation, descriptor prefetch) overlap the predecessor's tail.
 // pdl_wait() blocks until the predecessor grid has completed and its writes are visible; nothing
-// that reads or overwrites global memory may precede it.  pdl_launch_dependents() then lets the
-// successor begin its own prologue.  Because every kernel waits before it releases its successor,
-// at most two grids are in flight and completion order is transitive along the stream.
+// that reads or overwrites memory another kernel writes may precede it (weights, which no kernel
+// writes, may be requested earlier).  pdl_launch_dependents() lets the successor be scheduled and run
+// up to its own wait.  The tensor-core GEMMs release their successor only after their own wait; the
+// LayerNorm and attention kernels, whose successors do nothing but set up and request weights before
+// waiting, release it at once.  Completion order stays transitive along the stream (every kernel waits
+// for its predecessor, which waited for its own), and a grid is only launched once every CTA of its
+// predecessor is running, so a waiting successor never keeps a predecessor's CTA off an SM.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

@@ -1,72 +1,69 @@
-"""Host-side schedule of the method: which scale steps run densely, which run under the
-fidelity-refinement approximation and which are skipped, and the rank r of every block group.
+"""The method's schedule, as the C ABI exports it (include/fvar.h, "The method's schedule"): which scale
+steps run densely, which run under the fidelity-refinement approximation and which are skipped
+(Sec. 4.1), and the rank r of every block group (App. A.1; Sec. 3.2, Eq. "low_rank_percent").
 
-Sec. 4.1: the Infinity schedule keeps scales {1, ..., 32} dense and applies the approximation at
-{40, 48, 64} with thresholds alpha = {0.96, 0, 0}; alpha = 0 skips the step.  App. A.1 tabulates,
-for alpha = 0.96, the mean rank ratio of every block chunk at each late scale; a ratio is a
-fraction of n = min(M, d) (Sec. 3.2, Eq. "low_rank_percent").
+Argument marshalling only: the table, the thresholds and the rounding live in the library
+(csrc/schedule.cu).  These calls need no GPU.
 """
 from __future__ import annotations
 
-import math
-from typing import List, Sequence
+import ctypes as ct
+from typing import List, Sequence, Tuple
 
-DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
+from . import binding
 
-INFINITY_SCALES = (1, 2, 4, 6, 8, 12, 16, 20, 24, 32, 40, 48, 64)
+DENSE, LOWRANK_RTR, SKIP = binding.DENSE, binding.LOWRANK_RTR, binding.SKIP
 INFINITY_LATE_SCALES = (40, 48, 64)
-INFINITY_ALPHA = (0.96, 0.0, 0.0)
 
-# rows: block chunk 0..7, columns: scale 40, 48, 64 (alpha = 0.96)
-RANK_RATIO_ALPHA_096 = (
-    (0.016, 0.013, 0.008),
-    (0.136, 0.117, 0.054),
-    (0.210, 0.189, 0.083),
-    (0.250, 0.222, 0.066),
-    (0.256, 0.234, 0.056),
-    (0.198, 0.183, 0.029),
-    (0.157, 0.134, 0.038),
-    (0.191, 0.163, 0.055),
-)
+
+def _check(status: int, what: str) -> None:
+    if status != binding.OK:
+        raise binding.FvarError(status, what)
 
 
 def rank_from_keep_ratio(M: int, rho: float) -> int:
-    return max(1, min(M, int(math.floor(rho * M + 0.5))))
+    return int(binding.load_library().fvar_rank_from_keep_ratio(int(M), float(rho)))
 
 
 def rank_from_table_ratio(M: int, width: int, ratio: float) -> int:
-    n = min(M, width)
-    return max(1, min(M, int(math.floor(ratio * n + 0.5))))
+    return int(binding.load_library().fvar_rank_from_table_ratio(int(M), int(width), float(ratio)))
+
+
+def rank_ratio_table() -> Tuple[Tuple[float, ...], ...]:
+    """App. A.1 (alpha = 0.96): rows = block chunk 0..7, columns = scale 40, 48, 64."""
+    lib = binding.load_library()
+    rows = []
+    for chunk in range(8):
+        row = []
+        for side in INFINITY_LATE_SCALES:
+            v = ct.c_double()
+            _check(lib.fvar_infinity_rank_ratio(chunk, side, ct.byref(v)), "infinity_rank_ratio")
+            row.append(v.value)
+        rows.append(tuple(row))
+    return tuple(rows)
 
 
 def infinity_group_ranks(scale_side: int, width: int = 2048, n_groups: int = 8) -> List[int]:
-    """Rank per block group at a late Infinity scale (40, 48 or 64); groups other than 8 take the
-    ratio of the chunk at the nearest relative depth."""
-    col = INFINITY_LATE_SCALES.index(scale_side)
-    M = scale_side * scale_side
-    out = []
-    for g in range(n_groups):
-        chunk = min(7, int((g + 0.5) * 8 / n_groups))
-        out.append(rank_from_table_ratio(M, width, RANK_RATIO_ALPHA_096[chunk][col]))
-    return out
+    out = (ct.c_int * n_groups)()
+    _check(binding.load_library().fvar_infinity_group_ranks(int(scale_side), int(width), int(n_groups), out),
+           "infinity_group_ranks(%d)" % scale_side)
+    return list(out)
+
+
+def infinity_schedule(paper_schedule: bool = True) -> Tuple[List[int], List[int]]:
+    """(side length, mode) per scale step of the 13-step Infinity schedule."""
+    sides, modes, n = (ct.c_int * 16)(), (ct.c_int * 16)(), ct.c_int()
+    _check(binding.load_library().fvar_infinity_schedule(int(bool(paper_schedule)), 16, sides, modes, ct.byref(n)),
+           "infinity_schedule")
+    return list(sides[:n.value]), list(modes[:n.value])
 
 
 def infinity_stage_modes(paper_schedule: bool = True) -> List[int]:
-    """Mode per scale step of the 13-step Infinity schedule.  paper_schedule: alpha = {0.96, 0, 0},
-    i.e. scale 40 approximated and 48, 64 skipped; otherwise all three late scales approximated."""
-    modes = []
-    for s in INFINITY_SCALES:
-        if s not in INFINITY_LATE_SCALES:
-            modes.append(DENSE)
-        elif not paper_schedule or INFINITY_ALPHA[INFINITY_LATE_SCALES.index(s)] > 0:
-            modes.append(LOWRANK_RTR)
-        else:
-            modes.append(SKIP)
-    return modes
+    return infinity_schedule(paper_schedule)[1]
 
 
 def cache_rows(scales: Sequence[int]) -> List[int]:
-    """KV-cache length after each scale of a square schedule."""
+    """KV-cache length after each scale of a square schedule (prefix sums of side^2)."""
     acc, out = 0, []
     for s in scales:
         acc += s * s

@@ -1,6 +1,6 @@
 """Last-scale sweep on the Infinity-2B shape (one GPU): rows kept x batch, against the dense path.
 
-    python -m paper_2512_16483_b200.sweep [--steps K] [--ranks 4096,3072,...] [--batches 2,4,8,16]
+    python sweep.py [--steps K] [--ranks 4096,3072,...] [--batches 2,4,8,16]
 
 Every point is one run of `bench.py --workload infinity2b_last_r<R>_b<B>` in a process of its own (the
 KV cache and the workspace are sized by the batch): the 64 x 64 scale, 4096 query tokens per element over a
@@ -19,7 +19,7 @@ import os
 import subprocess
 import sys
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 
 
 def run_point(R: int, B: int, steps: int):

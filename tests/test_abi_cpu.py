@@ -1,5 +1,5 @@
 """CPU-side checks of the boundary: the library builds, loads and exports every symbol the public
-header declares; the host-side schedule agrees with the printed table.  No compute calls."""
+header declares; the schedule the library exports agrees with the printed table.  No compute calls."""
 import os
 import re
 
@@ -55,13 +55,16 @@ def test_schedule_matches_printed_table():
         for line in f:
             if line.strip() and not line.startswith("#"):
                 rows.append(tuple(float(v) for v in line.split()))
-    assert tuple(rows) == schedule.RANK_RATIO_ALPHA_096
+    assert tuple(rows) == schedule.rank_ratio_table()
     assert schedule.infinity_group_ranks(40) == [26, 218, 336, 400, 410, 317, 251, 306]
     assert schedule.infinity_group_ranks(64) == [16, 111, 170, 135, 115, 59, 78, 113]
     assert schedule.infinity_stage_modes(True) == [0] * 10 + [1, 2, 2]
     assert schedule.infinity_stage_modes(False) == [0] * 10 + [1, 1, 1]
     assert schedule.cache_rows(si.INFINITY_SCALES)[-1] == 10521 and schedule.cache_rows(si.VAR_SCALES)[-1] == 680
-    assert schedule.rank_from_keep_ratio(169, 0.5) == 85
+    assert schedule.rank_from_keep_ratio(169, 0.5) == 85 and schedule.rank_from_keep_ratio(100, 0.001) == 1
+    assert schedule.infinity_schedule(True)[0] == list(si.INFINITY_SCALES)
+    assert schedule.rank_from_table_ratio(1600, 2048, 0.016) == 26 and schedule.rank_from_table_ratio(4096, 2048, 0.083) == 170
+    assert schedule.infinity_group_ranks(48, 2048, 4) == [schedule.infinity_group_ranks(48)[c] for c in (1, 3, 5, 7)]
 
 
 def test_bf16_rounding_of_the_input_generator():

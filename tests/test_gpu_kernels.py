@@ -125,6 +125,31 @@ def test_gemm_bf16_every_form(fv, R, N, K, form, block_n):
     np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
 
 
+# The weight-streaming form (few rows; the weights are the M side of the MMA and the K range of a 128-feature tile is
+# spread over a cluster of S CTAs that reduce through distributed shared memory): one and two column chunks (R <= 256,
+# R > 256), every cluster size, ragged rows, a ragged last feature tile, a ragged last K block, more K ranges than
+# some sizes divide evenly, and the shapes of the Infinity-2B-shaped late steps.
+@pytest.mark.parametrize("R,N,K", [(1, 128, 64), (16, 256, 512), (17, 200, 136), (170, 2048, 2048), (256, 384, 1024),
+                                   (257, 128, 520), (410, 1024, 2048), (512, 256, 256), (50, 6144, 2048), (111, 2048, 8192),
+                                   (336, 8192, 2048)])
+@pytest.mark.parametrize("splits", [0, 1, 2, 3, 4, 5, 6, 7, 8])
+def test_gemm_bf16_weight_streaming_form(fv, R, N, K, splits):
+    rng = np.random.default_rng(11 * R + N + K)
+    A = si.normal_bf16(rng, (R, K))
+    W = si.normal_bf16(rng, (N, K), 0.05)
+    b = si.normal_bf16(rng, (N,))
+    num_kb = -(-K // 64)
+    if splits and -(-num_kb // -(-num_kb // splits)) != splits:
+        with pytest.raises(fv.FvarError):          # a K range would be empty: refused, not launched
+            fv.fvar_gemm_bf16_form(to_bf16_cuda(A), to_bf16_cuda(W), to_bf16_cuda(b), fv.GEMM_SKINNY, splits)
+        return
+    got = fv.fvar_gemm_bf16_form(to_bf16_cuda(A), to_bf16_cuda(W), to_bf16_cuda(b), fv.GEMM_SKINNY, splits).cpu().numpy()
+    _poll(fv)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T + b.astype(np.float64)
+    tol = 1e-5 * (np.abs(A).astype(np.float64) @ np.abs(W).astype(np.float64).T).max() + 1e-6
+    np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
+
+
 @pytest.mark.parametrize("R,N,K", [(128, 64, 64), (300, 200, 136), (1000, 1024, 512), (130, 1920, 344), (64, 2048, 8192)])
 @pytest.mark.parametrize("block_n", [0, 64, 128, 256])
 def test_gemm_bf16_second_operand_transposed(fv, R, N, K, block_n):
