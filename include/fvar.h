@@ -224,8 +224,10 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx);
  * FVAR_OPT_SKINNY_MAX_ROWS (default 64; 0 .. 512): GEMMs of a step with at most this many rows
  * R = B_eff * r take the weight-streaming form (the weights are the M side of the MMA, the K range of a
  * 128-feature tile is spread over a thread-block cluster that reduces through distributed shared memory),
- * which is bound by reading the weights once; 0 never uses it. */
-enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1, FVAR_OPT_SKINNY_MAX_ROWS = 2 };
+ * which is bound by reading the weights once; 0 never uses it.
+ * FVAR_OPT_WAIT_KCYCLES (default 0 = about half a second): budget, in thousands of clock cycles, of every
+ * bounded wait inside the step's kernels; a wait that runs out sets FVAR_ETIMEOUT (fvar_poll_status). */
+enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1, FVAR_OPT_SKINNY_MAX_ROWS = 2, FVAR_OPT_WAIT_KCYCLES = 3 };
 fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value);
 
 /* Measurement aid: while enabled, every kernel launch of this context is bracketed by CUDA events on
@@ -248,7 +250,9 @@ int fvar_cache_len(const fvar_ctx *ctx, int block);
 long long fvar_launch_count(const fvar_ctx *ctx);
 
 /* Synchronises the stream, reads the device status word and clears it.  FVAR_OK, FVAR_ETIMEOUT,
- * or FVAR_ECUDA. */
+ * FVAR_EINVAL (bad forced_indices) or FVAR_ECUDA.  After a timeout the results of the steps since the last
+ * poll are invalid; the library clears its reduction counters and drops its captured graphs, and the context
+ * can be used again.  ctx == NULL polls the status word of the kernel-level entry points on the current device. */
 fvar_status fvar_poll_status(fvar_ctx *ctx);
 
 /* Empties the KV cache and the group caches (host state only; device memory is not cleared). */
@@ -343,6 +347,12 @@ fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, 
  * transposed); out dev bf16 [B][r][H*D].  D in {64, 128}; L_cap % 8 == 0; 1 <= L <= L_cap. */
 fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B, int H, int r, int D, int L,
                            int L_cap, void *out, void *stream);
+
+/* Failure-detection self-test: launches one CTA that waits, with a budget of `cycles` clock cycles, on a
+ * barrier nothing ever signals.  The wait gives up, the kernel records FVAR_ETIMEOUT in the status word and
+ * returns; nothing faults or hangs.  The next fvar_poll_status(ctx) returns FVAR_ETIMEOUT, the one after
+ * FVAR_OK.  ctx == NULL uses the kernel-level status word and `stream`.  The paper has no counterpart. */
+fvar_status fvar_selftest_wait_timeout(fvar_ctx *ctx, long long cycles, void *stream);
 
 /* Asks the L2 cache to fetch [ptr, ptr + bytes) (ptr dev, 16-byte aligned; bytes rounded down to a multiple of
  * 16): a hint for data a later kernel will stream, e.g. the weights of the next layer while the current one

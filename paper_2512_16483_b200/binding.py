@@ -19,7 +19,7 @@ OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
 SELECT_TOPR, SELECT_SAMPLE = 0, 1
-OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS, OPT_SKINNY_MAX_ROWS = 0, 1, 2
+OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS, OPT_SKINNY_MAX_ROWS, OPT_WAIT_KCYCLES = 0, 1, 2, 3
 GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR, GEMM_SKINNY = 0, 1, 2, 3
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
@@ -109,6 +109,7 @@ def load_library() -> ct.CDLL:
         "fvar_rtr_fill": (i, [vp, i, i, i, i, i, i, vp, vp, vp]),
         "fvar_select_rows_static": (i, [vp, i, i, i, i, vp, vp, vp]),
         "fvar_l2_prefetch": (i, [vp, ct.c_size_t, vp]),
+        "fvar_selftest_wait_timeout": (i, [vp, ll, vp]),
         "fvar_rank_from_keep_ratio": (i, [i, f]),
         "fvar_rank_from_table_ratio": (i, [i, i, ct.c_double]),
         "fvar_infinity_rank_ratio": (i, [i, i, P(ct.c_double)]),
@@ -128,7 +129,7 @@ EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_proj
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
             "fvar_row_scores", "fvar_row_keys", "fvar_select_topr", "fvar_ln_modulate",
-            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_gemm_bf16_wt", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static", "fvar_l2_prefetch",
+            "fvar_gemm_bf16", "fvar_gemm_bf16_form", "fvar_gemm_bf16_wt", "fvar_cfg_combine", "fvar_attention", "fvar_rtr_fill", "fvar_select_rows_static", "fvar_l2_prefetch", "fvar_selftest_wait_timeout",
             "fvar_rank_from_keep_ratio", "fvar_rank_from_table_ratio", "fvar_infinity_rank_ratio", "fvar_infinity_group_ranks",
             "fvar_infinity_schedule")
 
@@ -446,6 +447,10 @@ class Fvar:
 
     def poll_status(self) -> int:
         return self.lib.fvar_poll_status(self.ctx)
+
+    def selftest_wait_timeout(self, cycles: int):
+        """Launches the one-CTA kernel whose bounded wait runs out after `cycles` clock cycles."""
+        self._check(self.lib.fvar_selftest_wait_timeout(self.ctx, int(cycles), None))
 
     def reset(self):
         self._check(self.lib.fvar_reset(self.ctx))

@@ -61,6 +61,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   auto o_full = [&](int t) { return bar_base + 8u * (5 + 2 * NR + t); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wb = wait_budget(p.wait_cycles);
   // Split-KV: kv_splits CTAs share one query tile pair, each covering a contiguous range of key
   // blocks; their unnormalised results are merged by whichever of them finishes last.
   const int splits = p.kv_splits > 1 ? p.kv_splits : 1;
@@ -115,7 +116,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int i = 0; i < 2 * nkv; ++i) {            // even i: K of block i/2, odd i: V^T of block i/2
         const int slot = i % NR, j = i >> 1;
         const uint32_t phase = (i / NR) & 1u;
-        if (!mbar_wait(ring_empty(slot), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+        if (!mbar_wait(ring_empty(slot), phase ^ 1u, p.status, &abort_flag, wb)) { ok = false; break; }
         mbar_expect_tx(ring_full(slot), Cfg::kTileBytes);
         const uint32_t dst = ring_smem + slot * Cfg::kTileBytes;
         if ((i & 1) == 0) {
@@ -163,8 +164,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         umma_commit(o_full(t));
       };
-      bool ok = mbar_wait(q_full, 0, p.status, &abort_flag);
-      if (ok) ok = mbar_wait(ring_full(0), 0, p.status, &abort_flag);
+      bool ok = mbar_wait(q_full, 0, p.status, &abort_flag, wb);
+      if (ok) ok = mbar_wait(ring_full(0), 0, p.status, &abort_flag, wb);
       if (ok) {
         tc_fence_after();
         for (int t = 0; t < ntiles; ++t) issue_s(t, t, 0);
@@ -176,13 +177,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         for (int j = 0; ok && j < nkv; ++j) {
           const int vi = 2 * j + 1, ki = 2 * j + 2;
           if (j + 1 < nkv) {
-            if (!mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+            if (!mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
             tc_fence_after();
             issue_s(0, (j + 1) & 1, ki % NR);
             umma_commit(ring_empty(ki % NR));
           }
-          if (!mbar_wait(p_full(0), j & 1u, p.status, &abort_flag)) { ok = false; break; }
-          if (!mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+          if (!mbar_wait(p_full(0), j & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
+          if (!mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
           tc_fence_after();
           issue_pv(0, j & 1, vi % NR, j > 0);
           umma_commit(ring_empty(vi % NR));
@@ -191,13 +192,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int j = 0; ok && j < nkv; ++j) {
         const int vi = 2 * j + 1, ki = 2 * j + 2;
         for (int t = 0; ok && t < ntiles; ++t) {
-          if (!mbar_wait(p_full(t), j & 1u, p.status, &abort_flag)) { ok = false; break; }
-          if (t == 0 && !mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+          if (!mbar_wait(p_full(t), j & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
+          if (t == 0 && !mbar_wait(ring_full(vi % NR), (vi / NR) & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
           tc_fence_after();
           issue_pv(t, t, vi % NR, j > 0);
           if (t == ntiles - 1) umma_commit(ring_empty(vi % NR));
           if (j + 1 < nkv) {
-            if (t == 0 && !mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag)) { ok = false; break; }
+            if (t == 0 && !mbar_wait(ring_full(ki % NR), (ki / NR) & 1u, p.status, &abort_flag, wb)) { ok = false; break; }
             tc_fence_after();
             issue_s(t, t, ki % NR);
             if (t == ntiles - 1) umma_commit(ring_empty(ki % NR));
@@ -222,7 +223,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       for (int j = 0; j < nkv; ++j) {
         const int sbuf = single ? (j & 1) : t;
         const uint32_t s_addr = s_base + sbuf * kKeys;
-        ok = __all_sync(0xffffffffu, mbar_wait(s_full(sbuf), (single ? (j >> 1) : j) & 1u, p.status, &abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(s_full(sbuf), (single ? (j >> 1) : j) & 1u, p.status, &abort_flag, wb));
         if (!ok) break;
         tc_fence_after();
         const int valid = p.L - (jb0 + j) * kKeys;       // keys of this block below L (>= 128: all)
@@ -248,7 +249,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const bool need = (m_cand - m_ref) * c > kRescaleThreshold;      // true on the first block (m_ref = -inf)
         if (j > 0) {
           // P V of block j-1 must be complete before P's buffer is overwritten or O is touched
-          ok = __all_sync(0xffffffffu, mbar_wait(o_full(t), (j - 1) & 1u, p.status, &abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(o_full(t), (j - 1) & 1u, p.status, &abort_flag, wb));
           if (!ok) break;
           tc_fence_after();
         }
@@ -295,7 +296,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tc_fence_before();
         mbar_arrive(p_full(t));
       }
-      if (ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag))) {
+      if (ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag, wb))) {
         tc_fence_after();
         const int rib = qt * 2 * kQRows + t * kQRows + row_local;
         bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;

@@ -569,6 +569,26 @@ cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_
   return launch_pdl(silu_bf16_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, in, out, n);
 }
 
+// Self-test of the bounded wait every kernel of the library relies on: one thread initialises an mbarrier that
+// nothing will ever signal and waits on it with the given budget.  The wait gives up, flags the status word
+// (kStatusTimeout) and the kernel returns normally: no trap, no fault, the context stays usable.
+__global__ void wait_selftest_kernel(long long cycles, unsigned *status) {
+  __shared__ unsigned long long bar;
+  __shared__ volatile int abort_flag;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+    mbar_wait(smem_u32(&bar), 0, status, &abort_flag, wait_budget(cycles));
+  }
+}
+
+cudaError_t launch_wait_selftest(long long cycles, unsigned *status, cudaStream_t st) {
+  return launch_pdl(wait_selftest_kernel, dim3(1), dim3(32), 0, st, cycles, status);
+}
+
 // Asks L2 to fetch [ptr, ptr + bytes): one bulk prefetch of up to 16 KiB per thread.  The range must hold data that no
 // kernel in flight writes (weights), so the requests go out before the wait that keeps stream order transitive.
 __global__ void l2_prefetch_kernel(const uint8_t *__restrict__ ptr, unsigned long long bytes) {

@@ -7,6 +7,7 @@
 
 #include <algorithm>
 #include <map>
+#include <mutex>
 
 #include <string>
 #include <vector>
@@ -80,13 +81,19 @@ __device__ unsigned g_kernel_status;
 
 static std::string g_init_error;
 
-bool pdl_enabled() {
-  static int v = -1;
-  if (v < 0) {
-    const char *e = getenv("FVAR_NO_PDL");
-    v = (e && e[0] == '1') ? 0 : 1;
+// Address of the status word on the current device (resolved once per device ordinal).
+static unsigned *kernel_status_ptr() {
+  static std::mutex mu;
+  static unsigned *cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cache[dev]) {
+    void *addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_kernel_status) != cudaSuccess) return nullptr;
+    cache[dev] = static_cast<unsigned *>(addr);
   }
-  return v != 0;
+  return cache[dev];
 }
 
 void set_global_error(const char *msg) { g_init_error = msg ? msg : ""; }
@@ -176,6 +183,7 @@ struct fvar_ctx {
   std::map<std::string, GraphEntry> graphs;
   bool use_graphs;
   int max_splits;                      // largest split-K factor the tile picker may use (1, 2 or 4)
+  long long wait_cycles;               // budget of the kernels' bounded waits (0: default)
   int skinny_max_rows;                 // GEMMs of at most this many rows take the weight-streaming form (0: never)
   void drop_graphs() {
     for (auto &kv : graphs) cudaGraphExecDestroy(kv.second.exec);
@@ -342,6 +350,7 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int 
         gemm_skinny_map(&tmW, ctx->w[wid][blk], g.N, g.K, g.K, 128, g.sk_nk)) {
       g.splits = S;
       g.status = ctx->status;
+      g.wait_cycles = ctx->wait_cycles;
       ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K,
                       2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K) +
                           (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N);
@@ -367,6 +376,7 @@ fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk
   g.partial = ctx->split_partial;
   g.counters = ctx->split_counters;
   g.status = ctx->status;
+  g.wait_cycles = ctx->wait_cycles;
   ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K * g.nbatch,
                   2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K * g.nbatch) +
                       (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N * g.nbatch);
@@ -545,6 +555,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->prof_on = false; c->ev_used = 0;
   c->max_splits = 1;
   c->skinny_max_rows = 64;
+  c->wait_cycles = 0;
   c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
@@ -601,6 +612,13 @@ fvar_status fvar_set_option(fvar_ctx *ctx, int option, int value) {
     FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
     ctx->drop_graphs();
     ctx->max_splits = value;
+    return FVAR_OK;
+  }
+  if (option == FVAR_OPT_WAIT_KCYCLES) {
+    if (value < 0) return fail(ctx, FVAR_EINVAL, "set_option: the wait budget must not be negative");
+    FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
+    ctx->drop_graphs();
+    ctx->wait_cycles = static_cast<long long>(value) * 1000;
     return FVAR_OK;
   }
   if (option == FVAR_OPT_SKINNY_MAX_ROWS) {
@@ -684,13 +702,17 @@ fvar_status fvar_poll_status(fvar_ctx *ctx) {
     FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
     FV_CUDA(ctx, cudaMemcpy(&word, ctx->status, sizeof(word), cudaMemcpyDeviceToHost), "status read");
     if (word) FV_CUDA(ctx, cudaMemset(ctx->status, 0, sizeof(word)), "status clear");
+    if (word & kStatusTimeout) {
+      // a kernel that gave up may have left arrival counters of a split reduction half counted
+      FV_CUDA(ctx, cudaMemset(ctx->split_counters, 0, kSplitCounters * sizeof(int)), "counters clear");
+      ctx->drop_graphs();
+    }
   } else {
     FV_CUDA(ctx, cudaDeviceSynchronize(), "device synchronize");
-    FV_CUDA(ctx, cudaMemcpyFromSymbol(&word, g_kernel_status, sizeof(word)), "status read");
-    if (word) {
-      const unsigned zero = 0;
-      FV_CUDA(ctx, cudaMemcpyToSymbol(g_kernel_status, &zero, sizeof(zero)), "status clear");
-    }
+    unsigned *ks = kernel_status_ptr();
+    if (!ks) return fail(ctx, FVAR_ECUDA, "status word");
+    FV_CUDA(ctx, cudaMemcpy(&word, ks, sizeof(word), cudaMemcpyDeviceToHost), "status read");
+    if (word) FV_CUDA(ctx, cudaMemset(ks, 0, sizeof(word)), "status clear");
   }
   if (word & kStatusTimeout) return fail(ctx, FVAR_ETIMEOUT, "a device-side wait ran out");
   if (word & kStatusBadIndex) return fail(ctx, FVAR_EINVAL, "forced_indices out of range or not ascending");
@@ -1003,6 +1025,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       ga.out_f32 = ctx->xs;
       ga.ld_out = C;
       ga.status = ctx->status;
+      ga.wait_cycles = ctx->wait_cycles;
       const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, Mk + M, ctx->num_sms);
       ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + 2.0 * E * M * C) + 4.0 * E * r * C);
       FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
@@ -1041,6 +1064,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
       {
         AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, ctx->split_partial,
                     ctx->split_counters};
+        aa.wait_cycles = ctx->wait_cycles;
         aa.kv_splits = attention_pick_splits(E, H, r, D, L_prev + r, ctx->num_sms, kSplitScratchBytes, kSplitCounters);
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * (L_prev + r) * C, 4.0 * E * (L_prev + r) * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
@@ -1066,6 +1090,7 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
         prefetch_next(gq, blk, W_CO);
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
         AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, nullptr, nullptr};
+        aa.wait_cycles = ctx->wait_cycles;
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
         ctx->launched();
@@ -1278,16 +1303,6 @@ fvar_status fvar_get_group_output(fvar_ctx *ctx, int group, float *out_dev) {
 }
 
 // ------------------------------------------------------------------------------------------------ kernel-level
-static unsigned *kernel_status_ptr() {
-  static unsigned *p = nullptr;
-  if (!p) {
-    void *addr = nullptr;
-    if (cudaGetSymbolAddress(&addr, g_kernel_status) != cudaSuccess) return nullptr;
-    p = static_cast<unsigned *>(addr);
-  }
-  return p;
-}
-
 static fvar_status kfail(fvar_status s, const char *m) { g_init_error = m; return s; }
 #define FK_CUDA(call, what)                                                                          \
   do {                                                                                               \
@@ -1428,6 +1443,17 @@ fvar_status fvar_cfg_combine(const void *pair, int B, long long per_elem, float 
     return kfail(FVAR_EINVAL, "cfg_combine: bad arguments");
   FK_CUDA(launch_cfg_combine(static_cast<const bf16 *>(pair), B / 2, per_elem, guidance, static_cast<bf16 *>(out),
                              static_cast<cudaStream_t>(stream)), "cfg_combine");
+  return FVAR_OK;
+}
+
+fvar_status fvar_selftest_wait_timeout(fvar_ctx *ctx, long long cycles, void *stream) {
+  if (cycles <= 0) return ctx ? fail(ctx, FVAR_EINVAL, "selftest: cycles must be positive") : kfail(FVAR_EINVAL, "selftest: cycles must be positive");
+  unsigned *status = ctx ? ctx->status : kernel_status_ptr();
+  if (!status) return kfail(FVAR_ECUDA, "selftest: status word");
+  cudaStream_t st = ctx ? ctx->st : static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_wait_selftest(cycles, status, st);
+  if (e != cudaSuccess) return ctx ? cuda_fail(ctx, e, "selftest") : kfail(FVAR_ECUDA, cudaGetErrorString(e));
+  if (ctx) ctx->launched();
   return FVAR_OK;
 }
 

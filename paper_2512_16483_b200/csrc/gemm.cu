@@ -5,8 +5,6 @@
 // warps 2-9 drain the other accumulator (tcgen05.ld) and apply the epilogue, so the epilogue of
 // tile i overlaps the main loop of tile i+1.  Every wait is bounded; on expiry the CTA flags the
 // status word, lets its outstanding copies land, frees its TMEM and returns.
-#include <stdlib.h>
-
 #include "gemm_common.cuh"
 
 namespace fvar {
@@ -17,11 +15,6 @@ __host__ __device__ constexpr int k_atoms(int bn) { return bn <= 128 ? 2 : 1; }
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int kSmemBudget = 196608;     // bytes of operand stages per CTA (192 KiB)
 
-#ifdef FVAR_TRACE
-// Debug build only (-DFVAR_TRACE): CTA 0 records, per K stage, the cycles its producer spent waiting
-// for a free slot / issuing the copies and its MMA thread spent waiting for data / issuing.
-__device__ long long g_gemm_trace[4 * 1024];
-#endif
 
 template <int BN>
 struct GemmCfg {
@@ -62,6 +55,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wb = wait_budget(p.wait_cycles);
   const int tiles_m = (p.R + kBlockM - 1) / kBlockM;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int tiles_per_batch = tiles_m * tiles_n;
@@ -114,13 +108,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int row_w = p.w_mn_major ? e * p.b_batch_rows : e * p.b_batch_rows + n_idx * BN;
         const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
-#ifdef FVAR_TRACE
-          const long long tr0 = clock64();
-#endif
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
-#ifdef FVAR_TRACE
-          const long long tr1 = clock64();
-#endif
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag, wb)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), a_tx_bytes + Cfg::kStageBytesB);
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
 #pragma unroll
@@ -139,12 +127,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           armed |= 1u << stage;
           last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
           if (++stage == S) { stage = 0; phase ^= 1u; }
-#ifdef FVAR_TRACE
-          if (blockIdx.x == 0 && work == 0 && kb - kb0 < 1024) {
-            g_gemm_trace[4 * (kb - kb0)] = tr1 - tr0;
-            g_gemm_trace[4 * (kb - kb0) + 1] = clock64() - tr1;
-          }
-#endif
         }
       }
       if (!ok) {
@@ -172,19 +154,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int kb0 = sp * kb_per_split, kb1 = min(num_kb, kb0 + kb_per_split);
         const int a = it & 1;
         const uint32_t aphase = (it >> 1) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag, wb));
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
-#ifdef FVAR_TRACE
-          const long long tr0 = clock64();
-#endif
-          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, p.status, &abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, p.status, &abort_flag, wb));
           if (!ok) break;
-#ifdef FVAR_TRACE
-          const long long tr1 = clock64();
-#endif
           tc_fence_after();
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
           // descriptors are computed by the whole warp (warp-uniform values); only the issue is elected
@@ -208,12 +184,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           __syncwarp();
           if (++stage == S) { stage = 0; phase ^= 1u; }
-#ifdef FVAR_TRACE
-          if (leader && blockIdx.x == 0 && work == 0 && kb - kb0 < 1024) {
-            g_gemm_trace[4 * (kb - kb0) + 2] = tr1 - tr0;
-            g_gemm_trace[4 * (kb - kb0) + 3] = clock64() - tr1;
-          }
-#endif
         }
         if (ok && leader) umma_commit(tfull_bar(a));
         __syncwarp();
@@ -257,7 +227,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           have_pre = true;
         }
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag, wb));
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
@@ -340,31 +310,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   }
 }
 
-// Tuning override: FVAR_GEMM_BLOCK_N=64|128|256 forces the tile width (when it divides the problem).
-static int forced_block_n() {
-  static int v = -1;
-  if (v < 0) {
-    const char *e = getenv("FVAR_GEMM_BLOCK_N");
-    v = e ? atoi(e) : 0;
-    if (v != 64 && v != 128 && v != 256) v = 0;
-  }
-  return v;
-}
-
 // Cost model fitted to measurements on B200: an SM takes in about 100 GB/s from L2, so one K step
 // of a 128 x BN tile (16 KiB of A + BN * 128 B of W) costs t_k microseconds; a wave of work items
 // costs its K steps plus an epilogue that is only hidden behind the next item of the same CTA.
 // Splitting K trades a reduction through the scratch area for more CTAs streaming the operands.
+// microseconds per K block and per epilogue of a single-CTA tile of 64 / 128 / 256 columns
+static const float kTileTk[3] = {0.24f, 0.30f, 0.47f}, kTileTepi[3] = {1.0f, 1.5f, 2.5f};
+
 void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits, size_t scratch_bytes, int *block_n,
                     int *splits) {
   const int cand[3] = {64, 128, 256};
-  const float t_k[3] = {0.24f, 0.30f, 0.47f}, t_epi[3] = {1.0f, 1.5f, 2.5f};
   const int num_kb = (K + kBlockK - 1) / kBlockK;
   float best_cost = 1e30f;
   *block_n = 64;
   *splits = 1;
   for (int i = 0; i < 3; ++i) {
-    if (forced_block_n() && cand[i] != forced_block_n()) continue;
     const long long tiles = static_cast<long long>(tiles_m_total) * ((N + cand[i] - 1) / cand[i]);
     for (int sp = 1; sp <= max_splits; sp *= 2) {
       // splitting pays only for long reductions that would otherwise leave most SMs idle (measured)
@@ -373,7 +333,7 @@ void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits
         break;
       const long long waves = (tiles * sp + num_sms - 1) / num_sms;
       const int kb = (num_kb + sp - 1) / sp;
-      float cost = waves * (kb * t_k[i] + t_epi[i]);
+      float cost = waves * (kb * kTileTk[i] + kTileTepi[i]);
       if (sp > 1) cost += 1.5f + 0.6f * sp * cand[i] / 128.0f;      // park + fixed-order reduction by one CTA
       if (cost < best_cost) {
         best_cost = cost;
@@ -384,47 +344,29 @@ void gemm_pick_tile(int tiles_m_total, int N, int K, int num_sms, int max_splits
   }
 }
 
-#ifdef FVAR_TRACE
-extern "C" int fvar_debug_read_gemm_trace(long long *host, int n) {
-  return cudaMemcpyFromSymbol(host, g_gemm_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 1;
-}
-#endif
-
-// FVAR_GEMM_PAIR=0 never uses CTA pairs, =1 uses them whenever the problem allows; unset: cost model.
-static int forced_pair() {
-  static int v = -2;
-  if (v == -2) {
-    const char *e = getenv("FVAR_GEMM_PAIR");
-    v = (e && (e[0] == '0' || e[0] == '1') && e[1] == 0) ? e[0] - '0' : -1;
-  }
-  return v;
-}
 
 GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_clusters, int max_splits, size_t scratch_bytes) {
   GemmPlan plan{false, 64, 1};
   const int tiles_m = (R + kBlockM - 1) / kBlockM * nbatch;
   gemm_pick_tile(tiles_m, N, K, num_sms, max_splits, scratch_bytes, &plan.block_n, &plan.splits);
-  if (nbatch != 1 || R <= kBlockM || max_clusters <= 0 || forced_pair() == 0) return plan;
-  // Cost of the single-CTA choice, recomputed with the same constants as gemm_pick_tile.
-  const float t_k1[3] = {0.24f, 0.30f, 0.47f}, t_epi1[3] = {1.0f, 1.5f, 2.5f};
+  if (nbatch != 1 || R <= kBlockM || max_clusters <= 0) return plan;
+  // Cost of the single-CTA choice.
   const int num_kb = (K + kBlockK - 1) / kBlockK;
   const int i1 = plan.block_n == 64 ? 0 : (plan.block_n == 128 ? 1 : 2);
   const long long tiles1 = static_cast<long long>(tiles_m) * ((N + plan.block_n - 1) / plan.block_n) * plan.splits;
-  float cost1 = ((tiles1 + num_sms - 1) / num_sms) * (((num_kb + plan.splits - 1) / plan.splits) * t_k1[i1] + t_epi1[i1]);
+  float cost1 = ((tiles1 + num_sms - 1) / num_sms) * (((num_kb + plan.splits - 1) / plan.splits) * kTileTk[i1] + kTileTepi[i1]);
   if (plan.splits > 1) cost1 += 1.5f + 0.6f * plan.splits * plan.block_n / 128.0f;
   // A pair CTA moves, per K step, what a single CTA of half the tile width moves, for twice the output.
   const int cand2[2] = {128, 256};
-  const float t_k2[2] = {0.24f, 0.30f}, t_epi2[2] = {1.5f, 2.5f};
   const int tiles_m2 = (R + 2 * kBlockM - 1) / (2 * kBlockM);
   float best2 = 1e30f;
   int bn2 = 0;
   for (int i = 0; i < 2; ++i) {
-    if (forced_block_n() && cand2[i] != forced_block_n()) continue;
     const long long t2 = static_cast<long long>(tiles_m2) * ((N + cand2[i] - 1) / cand2[i]);
-    const float c = ((t2 + max_clusters - 1) / max_clusters) * (num_kb * t_k2[i] + t_epi2[i]);
+    const float c = ((t2 + max_clusters - 1) / max_clusters) * (num_kb * kTileTk[i] + kTileTepi[i + 1]);
     if (c < best2) { best2 = c; bn2 = cand2[i]; }
   }
-  if (bn2 && (forced_pair() == 1 || best2 < cost1)) plan = GemmPlan{true, bn2, 1};
+  if (bn2 && best2 < cost1) plan = GemmPlan{true, bn2, 1};
   return plan;
 }
 

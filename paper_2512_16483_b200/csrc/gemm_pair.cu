@@ -54,6 +54,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * S + 2 + a); };   // used in rank 0: both CTAs' epilogue threads
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wb = wait_budget(p.wait_cycles);
   const uint32_t rank = cluster_ctarank();
   const int pair = static_cast<int>(cluster_id_x()), npairs = static_cast<int>(cluster_nctaid_x());
   const int tiles_m2 = (p.R + 2 * kBlockM - 1) / (2 * kBlockM);
@@ -99,7 +100,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int row_a = (2 * m2 + static_cast<int>(rank)) * kBlockM;
         const int row_w = n_idx * BN + static_cast<int>(rank) * Cfg::kHalfN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag, wb)) { ok = false; break; }
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2u * Cfg::kStageBytes);
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
           const uint32_t fb = full0 + 8u * stage;
@@ -132,12 +133,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int work = pair; ok && work < total_tiles; work += npairs, ++it) {
         const int a = it & 1;
         const uint32_t aphase = (it >> 1) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(a), aphase ^ 1u, p.status, &abort_flag, wb));
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, p.status, &abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), phase, p.status, &abort_flag, wb));
           if (!ok) break;
           tc_fence_after();
           const uint32_t sa = smem_base + stage * Cfg::kStageBytes;
@@ -198,7 +199,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           have_pre = true;
         }
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(a), aphase, p.status, &abort_flag, wb));
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + a * BN + (static_cast<uint32_t>(quad * 32) << 16);
@@ -316,7 +317,7 @@ static cudaError_t pair_launch_one(const CUtensorMap &tmA, const CUtensorMap &tm
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<BN, EPI>, tmA, tmW, a);
 }
 

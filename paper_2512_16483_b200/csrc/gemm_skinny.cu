@@ -129,6 +129,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   const uint32_t tfull_bar = bar_base + 8u * (2 * kSkinnyMaxStages);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long wb = wait_budget(p.wait_cycles);
   const int S = p.splits > 1 ? p.splits : 1;                 // cluster size = K ranges per tile
   const int sp = static_cast<int>(cluster_ctarank());
   const int tile = static_cast<int>(cluster_id_x());
@@ -196,7 +197,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
       for (int i = pre; ok && i < nst; ++i) {
         const int stage = i % nstages;
         const uint32_t phase = (i / nstages) & 1u;
-        if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(stage), phase ^ 1u, p.status, &abort_flag, wb)) { ok = false; break; }
         mbar_expect_tx(full_bar(stage), stage_bytes);
         load_w(i);
         load_a(i);
@@ -230,7 +231,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t idesc = umma_idesc_bf16(kBlockM, rp);
     for (int i = 0; i < nst; ++i) {
       const int stage = i % nstages;
-      ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), (i / nstages) & 1u, p.status, &abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(full_bar(stage), (i / nstages) & 1u, p.status, &abort_flag, wb));
       if (!ok) break;
       tc_fence_after();
       const uint32_t sa = ring + stage * stage_bytes;
@@ -259,7 +260,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   } else {
     pdl_wait();
     pdl_launch_dependents();
-    ok = nkb > 0 && __all_sync(0xffffffffu, mbar_wait(tfull_bar, 0, p.status, &abort_flag));
+    ok = nkb > 0 && __all_sync(0xffffffffu, mbar_wait(tfull_bar, 0, p.status, &abort_flag, wb));
     tc_fence_after();
   }
 
@@ -411,7 +412,7 @@ static cudaError_t skinny_launch_one(const CUtensorMap &tmA, const CUtensorMap &
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<EPI>, tmA, tmW, a);
 }
 

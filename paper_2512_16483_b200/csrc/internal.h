@@ -63,6 +63,7 @@ struct GemmArgs {
   // optional: weights the next GEMM of the chain will stream; every CTA asks L2 to prefetch its share
   const void *pf_ptr;
   unsigned long long pf_bytes;
+  long long wait_cycles;   // budget of every bounded wait (0: the default, about half a second)
 };
 
 // Tensor maps: bf16, 2-D {cols, rows} with a {64, box_rows} box and 128-byte swizzle, or the 3-D
@@ -124,15 +125,14 @@ struct AttnArgs {
   int kv_splits;
   float *part;
   int *counters;
+  long long wait_cycles;   // budget of every bounded wait (0: the default)
 };
 // Number of key ranges to split an attention launch into (1 = no split), given the scratch available.
 int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms, size_t scratch_bytes, int max_counters);
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                              const AttnArgs &a, cudaStream_t st);
 
-// Launch with programmatic stream serialization (see pdl_wait in ptx.cuh).  FVAR_NO_PDL=1 in the
-// environment turns the attribute off (plain stream order).
-bool pdl_enabled();
+// Launch with programmatic stream serialization (see pdl_wait in ptx.cuh).
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
   cudaLaunchConfig_t cfg = {};
@@ -144,7 +144,7 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
@@ -178,6 +178,9 @@ cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0,
                                  bool overwrite, float *F, cudaStream_t st);
 cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st);
 cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st);
+// Self-test of the bounded wait: one CTA waits on an mbarrier nobody signals with a budget of `cycles`, flags the
+// status word and returns.
+cudaError_t launch_wait_selftest(long long cycles, unsigned *status, cudaStream_t st);
 cudaError_t launch_l2_prefetch(const void *ptr, unsigned long long bytes, cudaStream_t st);
 cudaError_t launch_silu_bf16(const bf16 *in, bf16 *out, long long n, cudaStream_t st);
 cudaError_t launch_load_kv(const bf16 *K, const bf16 *V, int B, int L, int H, int D, int L_cap, bf16 *kc, bf16 *vt,

@@ -12,8 +12,10 @@ namespace fvar {
 // Bits of the device status word.
 enum : unsigned { kStatusTimeout = 1u, kStatusBadIndex = 2u };
 
-// A wait gives up after this many clock cycles (about half a second at boost clock).
+// Default budget of a bounded wait in clock cycles (about half a second at boost clock); kernels take the
+// budget as an argument (0 = this default), so that a test can make a wait run out in a millisecond.
 constexpr long long kWaitCycles = 1000000000ll;
+__host__ __device__ constexpr long long wait_budget(long long cycles) { return cycles > 0 ? cycles : kWaitCycles; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -67,8 +69,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: returns false (after flagging the status word and the CTA's abort flag) when the
-// phase has not completed within kWaitCycles, or as soon as another thread of the CTA has aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned *status, volatile int *abort_flag) {
+// phase has not completed within `budget` cycles, or as soon as another thread of the CTA has aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned *status, volatile int *abort_flag,
+                                          long long budget) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
@@ -76,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > budget) {
       *abort_flag = 1;
       atomicOr(status, kStatusTimeout);
       return false;

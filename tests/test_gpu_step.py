@@ -72,7 +72,12 @@ class Pair:
         assert self.gpu.poll_status() == self.fv.OK
 
 
-def _step_both(p: Pair, toks, k, *, mode, cfg="pair", ranks=None, keep_ratio=1.0, forced=True):
+def _step_both(p: Pair, toks, k, *, mode, cfg="pair", ranks=None, keep_ratio=1.0, forced=True, bar=2e-2):
+    """One step on both sides.  Besides returning the bf16 result and the oracle's, holds the fp32 output of every
+    block group (what the next group and the next scale read) to the block-output bar: max-abs error <= bar x RMS,
+    cosine >= 0.999, on the batch elements the step computed.  Under RP + RTR the bar of group g (0-based) is
+    bar x sqrt(g + 1): the projection carries the whole deviation of a group's rows into the rows of the next
+    one, so the groups' deviations add in quadrature (tests/test_tolerance_floor.py shows the law on the oracle)."""
     fv = p.fv
     pol = orc.Policy({fv.DENSE: "dense", fv.LOWRANK_RTR: "lowrank_rtr"}[mode], cfg, keep_ratio, ranks)
     ref = p.oracle.scale_step(toks, k, pol)
@@ -86,6 +91,13 @@ def _step_both(p: Pair, toks, k, *, mode, cfg="pair", ranks=None, keep_ratio=1.0
     out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=mode, cfg_mode=fv.CFG_NULL_ONLY if cfg == "null_only" else fv.CFG_PAIR,
                            keep_ratio=keep_ratio, rank_per_group=ranks, forced_indices=fi)
     p.check_ok()
+    els = list(range(1, p.B, 2)) if cfg == "null_only" else list(range(p.B))
+    if forced or mode == fv.DENSE:
+        for g in range(p.shp.n_groups):
+            g32 = p.gpu.get_group_output(g, toks.shape[1]).cpu().numpy()
+            assert_close(g32[els], np.stack([p.oracle.group_cache[g][b] for b in els]),
+                         max_rel=bar * (np.sqrt(g + 1.0) if mode == fv.LOWRANK_RTR else 1.0),
+                         what="fp32 output of group %d, scale %d" % (g, k))
     return bf16_to_numpy(out), ref
 
 

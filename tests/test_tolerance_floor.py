@@ -29,3 +29,40 @@ def test_bf16_operand_rounding_floor_by_shape():
     inf = _ffn_floor(si.shape_infinity_2b(n_blocks=1, blocks_per_group=1), 65)
     assert d16 < 1.0e-2, d16
     assert 1.0e-2 < inf < 2.5e-2, inf
+
+
+def test_deviations_add_in_quadrature_over_block_groups():
+    """Why a stack of G block groups is held to bar x sqrt(g) at group g.  RP keeps the energy of whatever it
+    projects (E|Q^T e|^2 = |e|^2 for Q_ij ~ N(0, 1/r), Sec. 3.3), so the deviation e_{g-1} that group g - 1 left in
+    its output rows is carried whole into the r rows group g sends through its blocks, where that group's own
+    deviation n_g is added: E|e_g|^2 = |e_{g-1}|^2 + |n_g|^2, while RTR's filled rows (copied from the cache) carry
+    none.  Checked here with the oracle's own RP / selection / RTR on a chain of 8 groups whose "blocks" are the
+    identity plus an independent perturbation of fixed energy: the deviation energy after g groups is g times
+    that of one group (within the spread of a random Q), and the max-abs deviation over the output RMS grows
+    with it.  A real block is not the identity, but its Jacobian on these shapes has gain close to 1 (residual
+    stream plus gated branches), which is what the GPU measures: 1.2e-2 after one Infinity-shaped group at the
+    64 x 64 scale, 4e-2 after eight."""
+    rng = np.random.default_rng(7)
+    M, C, r, G, eps = 1024, 64, 32, 8, 1e-2
+    hw = (32, 32)
+    cache = [rng.standard_normal((M, C)) for _ in range(G)]
+    X_exact = rng.standard_normal((M, C))
+    X_pert = X_exact.copy()
+    energy, ratio = [], []
+    for g in range(G):
+        Q = rng.standard_normal((M, r)) / np.sqrt(r)
+        idx = orc.select_top_r(orc.row_scores(X_exact), r)          # teacher-forced: one index set for both chains
+        Fe = orc.random_projection(Q, X_exact)
+        Fp = orc.random_projection(Q, X_pert)
+        n = rng.standard_normal((r, C))
+        n *= eps * np.linalg.norm(Fe) / np.linalg.norm(n)          # |n_g| = eps |F_r|, independent of everything else
+        up = orc.upsample_bilinear(cache[g], hw, hw)
+        X_exact = orc.rtr_restore(Fe, idx, up)
+        X_pert = orc.rtr_restore(Fp + n, idx, up)
+        e = X_pert - X_exact
+        assert np.count_nonzero(np.abs(e).sum(axis=1)) == r        # filled rows carry no deviation
+        energy.append(float((e ** 2).sum() / (n ** 2).sum()))
+        ratio.append(float(np.abs(e).max() / np.sqrt((X_exact ** 2).mean())))
+    for g in range(G):                                             # |e_g|^2 ~ (g + 1) |n|^2
+        assert 0.6 * (g + 1) <= energy[g] <= 1.6 * (g + 1), energy
+    assert ratio[-1] > 2.0 * ratio[0], ratio
