@@ -169,7 +169,9 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
                             void *out);
 
 /* Same step with HOST buffers: copies tokens host->dev, runs the step, copies out dev->host, and
- * synchronises the stream before returning.  Pinned host memory makes the copies asynchronous. */
+ * synchronises the stream before returning.  Pinned host memory makes the copies asynchronous.
+ * tokens_host is [B][M][C] as for fvar_scale_step; with FVAR_CFG_NULL_ONLY only the elements 2p + 1
+ * that the step reads are uploaded (one strided copy). */
 fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int scale_idx,
                                  const fvar_keep_policy *policy, void *out_host);
 

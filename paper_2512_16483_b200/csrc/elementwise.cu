@@ -503,34 +503,35 @@ cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned 
 }
 
 // ------------------------------------------------------------------------------------------------
+// bf16 tokens -> the fp32 work stream, for the E batch elements the step computes only: computed element e is read
+// at element e * smul + soff of `tok` and written at element e * bmul + boff of `x`.
 __global__ void tokens_to_f32_kernel(const bf16 *__restrict__ tok, float *__restrict__ x, long long n8, long long per8,
-                                     bf16 *__restrict__ xsplit, long long half8, int bmul, int boff) {
+                                     bf16 *__restrict__ xsplit, long long half8, int smul, int soff, int bmul, int boff) {
   pdl_wait();
   pdl_launch_dependents();
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n8) return;
-  const uint4 u = __ldg(reinterpret_cast<const uint4 *>(tok) + i);
-  if (xsplit != nullptr) {                       // hi = the token itself, lo = 0, for the elements that are computed
-    const long long b = i / per8, off = i - b * per8;
-    if (b >= boff && (b - boff) % bmul == 0) {
-      uint4 *dst = reinterpret_cast<uint4 *>(xsplit) + ((b - boff) / bmul) * 2 * half8 + off;
-      dst[0] = u;
-      dst[half8] = make_uint4(0u, 0u, 0u, 0u);
-    }
+  const long long e = i / per8, off = i - e * per8;
+  const uint4 u = __ldg(reinterpret_cast<const uint4 *>(tok) + (e * smul + soff) * per8 + off);
+  if (xsplit != nullptr) {                       // hi = the token itself, lo = 0
+    uint4 *dst = reinterpret_cast<uint4 *>(xsplit) + e * 2 * half8 + off;
+    dst[0] = u;
+    dst[half8] = make_uint4(0u, 0u, 0u, 0u);
   }
   const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
   const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]), c = __bfloat1622float2(h[2]),
                d = __bfloat1622float2(h[3]);
-  reinterpret_cast<float4 *>(x)[2 * i] = make_float4(a.x, a.y, b.x, b.y);
-  reinterpret_cast<float4 *>(x)[2 * i + 1] = make_float4(c.x, c.y, d.x, d.y);
+  float4 *dst = reinterpret_cast<float4 *>(x) + 2 * ((e * bmul + boff) * per8 + off);
+  dst[0] = make_float4(a.x, a.y, b.x, b.y);
+  dst[1] = make_float4(c.x, c.y, d.x, d.y);
 }
 
-cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, int M, int C, bf16 *xsplit, int mk, int bmul, int boff,
-                                 cudaStream_t st) {
-  const long long per8 = static_cast<long long>(M) * C / 8, n8 = static_cast<long long>(B) * per8;
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int E, int M, int C, bf16 *xsplit, int mk, int smul, int soff,
+                                 int bmul, int boff, cudaStream_t st) {
+  const long long per8 = static_cast<long long>(M) * C / 8, n8 = static_cast<long long>(E) * per8;
   if (n8 <= 0) return cudaSuccess;
   return launch_pdl(tokens_to_f32_kernel, dim3(static_cast<unsigned>((n8 + 255) / 256)), dim3(256), 0, st, tok, x, n8, per8, xsplit,
-                    static_cast<long long>(mk) * C / 8, bmul, boff);
+                    static_cast<long long>(mk) * C / 8, smul, soff, bmul, boff);
 }
 
 __global__ void out_to_bf16_kernel(const float *__restrict__ x, RowMap xmap, int M, int C, bf16 *__restrict__ out) {

@@ -909,7 +909,10 @@ fvar_status fvar_load_group_cache(fvar_ctx *ctx, int scale_idx, const float *cac
   return FVAR_OK;
 }
 
-fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, const fvar_keep_policy *pol, void *out) {
+// tokens_compact: `tokens` holds only the E elements the step computes, [E][M][C] (the host entry points upload
+// nothing else); otherwise all B elements, [B][M][C].
+static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool tokens_compact, int scale_idx,
+                                   const fvar_keep_policy *pol, void *out) {
   if (!ctx) return FVAR_EINVAL;
   if (!pol) return fail(ctx, FVAR_EINVAL, "scale_step: policy is NULL");
   if (pol->mode == FVAR_SKIP) return FVAR_OK;
@@ -960,11 +963,11 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   const size_t ada_blk = static_cast<size_t>(ctx->Bmax) * 6 * C;
   cudaStream_t st = ctx->st;
 
-  ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * B * M * C);
+  ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 6.0 * E * M * C);
   const int Mk = static_cast<int>(align_up(M, 64));
   // the projection of a late group reads its input rows as a hi / lo bf16 split, written by whoever produces them
-  FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, B, M, C, rank[0] < M ? ctx->xsplit[0] : nullptr, Mk,
-                                    bmul, boff, st), "tokens_to_f32");
+  FV_CUDA(ctx, launch_tokens_to_f32(static_cast<const bf16 *>(tokens), ctx->x0, E, M, C, rank[0] < M ? ctx->xsplit[0] : nullptr, Mk,
+                                    tokens_compact ? 1 : bmul, tokens_compact ? 0 : boff, bmul, boff, st), "tokens_to_f32");
   ctx->launched();
   const float *X_in = ctx->x0;
   const RowMap bmap{bmul, boff, M};              // buffers indexed by the caller's batch element
@@ -1213,6 +1216,19 @@ fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, co
   return FVAR_OK;
 }
 
+fvar_status fvar_scale_step(fvar_ctx *ctx, const void *tokens, int scale_idx, const fvar_keep_policy *pol, void *out) {
+  return scale_step_impl(ctx, tokens, false, scale_idx, pol, out);
+}
+
+// Host -> device copy of the token rows a step reads: every element, or with the null-prompt branch alone only
+// elements 2p + 1, packed [E][M][C] (one strided copy).
+static cudaError_t upload_tokens(fvar_ctx *ctx, bf16 *dst, const void *tokens_host, size_t per_elem_bytes, bool null_only,
+                                 cudaStream_t st) {
+  if (!null_only) return cudaMemcpyAsync(dst, tokens_host, per_elem_bytes * ctx->B, cudaMemcpyHostToDevice, st);
+  return cudaMemcpy2DAsync(dst, per_elem_bytes, static_cast<const uint8_t *>(tokens_host) + per_elem_bytes, 2 * per_elem_bytes,
+                           per_elem_bytes, static_cast<size_t>(ctx->B / 2), cudaMemcpyHostToDevice, st);
+}
+
 fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int scale_idx, const fvar_keep_policy *pol,
                                  void *out_host) {
   if (!ctx) return FVAR_EINVAL;
@@ -1222,10 +1238,11 @@ fvar_status fvar_scale_step_host(fvar_ctx *ctx, const void *tokens_host, int sca
   if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || ctx->B <= 0) return fail(ctx, FVAR_EINVAL, "scale_step_host: bad scale_idx or no cond");
   // Staging: the bf16 tokens land in the hidden-activation buffer (free until the first fc1) and
   // the bf16 output in the attention-output buffer (free after the last out-proj).
-  const size_t M = ctx->Mk[scale_idx], in_bytes = static_cast<size_t>(ctx->B) * M * ctx->C * 2;
-  const int E = pol->cfg_mode == FVAR_CFG_NULL_ONLY ? ctx->B / 2 : ctx->B;
-  FV_CUDA(ctx, cudaMemcpyAsync(ctx->hbuf, tokens_host, in_bytes, cudaMemcpyHostToDevice, ctx->st), "tokens H2D");
-  fvar_status s = fvar_scale_step(ctx, ctx->hbuf, scale_idx, pol, ctx->a);
+  const size_t M = ctx->Mk[scale_idx];
+  const bool null_only = pol->cfg_mode == FVAR_CFG_NULL_ONLY && ctx->B % 2 == 0;
+  const int E = null_only ? ctx->B / 2 : ctx->B;
+  FV_CUDA(ctx, upload_tokens(ctx, ctx->hbuf, tokens_host, M * ctx->C * 2, null_only, ctx->st), "tokens H2D");
+  fvar_status s = scale_step_impl(ctx, ctx->hbuf, null_only, scale_idx, pol, ctx->a);
   if (s != FVAR_OK) return s;
   FV_CUDA(ctx, cudaMemcpyAsync(out_host, ctx->a, static_cast<size_t>(E) * M * ctx->C * 2, cudaMemcpyDeviceToHost, ctx->st), "out D2H");
   FV_CUDA(ctx, cudaStreamSynchronize(ctx->st), "stream synchronize");
@@ -1240,18 +1257,19 @@ fvar_status fvar_scale_step_host_async(fvar_ctx *ctx, const void *tokens_host, i
   if (!tokens_host || !out_host) return fail(ctx, FVAR_EINVAL, "scale_step_host_async: NULL tokens / out");
   if (scale_idx < 0 || scale_idx >= ctx->cfg.n_scales || ctx->B <= 0) return fail(ctx, FVAR_EINVAL, "scale_step_host_async: bad scale_idx or no cond");
   if (!ctx->host_pipe_ok) return fail(ctx, FVAR_ECUDA, "scale_step_host_async: copy streams unavailable");
-  const size_t M = ctx->Mk[scale_idx], in_bytes = static_cast<size_t>(ctx->B) * M * ctx->C * 2;
-  const int E = pol->cfg_mode == FVAR_CFG_NULL_ONLY ? ctx->B / 2 : ctx->B;
+  const size_t M = ctx->Mk[scale_idx];
+  const bool null_only = pol->cfg_mode == FVAR_CFG_NULL_ONLY && ctx->B % 2 == 0;
+  const int E = null_only ? ctx->B / 2 : ctx->B;
   const int s = static_cast<int>(ctx->host_calls & 1);
   const bool reuse = ctx->host_calls >= 2;     // the slot was used two calls ago
   // host -> device on the upload stream, once the step that last read this slot has finished
   if (reuse) FV_CUDA(ctx, cudaStreamWaitEvent(ctx->h2d_st, ctx->ev_cmp[s], 0), "upload wait");
-  FV_CUDA(ctx, cudaMemcpyAsync(ctx->hin[s], tokens_host, in_bytes, cudaMemcpyHostToDevice, ctx->h2d_st), "tokens H2D");
+  FV_CUDA(ctx, upload_tokens(ctx, ctx->hin[s], tokens_host, M * ctx->C * 2, null_only, ctx->h2d_st), "tokens H2D");
   FV_CUDA(ctx, cudaEventRecord(ctx->ev_in[s], ctx->h2d_st), "upload record");
   // the step on the caller's stream, once its tokens are there and the slot's previous result has left
   FV_CUDA(ctx, cudaStreamWaitEvent(ctx->st, ctx->ev_in[s], 0), "step wait");
   if (reuse) FV_CUDA(ctx, cudaStreamWaitEvent(ctx->st, ctx->ev_out[s], 0), "step wait");
-  fvar_status rc = fvar_scale_step(ctx, ctx->hin[s], scale_idx, pol, ctx->hout[s]);
+  fvar_status rc = scale_step_impl(ctx, ctx->hin[s], null_only, scale_idx, pol, ctx->hout[s]);
   if (rc != FVAR_OK) return rc;
   FV_CUDA(ctx, cudaEventRecord(ctx->ev_cmp[s], ctx->st), "step record");
   // device -> host on the download stream

@@ -163,10 +163,11 @@ cudaError_t launch_ln_modulate(const float *x, RowMap xmap, int E, int rows, int
 // xsplit (optional): the filled rows also go out as their two-term bf16 split, [E][2][mk][C] (see GemmArgs::xsplit).
 cudaError_t launch_rtr_fill(const float *prev, float *out, int E, int bmul, int boff, int h0, int w0, int h1,
                             int w1, int C, const int *inv, bf16 *xsplit, int mk, cudaStream_t st);
-// xsplit (optional): the rows of the computed elements b = e * bmul + boff also go out as hi = token, lo = 0 in the
-// [E][2][mk][C] split layout (tokens are bf16 already).
-cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int B, int M, int C, bf16 *xsplit, int mk, int bmul, int boff,
-                                 cudaStream_t st);
+// The E computed elements only: element e is read at element e * smul + soff of `tok` and written at element
+// e * bmul + boff of `x`.  xsplit (optional): the rows also go out as hi = token, lo = 0 in the [E][2][mk][C] split
+// layout (tokens are bf16 already).
+cudaError_t launch_tokens_to_f32(const bf16 *tok, float *x, int E, int M, int C, bf16 *xsplit, int mk, int smul, int soff,
+                                 int bmul, int boff, cudaStream_t st);
 cudaError_t launch_out_to_bf16(const float *x, RowMap xmap, int E, int M, int C, bf16 *out, cudaStream_t st);
 cudaError_t launch_generate_projection(bf16 *qt, int M, int Mk, int r, unsigned long long seed, int group, int scale,
                                        cudaStream_t st);
