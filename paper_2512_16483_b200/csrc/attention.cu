@@ -11,6 +11,11 @@
 // bandwidth, and a P tile costs one write and one read on top.  O stays in TMEM for the whole key loop; its rows are rescaled only when the
 // running maximum has grown by more than 2^8 since the last rescale, so the common case costs no
 // TMEM round trip.  Keys at or beyond L are masked.  Every wait is bounded (see ptx.cuh).
+//
+// Few queries over a long cache (few CTAs, many key blocks): the key range is split over a thread-block cluster of
+// up to 8 CTAs.  Each parks its unnormalised (O, m, l) in its own shared memory; after a cluster barrier every
+// CTA merges a slice of the query rows over all ranges through distributed shared memory, in range order (the
+// result does not depend on timing), normalises and stores.  Nothing goes through global scratch.
 #include <math.h>
 
 #include "internal.h"
@@ -47,7 +52,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t tmem_base_holder;
   __shared__ volatile int abort_flag;
-  __shared__ volatile int merge_last[2];
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_smem = smem_base;
@@ -62,10 +66,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long wb = wait_budget(p.wait_cycles);
-  // Split-KV: kv_splits CTAs share one query tile pair, each covering a contiguous range of key
-  // blocks; their unnormalised results are merged by whichever of them finishes last.
+  // kv_splits CTAs (one cluster) share a query tile pair, each covering a contiguous range of key blocks.
   const int splits = p.kv_splits > 1 ? p.kv_splits : 1;
-  const int qt = blockIdx.x / splits, sp = blockIdx.x - qt * splits, h = blockIdx.y, e = blockIdx.z;
+  const int qt = blockIdx.x / splits, sp = blockIdx.x - qt * splits, h = blockIdx.y, e = blockIdx.z;   // sp = rank in the cluster
   const int b = e * p.bmul + p.boff;
   const int bh = b * p.H + h;
   const int nkv_total = (p.L + kKeys - 1) / kKeys;
@@ -101,6 +104,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t tmem_base = tmem_base_holder;
   pdl_launch_dependents();      // the successor (a GEMM) only requests weights before its own wait
   pdl_wait();
+  float m_ref = -INFINITY, l_run = 0.f;      // softmax threads: running maximum and sum of this thread's query row
+  bool final_ok = false;                      // softmax threads: the last P V of the row's tile has completed
 
   if (warp == 0) {
     if (lane == 0) {
@@ -217,7 +222,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint32_t s_base = tmem_base + lane_addr;
       const uint32_t o_addr = tmem_base + 256 + t * D + lane_addr;
       const float c = p.scale_log2;
-      float m_ref = -INFINITY, l_run = 0.f;
       bool ok = true;
 
       for (int j = 0; j < nkv; ++j) {
@@ -296,93 +300,103 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tc_fence_before();
         mbar_arrive(p_full(t));
       }
-      if (ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag, wb))) {
+      final_ok = ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag, wb));
+      if (final_ok && splits == 1) {
         tc_fence_after();
         const int rib = qt * 2 * kQRows + t * kQRows + row_local;
         bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;
-        auto store_chunk = [&](int cc, const float (&o)[32], float scale) {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint32_t w[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              __nv_bfloat162 v2 = __floats2bfloat162_rn(o[q * 8 + u * 2] * scale, o[q * 8 + u * 2 + 1] * scale);
-              w[u] = *reinterpret_cast<uint32_t *>(&v2);
-            }
-            reinterpret_cast<uint4 *>(dst + cc * 32)[q] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        };
-        if (splits == 1) {
-          const float inv_l = 1.0f / l_run;
+        const float inv_l = 1.0f / l_run;
 #pragma unroll 1
-          for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(o_addr + cc * 32, v);
-            tmem_ld_wait();
-            float o[32];
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(o_addr + cc * 32, v);
+          tmem_ld_wait();
+          if (rib < p.r) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
-            if (rib < p.r) store_chunk(cc, o, inv_l);
-          }
-        } else {
-          // Park (O, m, l) of this key range.  Layout per (tile slot, split): float4 number d4 * 128 + row
-          // (coalesced across the lanes of a warp), then m[128] and l[128].
-          const int tslot = ((e * p.H + h) * static_cast<int>(gridDim.x / splits) + qt) * 2 + t;
-          const size_t per_split = static_cast<size_t>(D + 2) * kQRows;            // floats
-          float *mine = p.part + (static_cast<size_t>(tslot) * splits + sp) * per_split;
-#pragma unroll 1
-          for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t v[32];
-            tmem_ld32(o_addr + cc * 32, v);
-            tmem_ld_wait();
+            for (int q = 0; q < 4; ++q) {
+              uint32_t w[4];
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-              __stcg(reinterpret_cast<float4 *>(mine) + (cc * 8 + q) * kQRows + row_local,
-                     make_float4(__uint_as_float(v[q * 4]), __uint_as_float(v[q * 4 + 1]), __uint_as_float(v[q * 4 + 2]),
-                                 __uint_as_float(v[q * 4 + 3])));
-          }
-          __stcg(mine + D * kQRows + row_local, m_ref);
-          __stcg(mine + (D + 1) * kQRows + row_local, l_run);
-          __threadfence();
-          if (t == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
-          if (row_local == 0) merge_last[t] = (atomicAdd(p.counters + tslot, 1) == splits - 1) ? 1 : 0;
-          if (t == 0) asm volatile("bar.sync 1, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
-          if (merge_last[t]) {
-            __threadfence();
-            const float *base = p.part + static_cast<size_t>(tslot) * splits * per_split;
-            float m_all = -INFINITY;
-            for (int s2 = 0; s2 < splits; ++s2) m_all = fmaxf(m_all, __ldcg(base + s2 * per_split + D * kQRows + row_local));
-            float l_all = 0.f;
-            for (int s2 = 0; s2 < splits; ++s2) {
-              const float *ps = base + s2 * per_split;
-              l_all += __ldcg(ps + (D + 1) * kQRows + row_local) * exp2f((__ldcg(ps + D * kQRows + row_local) - m_all) * c);
-            }
-            const float inv_l = 1.0f / l_all;
-#pragma unroll 1
-            for (int cc = 0; cc < D / 32; ++cc) {
-              float o[32];
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = 0.f;
-              for (int s2 = 0; s2 < splits; ++s2) {                 // fixed order: the sum does not depend on timing
-                const float *ps = base + s2 * per_split;
-                const float w = exp2f((__ldcg(ps + D * kQRows + row_local) - m_all) * c);
-                const float4 *src = reinterpret_cast<const float4 *>(ps) + cc * 8 * kQRows + row_local;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                  const float4 v = __ldcg(src + q * kQRows);
-                  o[q * 4] = fmaf(w, v.x, o[q * 4]);
-                  o[q * 4 + 1] = fmaf(w, v.y, o[q * 4 + 1]);
-                  o[q * 4 + 2] = fmaf(w, v.z, o[q * 4 + 2]);
-                  o[q * 4 + 3] = fmaf(w, v.w, o[q * 4 + 3]);
-                }
+              for (int u = 0; u < 4; ++u) {
+                __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(v[q * 8 + u * 2]) * inv_l, __uint_as_float(v[q * 8 + u * 2 + 1]) * inv_l);
+                w[u] = *reinterpret_cast<uint32_t *>(&v2);
               }
-              if (rib < p.r) store_chunk(cc, o, inv_l);
+              reinterpret_cast<uint4 *>(dst + cc * 32)[q] = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            if (row_local == 0) p.counters[tslot] = 0;               // ready for the next launch
           }
         }
       }
     }
+  }
+
+  if (splits > 1) {
+    // ---------------------------------------------------------------- merge of the key ranges over the cluster
+    // Every thread of every CTA of the cluster passes the same barriers, whatever happened to its waits.
+    constexpr uint32_t kPitch = (D + 4) * 4;                       // bytes per parked row: conflict-free 16-byte accesses
+    const uint32_t part_o = ring_smem;                             // [2 tiles][128 rows][D + 4] fp32; the ring is idle by now
+    const uint32_t part_m = part_o + 2 * kQRows * kPitch;          // [2][128] running maxima, then [2][128] sums
+    tc_fence_before();
+    __syncthreads();                                               // all roles done: no MMA reads the ring any more
+    if (warp >= 2 && final_ok) {
+      tc_fence_after();
+      const int t = (warp - 2) >> 2, row_local = (warp & 3) * 32 + lane;
+      const uint32_t o_addr = tmem_base + 256 + t * D + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+      const uint32_t dst = part_o + static_cast<uint32_t>(t * kQRows + row_local) * kPitch;
+#pragma unroll 1
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t v[32];
+        tmem_ld32(o_addr + cc * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (cc * 32 + q * 4) * 4), "r"(v[q * 4]), "r"(v[q * 4 + 1]),
+                       "r"(v[q * 4 + 2]), "r"(v[q * 4 + 3]) : "memory");
+      }
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_m + (t * kQRows + row_local) * 4), "f"(m_ref) : "memory");
+      asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_m + (2 * kQRows + t * kQRows + row_local) * 4), "f"(l_run) : "memory");
+    }
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp >= 2 && abort_flag == 0) {
+      constexpr int G = D / 4;                                     // threads per row, one float4 each
+      const int st = static_cast<int>(threadIdx.x) - 64, d4 = (st % G) * 4;
+      uint32_t peer_o[8], peer_m[8];
+#pragma unroll
+      for (int s2 = 0; s2 < 8; ++s2) {
+        peer_o[s2] = mapa_shared(part_o, static_cast<uint32_t>(s2 < splits ? s2 : 0));
+        peer_m[s2] = mapa_shared(part_m, static_cast<uint32_t>(s2 < splits ? s2 : 0));
+      }
+      const float c = p.scale_log2;
+      for (int tt = 0; tt < ntiles; ++tt) {
+        const int rows_valid = min(kQRows, p.r - qt * 2 * kQRows - tt * kQRows);
+        const int rpr = (rows_valid + splits - 1) / splits;        // this CTA merges rows [lo, hi) of the tile
+        const int lo = sp * rpr, hi = min(rows_valid, lo + rpr);
+        for (int row = lo + st / G; row < hi; row += 256 / G) {
+          const uint32_t moff = static_cast<uint32_t>(tt * kQRows + row) * 4;
+          float ms[8], m_all = -INFINITY;
+#pragma unroll
+          for (int s2 = 0; s2 < 8; ++s2)
+            if (s2 < splits) { ms[s2] = ld_dsmem_f32(peer_m[s2] + moff); m_all = fmaxf(m_all, ms[s2]); }
+          float l_all = 0.f;
+          float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+          const uint32_t ooff = static_cast<uint32_t>(tt * kQRows + row) * kPitch + d4 * 4;
+#pragma unroll
+          for (int s2 = 0; s2 < 8; ++s2)
+            if (s2 < splits) {                                     // range order: the sum does not depend on timing
+              const float w = exp2f((ms[s2] - m_all) * c);
+              l_all = fmaf(ld_dsmem_f32(peer_m[s2] + 2 * kQRows * 4 + moff), w, l_all);
+              const float4 v = ld_dsmem_f4(peer_o[s2] + ooff);
+              o.x = fmaf(w, v.x, o.x); o.y = fmaf(w, v.y, o.y); o.z = fmaf(w, v.z, o.z); o.w = fmaf(w, v.w, o.w);
+            }
+          const float inv_l = 1.0f / l_all;
+          const int rib = qt * 2 * kQRows + tt * kQRows + row;
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(o.x * inv_l, o.y * inv_l), h1 = __floats2bfloat162_rn(o.z * inv_l, o.w * inv_l);
+          *reinterpret_cast<uint2 *>(p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D + d4) =
+              make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
+        }
+      }
+    }
+    __syncwarp();
+    cluster_sync_all();                                            // nobody leaves while a peer still reads its rows
   }
 
   tc_fence_before();
@@ -416,20 +430,33 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   cudaError_t err = set_attr<D>();
   if (err != cudaSuccess) return err;
   const int splits = a.kv_splits > 1 ? a.kv_splits : 1;
-  dim3 grid((a.r + 2 * kQRows - 1) / (2 * kQRows) * splits, a.H, a.B_eff);
-  return launch_pdl(attention_kernel<D>, grid, dim3(kAttnThreads), Cfg::kSmemBytes, st, tmQ, tmK, tmV, a);
+  if (splits > 8) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((a.r + 2 * kQRows - 1) / (2 * kQRows) * splits, a.H, a.B_eff);
+  cfg.blockDim = dim3(kAttnThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;            // the key ranges of one query tile pair form a cluster
+  attr[0].val.clusterDim.x = splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, attention_kernel<D>, tmQ, tmK, tmV, a);
 }
 
-int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms, size_t scratch_bytes, int max_counters) {
+int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms) {
+  (void)D;
   const int qtiles = (r + 2 * kQRows - 1) / (2 * kQRows);
   const long long ctas = static_cast<long long>(qtiles) * H * B_eff;
   const int nkv = (L + kKeys - 1) / kKeys;
   if (ctas * 2 > num_sms || nkv < 8) return 1;            // enough CTAs already, or too few key blocks to share
   int splits = static_cast<int>(num_sms / ctas);
   if (splits > nkv / 4) splits = nkv / 4;                  // at least four key blocks per range
-  if (splits > 16) splits = 16;
-  while (splits > 1 && (static_cast<size_t>(ctas) * 2 * splits * (D + 2) * kQRows * 4 > scratch_bytes || ctas * 2 > max_counters))
-    --splits;
+  if (splits > 8) splits = 8;                              // a portable cluster
   if (splits < 2) return 1;
   const int per = (nkv + splits - 1) / splits;
   return (nkv + per - 1) / per;                            // every range gets at least one block

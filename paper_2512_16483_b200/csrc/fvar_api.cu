@@ -1065,10 +1065,9 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         if ((s = run_gemm(ctx, EPI_QKV, ctx->y_map, blk, W_QKV, ga, "qkv gemm")) != FVAR_OK) return s;
       }
       {
-        AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, ctx->split_partial,
-                    ctx->split_counters};
+        AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1};
         aa.wait_cycles = ctx->wait_cycles;
-        aa.kv_splits = attention_pick_splits(E, H, r, D, L_prev + r, ctx->num_sms, kSplitScratchBytes, kSplitCounters);
+        aa.kv_splits = attention_pick_splits(E, H, r, D, L_prev + r, ctx->num_sms);
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * (L_prev + r) * C, 4.0 * E * (L_prev + r) * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
         ctx->launched();
@@ -1092,7 +1091,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         gq.out_bf16 = ctx->q; gq.ld_out = C;
         prefetch_next(gq, blk, W_CO);
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
-        AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1, nullptr, nullptr};
+        AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1};
         aa.wait_cycles = ctx->wait_cycles;
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
@@ -1449,7 +1448,11 @@ fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B,
       !tmap_3d(&tv, Vt, L_cap, D, BH, L_cap, static_cast<uint64_t>(L_cap) * D, 64, D))
     return kfail(FVAR_EINVAL, "attention: operands must be 16-byte aligned");
   AttnArgs a{B, H, r, D, L, L_cap, 1, 0, static_cast<bf16 *>(out), 1.4426950408889634f / sqrtf(static_cast<float>(D)),
-             kernel_status_ptr(), 1, nullptr, nullptr};
+             kernel_status_ptr(), 1};
+  int dev = 0, sms = 0;
+  FK_CUDA(cudaGetDevice(&dev), "get device");
+  FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
+  a.kv_splits = attention_pick_splits(B, H, r, D, L, sms);
   if (!a.status) return kfail(FVAR_ECUDA, "attention: status word");
   FK_CUDA(launch_attention(tq, tk, tv, a, static_cast<cudaStream_t>(stream)), "attention");
   return FVAR_OK;

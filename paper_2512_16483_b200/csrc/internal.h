@@ -121,14 +121,13 @@ struct AttnArgs {
   bf16 *out;               // [B_eff * r][H * D]
   float scale_log2;        // log2(e) / sqrt(D)
   unsigned *status;
-  // split-KV (kv_splits > 1): scratch for the per-range (O, m, l) and one arrival counter per 128-row tile
+  // kv_splits > 1: the key range is split over a cluster of that many CTAs (at most 8), merged through
+  // distributed shared memory
   int kv_splits;
-  float *part;
-  int *counters;
   long long wait_cycles;   // budget of every bounded wait (0: the default)
 };
-// Number of key ranges to split an attention launch into (1 = no split), given the scratch available.
-int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms, size_t scratch_bytes, int max_counters);
+// Number of key ranges to split an attention launch into (1 = no split; at most 8, a portable cluster).
+int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms);
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                              const AttnArgs &a, cudaStream_t st);
 

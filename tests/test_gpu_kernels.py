@@ -189,10 +189,14 @@ def _cache_layout(K, V, H, D, L_cap):
     return Kc, Vt
 
 
+# The last five shapes have few (element, head, query tile) CTAs over a long cache, so the key range is split over a
+# cluster (2, 4 and 8 ranges; one and two query tiles; a ragged last range; a single query row).
 @pytest.mark.parametrize("B,H,D,r,L,L_cap", [(2, 16, 64, 256, 680, 768), (1, 4, 128, 170, 1000, 1024),
                                              (2, 2, 64, 32, 456, 768), (1, 2, 128, 300, 129, 136),
                                              (1, 1, 64, 1, 1, 8), (2, 3, 64, 130, 128, 128),
-                                             (1, 2, 64, 128, 2000, 2048)])
+                                             (1, 2, 64, 128, 2000, 2048), (1, 16, 128, 16, 6441, 6528),
+                                             (1, 16, 128, 170, 6595, 6656), (2, 4, 64, 300, 3000, 3072),
+                                             (1, 3, 128, 1, 1100, 1104), (1, 5, 64, 77, 2500, 2560)])
 def test_attention(fv, B, H, D, r, L, L_cap):
     rng = np.random.default_rng(B * 1000 + r + L)
     C = H * D
