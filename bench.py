@@ -438,9 +438,9 @@ def main():
             ctx.kv_append(k)
             fo = out if null_at[k] else fv.fvar_cfg_combine(out, LOOP_GUIDANCE)
             more = i + 1 < len(run)
-            _, nxt = ctx.scale_transition(fo, k, Ms[k + 1] if more else None)
+            _, nxt = ctx.scale_transition(fo, k, Ms[k + 1] if more else None, pairs=True)   # both branches see the same tokens
             if more:
-                tok = nxt.repeat_interleave(2, dim=0)               # both branches of a pair see the same tokens
+                tok = nxt
         if host:
             feat_host.copy_(ctx.get_feature(B // 2, Ms[-1], shp.width), non_blocking=True)
             torch.cuda.synchronize()

@@ -147,6 +147,12 @@ fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V);
  * context's stream; allocates nothing. */
 fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens);
 
+/* The same transition with the next step's tokens written for both branches of every CFG pair: next_tokens_pairs
+ * dev bf16 [2 B][M_{k+1}][C], elements 2p and 2p + 1 both hold the tokens of image p (fo and codes as above, one
+ * row set per image).  What a closed generation loop needs while the next step still runs both branches. */
+fvar_status fvar_scale_transition_pairs(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes,
+                                        void *next_tokens_pairs);
+
 /* Classifier-free guidance on the outputs of a step that ran both branches: out[p] = null + guidance *
  * (prompt - null) for the CFG pair p = elements (2p, 2p + 1) = (prompt, null prompt) of `pair`.  The paper
  * only states that VAR combines the prompt and null-prompt branches by classifier-free guidance and that

@@ -75,6 +75,7 @@ def load_library() -> ct.CDLL:
         "fvar_generate_projection": (i, [vp, i, i, i, ct.c_ulonglong]),
         "fvar_set_codebook": (i, [vp, vp, i]),
         "fvar_scale_transition": (i, [vp, vp, i, i, vp, vp]),
+        "fvar_scale_transition_pairs": (i, [vp, vp, i, i, vp, vp]),
         "fvar_get_feature": (i, [vp, vp]),
         "fvar_cfg_combine": (i, [vp, i, ll, f, vp, vp]),
         "fvar_get_projection": (i, [vp, i, i, vp, P(i)]),
@@ -124,7 +125,7 @@ def load_library() -> ct.CDLL:
 
 
 EXPORTED = ("fvar_workspace_bytes", "fvar_init", "fvar_set_cond", "fvar_set_projection", "fvar_generate_projection",
-            "fvar_get_projection", "fvar_set_codebook", "fvar_scale_transition", "fvar_get_feature", "fvar_scale_step",
+            "fvar_get_projection", "fvar_set_codebook", "fvar_scale_transition", "fvar_scale_transition_pairs", "fvar_get_feature", "fvar_scale_step",
             "fvar_scale_step_host", "fvar_scale_step_host_async", "fvar_host_sync", "fvar_kv_append", "fvar_get_indices", "fvar_get_group_output", "fvar_load_kv",
             "fvar_load_group_cache", "fvar_cache_len", "fvar_launch_count", "fvar_poll_status", "fvar_reset",
             "fvar_destroy", "fvar_last_error", "fvar_restore_loaded", "fvar_set_option", "fvar_profile_enable", "fvar_profile_read", "fvar_profile_dump",
@@ -346,13 +347,15 @@ class Fvar:
         self._codebook = Z
         self._check(self.lib.fvar_set_codebook(self.ctx, Z.data_ptr(), Z.shape[0]))
 
-    def scale_transition(self, fo: torch.Tensor, scale_idx: int, next_M: Optional[int]):
-        """fo bf16 [B][M_k][C] -> (codes int32 [B][M_k], next tokens bf16 [B][next_M][C] or None at the last scale)."""
+    def scale_transition(self, fo: torch.Tensor, scale_idx: int, next_M: Optional[int], pairs: bool = False):
+        """fo bf16 [B][M_k][C] -> (codes int32 [B][M_k], next tokens bf16 [B][next_M][C] or None at the last scale).
+        pairs: the next tokens come out as [2 B][next_M][C], every image's rows twice (both branches of its CFG pair)."""
         _dev(fo, torch.bfloat16)
         B, M, C = fo.shape
         codes = torch.empty((B, M), dtype=torch.int32, device=fo.device)
-        nxt = torch.empty((B, next_M, C), dtype=torch.bfloat16, device=fo.device) if next_M else None
-        self._check(self.lib.fvar_scale_transition(self.ctx, fo.data_ptr(), scale_idx, B, codes.data_ptr(), _ptr(nxt)))
+        nxt = torch.empty(((2 * B if pairs else B), next_M, C), dtype=torch.bfloat16, device=fo.device) if next_M else None
+        fn = self.lib.fvar_scale_transition_pairs if pairs else self.lib.fvar_scale_transition
+        self._check(fn(self.ctx, fo.data_ptr(), scale_idx, B, codes.data_ptr(), _ptr(nxt)))
         return codes, nxt
 
     def get_feature(self, B: int, M_last: int, C: int) -> torch.Tensor:

@@ -815,7 +815,7 @@ fvar_status fvar_set_codebook(fvar_ctx *ctx, const void *Z, int V) {
   return FVAR_OK;
 }
 
-fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens) {
+static fvar_status transition_impl(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens, bool dup) {
   if (!ctx) return FVAR_EINVAL;
   if (!ctx->codebook) return fail(ctx, FVAR_ESTATE, "scale_transition before set_codebook");
   const int nS = ctx->cfg.n_scales;
@@ -859,12 +859,20 @@ fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, 
   if (next_tokens) {
     const int hn = ctx->hw[2 * (scale_idx + 1)], wn = ctx->hw[2 * (scale_idx + 1) + 1];
     ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * B * hK * wK * C + 2.0 * B * hn * wn * C);
-    FV_CUDA(ctx, launch_down_area(ctx->tr_F, B, hK, wK, hn, wn, C, static_cast<bf16 *>(next_tokens), st), "down_area");
+    FV_CUDA(ctx, launch_down_area(ctx->tr_F, B, hK, wK, hn, wn, C, static_cast<bf16 *>(next_tokens), dup, st), "down_area");
     ctx->launched();
   }
   ctx->tr_scale = scale_idx;
   ctx->tr_B = B;
   return FVAR_OK;
+}
+
+fvar_status fvar_scale_transition(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens) {
+  return transition_impl(ctx, fo, scale_idx, B, codes, next_tokens, false);
+}
+
+fvar_status fvar_scale_transition_pairs(fvar_ctx *ctx, const void *fo, int scale_idx, int B, int *codes, void *next_tokens_pairs) {
+  return transition_impl(ctx, fo, scale_idx, B, codes, next_tokens_pairs, true);
 }
 
 fvar_status fvar_get_feature(fvar_ctx *ctx, float *F_out) {

@@ -177,7 +177,8 @@ cudaError_t launch_unpack_codes(const unsigned long long *best, long long n, int
 cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0, int w0, int h1, int w1, int C,
                                  bool overwrite, float *F, cudaStream_t st);
 cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st);
-cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st);
+// dup: every element is written twice, [2B][h1 * w1][C] (the two branches of a CFG pair).
+cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, bool dup, cudaStream_t st);
 // Self-test of the bounded wait: one CTA waits on an mbarrier nobody signals with a budget of `cycles`, flags the
 // status word and returns.
 cudaError_t launch_wait_selftest(long long cycles, unsigned *status, cudaStream_t st);

@@ -119,7 +119,7 @@ cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0,
 // One warp per target cell: the lanes walk the channels four float4 groups at a time (so that several
 // loads per lane are in flight), the window cell by cell inside.  C % 4 == 0.
 __global__ void __launch_bounds__(256) down_area_kernel(const float *__restrict__ F, int B, int h0, int w0, int h1, int w1,
-                                                        int C, bf16 *__restrict__ tokens) {
+                                                        int C, bf16 *__restrict__ tokens, int dup) {
   pdl_wait();
   pdl_launch_dependents();
   const int M1 = h1 * w1, lane = threadIdx.x & 31;
@@ -131,7 +131,9 @@ __global__ void __launch_bounds__(256) down_area_kernel(const float *__restrict_
   const int xa = (x * w0) / w1, xb = ((x + 1) * w0 + w1 - 1) / w1;
   const float inv = 1.0f / static_cast<float>((yb - ya) * (xb - xa));
   const float4 *src = reinterpret_cast<const float4 *>(F + static_cast<long long>(b) * h0 * w0 * C);
-  uint2 *dst = reinterpret_cast<uint2 *>(tokens + (static_cast<long long>(b) * M1 + q) * C);
+  // dup: element b is written twice, as elements 2b and 2b + 1 (both branches of a CFG pair read the same tokens)
+  uint2 *dst = reinterpret_cast<uint2 *>(tokens + (static_cast<long long>(dup ? 2 * b : b) * M1 + q) * C);
+  const long long dup_off = static_cast<long long>(M1) * C / 4;      // one element further on, in uint2 units
   const int ngroups = C / 4, row4 = C / 4;
   for (int g0 = lane; g0 < ngroups; g0 += 128) {
     float4 acc[4];
@@ -159,17 +161,18 @@ __global__ void __launch_bounds__(256) down_area_kernel(const float *__restrict_
         pk.x = *reinterpret_cast<const uint32_t *>(&o0);
         pk.y = *reinterpret_cast<const uint32_t *>(&o1);
         dst[g] = pk;
+        if (dup) dst[g + dup_off] = pk;
       }
     }
   }
 }
 
-cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, cudaStream_t st) {
+cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, bool dup, cudaStream_t st) {
   if (C % 4 != 0) return cudaErrorInvalidValue;
   const long long warps = static_cast<long long>(B) * h1 * w1;
   if (warps <= 0) return cudaSuccess;
   return launch_pdl(down_area_kernel, dim3(static_cast<unsigned>((warps + 7) / 8)), dim3(256), 0, st, F, B, h0, w0, h1, w1, C,
-                    tokens);
+                    tokens, dup ? 1 : 0);
 }
 
 // Classifier-free guidance on CFG pairs: out[p] = null + s (prompt - null) with (prompt, null) = elements

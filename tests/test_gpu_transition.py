@@ -148,3 +148,59 @@ def test_transition_at_the_infinity_shape(fv):
         np.testing.assert_allclose(got_F, F_ref, rtol=0, atol=2e-5 * (k + 1) * np.abs(Z).max())
         if k == 0:
             np.testing.assert_allclose(bf16_to_numpy(nxt[0]), n_ref, rtol=2 ** -8, atol=1e-5 * np.abs(Z).max())
+
+
+def test_closed_generation_loop_matches_oracle(fv):
+    """Algorithm 1 as a closed loop on a tiny stack, the library and the oracle each feeding themselves: a start token,
+    then for every scale step -> (CFG combination of the two branches) -> R_k = Q(F_k^o), F_k = F_{k-1} + Up(R_k),
+    next tokens = Down(F_k) -> next step.  Scales 0 and 1 run densely with both branches (guidance 3), scales 2 and 3
+    under RP + RTR on the null-prompt branch alone (teacher-forced index sets), scale 4 is skipped (Sec. 4.1: alpha = 0),
+    so the map accumulated after scale 3 is the result.  Both sides see the same interface types: the step returns
+    bf16, the combination returns bf16, the next tokens are bf16.  Codes must agree at every scale; F_k then agrees to
+    fp32 accumulation accuracy and the next tokens to one bf16 rounding."""
+    from test_gpu_step import Pair
+    shp = si.shape_tiny(n_blocks=4, blocks_per_group=2, width=128, n_heads=2, head_dim=64, ffn_dim=256, scales=(1, 2, 3, 5, 8))
+    B, V, guidance = 2, 48, 3.0
+    p = Pair(fv, shp, seed=77, B=B, std=0.05)
+    C, Ms, hw = shp.width, shp.tokens_per_scale(), shp.hw()
+    Z = si.make_codebook(77, V, C)
+    p.gpu.set_codebook(to_bf16_cuda(Z))
+    ranks = {2: [4, 5], 3: [10, 12]}
+    for k, rk in ranks.items():
+        p.set_projections(k, rk)
+    bf = lambda a: si.round_to_bf16(np.asarray(a, np.float32)).astype(np.float64)
+    start = si.make_tokens(77, 1, 1, C)
+    tok_o = np.concatenate([start, start], axis=0)                      # both branches of the pair start alike
+    tok_g = to_bf16_cuda(tok_o)
+    F_o = np.zeros((Ms[-1], C))
+    for k in range(4):
+        late, more = k in ranks, k < 3
+        if late:
+            pol = orc.Policy("lowrank_rtr", "null_only", rank_per_group=ranks[k])
+            out_o = p.oracle.scale_step(tok_o, k, pol)
+            out_g = p.gpu.scale_step(tok_g, k, mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY, rank_per_group=ranks[k],
+                                     forced_indices=p.forced_tensor(ranks[k], 1))
+            fo_o, fo_g = bf(out_o[0]), out_g                             # CFG = 0: the null-prompt branch is the output
+        else:
+            out_o = p.oracle.scale_step(tok_o, k, orc.Policy("dense", "pair"))
+            out_g = p.gpu.scale_step(tok_g, k, mode=fv.DENSE)
+            fo_o = bf(orc.cfg_combine(bf(out_o[0]), bf(out_o[1]), guidance))
+            fo_g = fv.fvar_cfg_combine(out_g, guidance)
+        p.check_ok()
+        p.gpu.kv_append(k)
+        p.oracle.kv_append(k)
+        codes_g, nxt_g = p.gpu.scale_transition(fo_g, k, Ms[k + 1] if more else None, pairs=True)
+        codes_o, F_o, nxt_o = orc.scale_transition(F_o, fo_o, Z, hw[k], hw[-1], hw[k + 1] if more else None)
+        assert np.array_equal(codes_g.cpu().numpy()[0], codes_o), (k, codes_g.cpu().numpy()[0], codes_o)
+        got_F = p.gpu.get_feature(1, Ms[-1], C).cpu().numpy()[0].astype(np.float64)
+        np.testing.assert_allclose(got_F, F_o, rtol=0, atol=2e-5 * (k + 1) * np.abs(Z).max())
+        if more:
+            assert nxt_g.shape == (2, Ms[k + 1], C) and torch.equal(nxt_g[0], nxt_g[1])       # written for both branches
+            np.testing.assert_allclose(bf16_to_numpy(nxt_g[0]), nxt_o, rtol=2 ** -8, atol=1e-5 * np.abs(Z).max())
+            tok_o = np.stack([bf(nxt_o), bf(nxt_o)])
+            tok_g = nxt_g
+        else:
+            assert nxt_g is None
+    # the skipped scale: nothing is enqueued, nothing staged, the accumulated map stands as the result
+    assert p.gpu.scale_step(tok_g, 4, mode=fv.SKIP) is None
+    assert p.gpu.poll_status() == fv.OK
