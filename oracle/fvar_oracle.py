@@ -278,6 +278,31 @@ def rtr_restore(F_r_out: np.ndarray, idx: np.ndarray, cache_up: np.ndarray) -> n
     return out
 
 
+def lls_restoration_matrix(F_r: np.ndarray, F_full: np.ndarray) -> np.ndarray:
+    """Eq. "lstsq" (Sec. 3.3 RP): the restoration matrix W in R^{M x r} that minimises || F_r^T W^T - F_full^T ||_F,
+    i.e. the least-squares map from the r-row feature F_r [r][d] back to the M-row feature F_full [M][d].  With
+    F_r of full row rank the normal equations give W = F_full F_r^T (F_r F_r^T)^-1; solved in fp64 through the
+    Cholesky factor of the r x r Gram matrix."""
+    F_r, F_full = np.asarray(F_r, dtype=np.float64), np.asarray(F_full, dtype=np.float64)
+    G = F_r @ F_r.T
+    L = np.linalg.cholesky(G)
+    P = F_full @ F_r.T                                   # [M][r]
+    Y = np.linalg.solve(L, P.T)                          # L Y = P^T
+    return np.linalg.solve(L.T, Y).T                     # L^T W^T = Y
+
+
+def lls_restore(F_r_out: np.ndarray, F_hat: np.ndarray, F_tilde: np.ndarray, Q: np.ndarray, cache_up: np.ndarray) -> np.ndarray:
+    """The LLS restoration the paper tries before RTR (Sec. 3.3 RP, Eq. "lstsq"; App. A.3; Tab. "lowrank" row 5):
+    F_k^o = W_r^o F_r^o with W_r^o ~ W_hat_r + W_r^{o,cache}.  W_hat_r restores the step's input from its projection
+    (F_tilde from F_hat = Q^T F_tilde).  W_r^{o,cache} is "obtained by solving the LLS problem" for the cached
+    counterpart feature; the paper does not name the r-row feature of that second problem -- read here as the
+    projection of the cached feature by the same Q, Q^T Up(F_{k-1}^o), restored to Up(F_{k-1}^o).  The sum of the
+    two matrices is taken as the paper writes it."""
+    W_hat = lls_restoration_matrix(F_hat, F_tilde)
+    W_cache = lls_restoration_matrix(random_projection(Q, cache_up), cache_up)
+    return (W_hat + W_cache) @ np.asarray(F_r_out, dtype=np.float64)
+
+
 def rank_from_keep_ratio(M: int, rho: float) -> int:
     return max(1, min(M, int(math.floor(rho * M + 0.5))))
 
@@ -352,8 +377,11 @@ class Policy:
     """Per-call policy of a scale step (mirrors the C ABI's keep policy)."""
 
     def __init__(self, mode: str = "dense", cfg_mode: str = "pair", keep_ratio: float = 1.0,
-                 rank_per_group: Optional[Sequence[int]] = None, forced_indices=None, sample_noise=None):
+                 rank_per_group: Optional[Sequence[int]] = None, forced_indices=None, sample_noise=None,
+                 restore: str = "rtr"):
         assert mode in ("dense", "lowrank_rtr", "skip")
+        assert restore in ("rtr", "lls")
+        self.restore = restore                    # how the M rows come back from the r rows: RTR (the method) or LLS (variant 5)
         assert cfg_mode in ("pair", "null_only")
         self.mode, self.cfg_mode = mode, cfg_mode
         self.keep_ratio, self.rank_per_group = keep_ratio, rank_per_group
@@ -455,13 +483,16 @@ class Oracle:
                     x = X
                     idx = np.arange(M, dtype=np.int32)
                 else:
-                    if pol.forced_indices is not None:
+                    if pol.restore == "lls":
+                        idx = np.zeros(0, dtype=np.int32)  # no index set: every row comes from W F_r^o
+                    elif pol.forced_indices is not None:
                         idx = np.asarray(pol.forced_indices[e][g], dtype=np.int32)
                     elif pol.sample_noise is not None:
                         idx = select_top_r(sampling_keys(row_scores(X, np.float32), pol.sample_noise[g][e]), r)
                     else:
                         idx = select_top_r(row_scores(X, np.float32), r)
                     x = random_projection(self.proj[(scale_idx, g)], X)
+                    x_hat = x
                 for blk in blocks:
                     ckv = self.cross_kv[blk][b] if self.cross else None
                     x, k, v = block_forward(x, self.ada[blk][b], self.w[blk], self.K[blk][b],
@@ -473,7 +504,8 @@ class Oracle:
                     assert self.group_cache is not None and self.cache_scale >= 0
                     up = upsample_bilinear(self.group_cache[g][b], self.hw[self.cache_scale],
                                            self.hw[scale_idx])
-                    out = rtr_restore(x, idx, up)
+                    out = (lls_restore(x, x_hat, X, self.proj[(scale_idx, g)], up) if pol.restore == "lls"
+                           else rtr_restore(x, idx, up))
                 indices[e][g] = idx
                 new_cache[g][b] = out
                 X = out

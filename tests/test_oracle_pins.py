@@ -624,3 +624,77 @@ def test_cfg_combine_end_points_and_linearity():
     np.testing.assert_allclose(orc.cfg_combine(a, b, 1.0), a, atol=1e-15)
     np.testing.assert_allclose(orc.cfg_combine(a, b, 3.0), 3.0 * a - 2.0 * b, atol=1e-14)
     np.testing.assert_allclose(orc.cfg_combine(a, a, 7.5), a, atol=1e-14)  # equal branches: guidance changes nothing
+
+
+# ----------------------------------------------------------------------------- LLS restoration (Eq. "lstsq", App. A.3)
+
+def test_lls_restoration_matrix_is_the_least_squares_solution():
+    """Against numpy's SVD-based lstsq on the transposed problem F_r^T W^T ~ F^T, and the normal-equation residual
+    property: the residual is orthogonal to the rows of F_r."""
+    rng = np.random.default_rng(41)
+    M, r, d = 37, 9, 24
+    F = rng.standard_normal((M, d))
+    F_r = rng.standard_normal((r, d))
+    W = orc.lls_restoration_matrix(F_r, F)
+    ref = np.linalg.lstsq(F_r.T, F.T, rcond=None)[0].T
+    np.testing.assert_allclose(W, ref, rtol=1e-9, atol=1e-10)
+    np.testing.assert_allclose((W @ F_r - F) @ F_r.T, 0.0, atol=1e-9)
+    # brute force on one row: no other w gives a smaller residual
+    w0, f0 = W[3], F[3]
+    base = np.linalg.norm(w0 @ F_r - f0)
+    for _ in range(50):
+        assert np.linalg.norm((w0 + 1e-3 * rng.standard_normal(r)) @ F_r - f0) >= base - 1e-12
+
+
+def test_lls_restores_exactly_what_lies_in_the_row_space():
+    """rank(F) <= r: F_hat = Q^T F spans the row space of F, so W_hat F_hat = F exactly.  r = M with Q = I: W_hat = I."""
+    rng = np.random.default_rng(42)
+    M, r, d = 40, 6, 30
+    F = rng.standard_normal((M, 5)) @ rng.standard_normal((5, d))          # rank 5 <= r ... plus one direction so F_hat has rank r
+    F = F + np.outer(rng.standard_normal(M), rng.standard_normal(d))
+    Q = rng.standard_normal((M, r)) / np.sqrt(r)
+    F_hat = orc.random_projection(Q, F)
+    W = orc.lls_restoration_matrix(F_hat, F)
+    np.testing.assert_allclose(W @ F_hat, F, rtol=1e-8, atol=1e-8)
+    F2 = rng.standard_normal((8, 20))
+    np.testing.assert_allclose(orc.lls_restoration_matrix(orc.random_projection(np.eye(8), F2), F2), np.eye(8), atol=1e-10)
+
+
+def test_lls_restore_is_the_sum_of_the_two_restorations():
+    """F_k^o = (W_hat + W^{o,cache}) F_r^o.  If the blocks were the identity (F_r^o = F_hat) and the cache equalled the
+    input, each term would restore the best rank-r fit of the input, so the result is twice that fit."""
+    rng = np.random.default_rng(43)
+    M, r, d = 30, 7, 16
+    F = rng.standard_normal((M, d))
+    Q = rng.standard_normal((M, r)) / np.sqrt(r)
+    F_hat = orc.random_projection(Q, F)
+    fit = orc.lls_restoration_matrix(F_hat, F) @ F_hat
+    np.testing.assert_allclose(orc.lls_restore(F_hat, F_hat, F, Q, F), 2.0 * fit, rtol=1e-9, atol=1e-10)
+    # linear in the block output
+    Fo1, Fo2 = rng.standard_normal((r, d)), rng.standard_normal((r, d))
+    cache = rng.standard_normal((M, d))
+    a = orc.lls_restore(Fo1, F_hat, F, Q, cache) + 2.0 * orc.lls_restore(Fo2, F_hat, F, Q, cache)
+    np.testing.assert_allclose(orc.lls_restore(Fo1 + 2.0 * Fo2, F_hat, F, Q, cache), a, rtol=1e-9, atol=1e-9)
+
+
+def test_lls_step_structure():
+    """A late step under LLS restoration: every row of the group output comes from W F_r^o (no row is a copy of the
+    upsampled cache), the cache grows by r rows per block as under RTR, and no index set is produced."""
+    shp = si.shape_tiny(n_blocks=2, blocks_per_group=1, width=64, n_heads=1, head_dim=64, ffn_dim=128, scales=(2, 3, 4))
+    w = si.make_weights(44, shp, 0.05)
+    o = orc.Oracle(w, shp.n_heads, shp.blocks_per_group, shp.hw(), shp.ln_eps)
+    o.set_cond(si.make_cond(44, 2, 64))
+    for k in (0, 1):
+        o.scale_step(si.make_tokens(44, 2, shp.tokens_per_scale()[k], 64), k, orc.Policy("dense"))
+        o.kv_append(k)
+    r = 5
+    for g in range(2):
+        o.set_projection(2, g, si.make_projection(44, 2, g, 16, r))
+    up = [orc.upsample_bilinear(o.group_cache[g][1], (3, 3), (4, 4)) for g in range(2)]
+    out = o.scale_step(si.make_tokens(44, 2, 16, 64), 2, orc.Policy("lowrank_rtr", "null_only", rank_per_group=[r, r], restore="lls"))
+    assert out.shape == (1, 16, 64) and all(len(o.last_indices[0][g]) == 0 for g in range(2))
+    for g in range(2):
+        assert np.abs(o.group_cache[g][1] - up[g]).min(axis=1).max() > 0      # no row copied from the cache
+        assert np.linalg.matrix_rank(o.group_cache[g][1], tol=1e-8) <= r       # M rows spanned by the r block-output rows
+    o.kv_append(2)
+    assert o.cache_len(0, 1) == 4 + 9 + r and o.cache_len(0, 0) == 4 + 9
