@@ -46,6 +46,7 @@ typedef enum {
 enum { FVAR_DENSE = 0, FVAR_LOWRANK_RTR = 1, FVAR_SKIP = 2 };      /* fvar_keep_policy.mode     */
 enum { FVAR_CFG_PAIR = 0, FVAR_CFG_NULL_ONLY = 1 };                /* fvar_keep_policy.cfg_mode */
 enum { FVAR_SELECT_TOPR = 0, FVAR_SELECT_SAMPLE = 1 };             /* fvar_keep_policy.select   */
+enum { FVAR_RESTORE_RTR = 0, FVAR_RESTORE_LLS = 1 };               /* fvar_keep_policy.restore  */
 
 /* Static shape of the block stack. */
 typedef struct {
@@ -89,6 +90,15 @@ typedef struct {
                                  proportional to the row score (the sampling reading of Sec. 3.3 RTR): the r
                                  largest keys s_i / E_i, E_i ~ Exp(1) given in sample_noise                     */
   const float *sample_noise;  /* dev fp32 [n_groups][B_eff][M] of Exp(1) variates (> 0) for FVAR_SELECT_SAMPLE     */
+  int restore;                /* how the M rows come back from the r rows of a FVAR_LOWRANK_RTR step.
+                                 FVAR_RESTORE_RTR (default, 0): representative token restoration, the method
+                                 (Sec. 3.3 RTR).  FVAR_RESTORE_LLS: the least-squares restoration the paper tries first
+                                 (Sec. 3.3 RP, Eq. "lstsq"; App. A.3; Tab. "lowrank" row 5): F_k^o = (W_hat + W^{o,cache})
+                                 F_r^o, W_hat the least-squares map from Q^T F back to the group's input F, W^{o,cache}
+                                 the same for the upsampled cached group output (this library's reading: its r-row
+                                 feature is its projection by the same Q).  No index set is chosen; r <= 192 per
+                                 group (FVAR_EUNSUPPORTED beyond).  fp32 arithmetic; a Gram matrix that is not
+                                 positive definite is reported as FVAR_EINVAL by fvar_poll_status.                  */
 } fvar_keep_policy;
 
 /* Bytes of device workspace fvar_init needs for this shape (0 if the shape is invalid). */

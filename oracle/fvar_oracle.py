@@ -284,6 +284,7 @@ def lls_restoration_matrix(F_r: np.ndarray, F_full: np.ndarray) -> np.ndarray:
     F_r of full row rank the normal equations give W = F_full F_r^T (F_r F_r^T)^-1; solved in fp64 through the
     Cholesky factor of the r x r Gram matrix."""
     F_r, F_full = np.asarray(F_r, dtype=np.float64), np.asarray(F_full, dtype=np.float64)
+    assert F_r.shape[0] <= min(F_full.shape), "the r-row feature cannot have full row rank"
     G = F_r @ F_r.T
     L = np.linalg.cholesky(G)
     P = F_full @ F_r.T                                   # [M][r]
@@ -297,7 +298,8 @@ def lls_restore(F_r_out: np.ndarray, F_hat: np.ndarray, F_tilde: np.ndarray, Q: 
     (F_tilde from F_hat = Q^T F_tilde).  W_r^{o,cache} is "obtained by solving the LLS problem" for the cached
     counterpart feature; the paper does not name the r-row feature of that second problem -- read here as the
     projection of the cached feature by the same Q, Q^T Up(F_{k-1}^o), restored to Up(F_{k-1}^o).  The sum of the
-    two matrices is taken as the paper writes it."""
+    two matrices is taken as the paper writes it.  Both problems need their r-row feature of full row rank, so
+    r <= min(M_{k-1}, d): bilinear upsampling does not raise the rank of the cached M_{k-1} rows."""
     W_hat = lls_restoration_matrix(F_hat, F_tilde)
     W_cache = lls_restoration_matrix(random_projection(Q, cache_up), cache_up)
     return (W_hat + W_cache) @ np.asarray(F_r_out, dtype=np.float64)

@@ -19,6 +19,7 @@ OK, EINVAL, ENOMEM, ESTATE, ECUDA, ETIMEOUT, EUNSUPPORTED = range(7)
 DENSE, LOWRANK_RTR, SKIP = 0, 1, 2
 CFG_PAIR, CFG_NULL_ONLY = 0, 1
 SELECT_TOPR, SELECT_SAMPLE = 0, 1
+RESTORE_RTR, RESTORE_LLS = 0, 1
 OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS, OPT_SKINNY_MAX_ROWS, OPT_WAIT_KCYCLES = 0, 1, 2, 3
 GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR, GEMM_SKINNY = 0, 1, 2, 3
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "rtr_fill", "convert")
@@ -50,7 +51,7 @@ class _Weights(ct.Structure):
 class _Policy(ct.Structure):
     _fields_ = [("mode", ct.c_int), ("cfg_mode", ct.c_int), ("rank_per_group", ct.POINTER(ct.c_int)),
                 ("keep_ratio", ct.c_float), ("forced_indices", ct.c_void_p), ("select", ct.c_int),
-                ("sample_noise", ct.c_void_p)]
+                ("sample_noise", ct.c_void_p), ("restore", ct.c_int)]
 
 
 _lib = None
@@ -364,8 +365,8 @@ class Fvar:
         self._check(self.lib.fvar_get_feature(self.ctx, out.data_ptr()))
         return out
 
-    def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise=None):
-        pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None, SELECT_TOPR, None)
+    def _policy(self, mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise=None, restore=RESTORE_RTR):
+        pol = _Policy(mode, cfg_mode, None, float(keep_ratio), None, SELECT_TOPR, None, int(restore))
         if sample_noise is not None:
             _dev(sample_noise, torch.float32)
             pol.select, pol.sample_noise = SELECT_SAMPLE, sample_noise.data_ptr()
@@ -387,9 +388,9 @@ class Fvar:
 
     def scale_step(self, tokens: torch.Tensor, scale_idx: int, *, mode: int = DENSE, cfg_mode: int = CFG_PAIR,
                    keep_ratio: float = 1.0, rank_per_group=None, forced_indices=None, sample_noise=None,
-                   out: Optional[torch.Tensor] = None) -> Optional[torch.Tensor]:
+                   out: Optional[torch.Tensor] = None, restore: int = RESTORE_RTR) -> Optional[torch.Tensor]:
         _dev(tokens, torch.bfloat16)
-        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise)
+        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, forced_indices, sample_noise, restore)
         if mode == SKIP:
             self._check(self.lib.fvar_scale_step(self.ctx, tokens.data_ptr(), scale_idx, ct.byref(pol), None))
             return None

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfvar.so")
 OBJDIR = os.path.join(HERE, "_build")
-SOURCES = ("gemm.cu", "gemm_pair.cu", "gemm_skinny.cu", "attention.cu", "elementwise.cu", "transition.cu", "fvar_api.cu", "no_alloc.cu", "schedule.cu")
+SOURCES = ("gemm.cu", "gemm_pair.cu", "gemm_skinny.cu", "attention.cu", "elementwise.cu", "transition.cu", "lls.cu", "fvar_api.cu", "no_alloc.cu", "schedule.cu")
 NVCC_FLAGS = os.environ.get("FVAR_NVCC_EXTRA", "").split() + ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"]
 

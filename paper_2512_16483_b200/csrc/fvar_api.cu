@@ -135,6 +135,12 @@ struct fvar_ctx {
   bf16 *kc, *vt, *ckc, *cvt, *silu_c, *y, *q, *a, *hbuf, *qt_pool;
   bf16 *xsplit[2];                     // hi / lo bf16 split of a group's input rows, [E][2][Mk][C]; groups alternate
   float *ada, *gcache, *x0, *xs, *scores, *split_partial;
+  // LLS restoration: upsampled cached group output (and its bf16 split), the two projections, G / G^-1, T and P
+  float *cup, *lls_xhat, *lls_chat, *lls_G, *lls_Ginv, *lls_T, *lls_P;
+  bf16 *csplit;
+  std::vector<CUtensorMap> csplit_map; // [scale]
+  int lls_rank_cap;                    // min(kLlsMaxRank, Mmax)
+  bool last_lls;                       // the last step restored by LLS (no index sets)
   // transition between scale steps: codebook (caller's memory), half-norms, packed arg-max words, codes and
   // the accumulated feature map F_k at the last scale's resolution
   const bf16 *codebook;
@@ -239,6 +245,7 @@ namespace {
 
 struct Layout {
   size_t status, split_partial, split_counters, kc, vt, ckc, cvt, ada, silu_c, gcache, x0, xs, y, q, a, hbuf, xsplit[2], scores, idx, inv, qt_pool, total;
+  size_t cup, csplit, lls_xhat, lls_chat, lls_G, lls_Ginv, lls_T, lls_P;
   size_t tr_hn, tr_best, tr_codes, tr_F;
   size_t hin[2], hout[2];
   std::vector<size_t> qt_off;
@@ -291,6 +298,17 @@ Layout make_layout(const fvar_cfg *c) {
   L.hbuf = take(B * Mmax * F * 2);
   L.xsplit[0] = take(B * 2 * Mk * C * 2);
   L.xsplit[1] = take(B * 2 * Mk * C * 2);
+  {
+    const size_t R = Mmax < static_cast<size_t>(kLlsMaxRank) ? Mmax : static_cast<size_t>(kLlsMaxRank);
+    L.cup = take(B * Mmax * C * 4);
+    L.csplit = take(B * 2 * Mk * C * 2);
+    L.lls_xhat = take(B * R * C * 4);
+    L.lls_chat = take(B * R * C * 4);
+    L.lls_G = take(2 * B * R * R * 4);
+    L.lls_Ginv = take(2 * B * R * R * 4);
+    L.lls_T = take(2 * B * R * C * 4);
+    L.lls_P = take(2 * B * Mmax * R * 4);
+  }
   L.scores = take(B * Mmax * 4);
   L.idx = take(G * B * Mmax * 4);
   L.inv = take(G * B * Mmax * 4);
@@ -466,6 +484,12 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->a = reinterpret_cast<bf16 *>(at(L.a)); c->hbuf = reinterpret_cast<bf16 *>(at(L.hbuf));
   c->xsplit[0] = reinterpret_cast<bf16 *>(at(L.xsplit[0])); c->xsplit[1] = reinterpret_cast<bf16 *>(at(L.xsplit[1]));
   c->scores = reinterpret_cast<float *>(at(L.scores));
+  c->cup = reinterpret_cast<float *>(at(L.cup)); c->csplit = reinterpret_cast<bf16 *>(at(L.csplit));
+  c->lls_xhat = reinterpret_cast<float *>(at(L.lls_xhat)); c->lls_chat = reinterpret_cast<float *>(at(L.lls_chat));
+  c->lls_G = reinterpret_cast<float *>(at(L.lls_G)); c->lls_Ginv = reinterpret_cast<float *>(at(L.lls_Ginv));
+  c->lls_T = reinterpret_cast<float *>(at(L.lls_T)); c->lls_P = reinterpret_cast<float *>(at(L.lls_P));
+  c->lls_rank_cap = c->Mmax < kLlsMaxRank ? c->Mmax : kLlsMaxRank;
+  c->last_lls = false;
   c->idx = reinterpret_cast<int *>(at(L.idx)); c->inv = reinterpret_cast<int *>(at(L.inv));
   c->qt_pool = reinterpret_cast<bf16 *>(at(L.qt_pool));
   c->tr_hn = reinterpret_cast<float *>(at(L.tr_hn)); c->tr_F = reinterpret_cast<float *>(at(L.tr_F));
@@ -531,6 +555,9 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   for (int k = 0; k < cfg->n_scales && ok; ++k)
     for (int t = 0; t < 2 && ok; ++t)
       ok = tmap_2d(&c->xsplit_map[k * 2 + t], c->xsplit[t], C, static_cast<size_t>(c->Bmax) * 2 * align_up(c->Mk[k], 64), C, 64);
+  c->csplit_map.resize(cfg->n_scales);
+  for (int k = 0; k < cfg->n_scales && ok; ++k)
+    ok = tmap_2d(&c->csplit_map[k], c->csplit, C, static_cast<size_t>(c->Bmax) * 2 * align_up(c->Mk[k], 64), C, 64);
   c->kmap.resize(nb); c->vmap.resize(nb); c->ckmap.resize(nb); c->cvmap.resize(nb);
   const int BH = c->Bmax * c->H, D = c->D;
   for (int b = 0; b < nb && ok; ++b) {
@@ -566,7 +593,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
     c->host_pipe_ok = cudaEventCreateWithFlags(&c->ev_in[s2], cudaEventDisableTiming) == cudaSuccess &&
                       cudaEventCreateWithFlags(&c->ev_cmp[s2], cudaEventDisableTiming) == cudaSuccess &&
                       cudaEventCreateWithFlags(&c->ev_out[s2], cudaEventDisableTiming) == cudaSuccess;
-  if (gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || gemm_skinny_prepare() != cudaSuccess ||
+  if (lls_prepare() != cudaSuccess || gemm_prepare() != cudaSuccess || gemm_pair_prepare() != cudaSuccess || gemm_skinny_prepare() != cudaSuccess ||
       attention_prepare() != cudaSuccess)
     return destroy_fail(FVAR_ECUDA, "kernel attribute set-up failed");
   c->max_clusters = gemm_pair_max_clusters();
@@ -933,6 +960,8 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
   if (pol->select != FVAR_SELECT_TOPR && pol->select != FVAR_SELECT_SAMPLE) return fail(ctx, FVAR_EINVAL, "scale_step: bad select");
   const bool sampled = pol->select == FVAR_SELECT_SAMPLE;
   if (sampled && !pol->sample_noise) return fail(ctx, FVAR_EINVAL, "scale_step: sampled selection needs sample_noise");
+  if (pol->restore != FVAR_RESTORE_RTR && pol->restore != FVAR_RESTORE_LLS) return fail(ctx, FVAR_EINVAL, "scale_step: bad restore");
+  const bool lls = pol->mode == FVAR_LOWRANK_RTR && pol->restore == FVAR_RESTORE_LLS;
   const bool null_only = pol->cfg_mode == FVAR_CFG_NULL_ONLY;
   if (null_only && (ctx->B % 2)) return fail(ctx, FVAR_EINVAL, "scale_step: null-only needs an even batch");
   if (!null_only && ctx->null_only_seen) return fail(ctx, FVAR_ESTATE, "scale_step: pair step after a null-only step");
@@ -956,6 +985,9 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
       r_max = rank[g] > r_max ? rank[g] : r_max;
       if (ctx->qt_r[static_cast<size_t>(scale_idx) * G + g] != rank[g])
         return fail(ctx, FVAR_ESTATE, "scale_step: no projection of this rank set for a group");
+      if (lls && rank[g] > ctx->lls_rank_cap) return fail(ctx, FVAR_EUNSUPPORTED, "scale_step: LLS restoration takes ranks up to 192");
+      if (lls && ctx->cache_scale >= 0 && rank[g] > ctx->Mk[ctx->cache_scale])
+        return fail(ctx, FVAR_EINVAL, "scale_step: LLS restoration needs r <= the tokens of the cached scale (the upsampled cache has no higher rank)");
     }
     for (int blk = g * bpg; blk < (g + 1) * bpg; ++blk)
       if (ctx->len[blk] + rank[g] > ctx->L_cap) return fail(ctx, FVAR_ESTATE, "scale_step: KV cache is full");
@@ -1007,7 +1039,13 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         FV_CUDA(ctx, cudaStreamWaitEvent(ctx->cap_st2, ctx->ev_fork, 0), "fork wait");
         side = ctx->cap_st2;
       }
-      if (pol->forced_indices) {
+      if (lls) {
+        // LLS restoration: no index set; the whole upsampled cache (Eq. "upcache") and its bf16 split, for its own
+        // projection and restoration matrix
+        ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M) + h0 * w0) + 4.0 * E * M * C, side);
+        FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), ctx->cup, E, bmul, boff, h0, w0, h1, w1, C, nullptr, ctx->csplit, Mk, side), "cache upsample");
+        ctx->launched(side);
+      } else if (pol->forced_indices) {
         ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 4.0 * E * (M + 2.0 * r), side);
         FV_CUDA(ctx, launch_copy_indices(pol->forced_indices + static_cast<size_t>(g) * E * r_max, E, M, r, r_max, idx_g,
                                          inv_g, ctx->status, side), "copy_indices");
@@ -1021,10 +1059,12 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         FV_CUDA(ctx, launch_select_topr(ctx->scores, E, M, r, idx_g, inv_g, side), "select_topr");
         ctx->launched(side);
       }
-      // restoration fill: rows outside the index set, from the upsampled cache of the previous scale
-      ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M, side);
-      FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, next_split, Mk, side), "rtr_fill");
-      ctx->launched(side);
+      if (!lls) {
+        // restoration fill: rows outside the index set, from the upsampled cache of the previous scale
+        ctx->prof_begin(FVAR_KCLASS_RTR_FILL, 0.0, 4.0 * E * C * (static_cast<double>(M - r) + h0 * w0) + 4.0 * E * M, side);
+        FV_CUDA(ctx, launch_rtr_fill(ctx->gslot(prev_slot, g), gout, E, bmul, boff, h0, w0, h1, w1, C, inv_g, next_split, Mk, side), "rtr_fill");
+        ctx->launched(side);
+      }
       if (forked) FV_CUDA(ctx, cudaEventRecord(ctx->ev_join, side), "join record");
       // random projection: xs[e] = Qt * X[e]  (r x M times M x C), batched over e.  The reduction runs over the hi
       // and lo bf16 parts of X ([Qt | Qt] against [hi ; lo]); X's rows are read in place as an MN-major operand.
@@ -1033,7 +1073,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
       ga.a_batch_rows = 0;
       ga.b_batch_rows = 2 * Mk;
       ga.w_mn_major = 1;
-      ga.out_f32 = ctx->xs;
+      ga.out_f32 = lls ? ctx->lls_xhat : ctx->xs;   // LLS keeps the projection: the blocks work on a copy of their own
       ga.ld_out = C;
       ga.status = ctx->status;
       ga.wait_cycles = ctx->wait_cycles;
@@ -1047,7 +1087,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
     for (int t = 0; t < bpg; ++t) {
       const int blk = g * bpg + t;
       const bool first_dense = (t == 0) && !late, last = (t == bpg - 1);
-      const float *in_ptr = first_dense ? X_in : ctx->xs;
+      const float *in_ptr = first_dense ? X_in : ((lls && late && t == 0) ? ctx->lls_xhat : ctx->xs);
       const RowMap in_map = first_dense ? bmap : smap;
       const float *ada = ctx->ada + blk * ada_blk;
       const int L_prev = ctx->len[blk];
@@ -1127,7 +1167,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         ga.rows_per_batch = r; ga.bmul = bmul; ga.boff = boff;
         ga.resid = ctx->xs; ga.rmap = smap; ga.ld_out = C;
         ga.gate = ada + 5 * C; ga.gate_stride = 6 * C;
-        if (last) {
+        if (last && !(lls && late)) {
           if (forked) FV_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0), "join wait");
           ga.out_f32 = gout; ga.omap = bmap;
           ga.scatter = late ? idx_g : nullptr;
@@ -1139,6 +1179,50 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         if ((s = run_gemm(ctx, EPI_RESID, ctx->h_map, blk, W_FC2, ga, "fc2 gemm")) != FVAR_OK) return s;
       }
       ctx->staged[blk] = r;
+    }
+    if (lls && late) {
+      // F_k^o = (W_hat + W^{o,cache}) F_r^o (Eq. "lstsq", App. A.3) as P1 (G1^-1 F_r^o) + P2 (G2^-1 F_r^o) with
+      // G1 = F_hat F_hat^T, P1 = F F_hat^T for the group's input F and its projection F_hat, and G2, P2 the same for
+      // the upsampled cached output and its projection.  fp32 throughout.
+      if (forked) FV_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0), "join wait");
+      {
+        GemmArgs ga = gemm_args(r, C, Mk + M);               // projection of the upsampled cache by the same Q
+        ga.nbatch = E; ga.b_batch_rows = 2 * Mk; ga.w_mn_major = 1;
+        ga.out_f32 = ctx->lls_chat; ga.ld_out = C;
+        ga.status = ctx->status; ga.wait_cycles = ctx->wait_cycles;
+        const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, Mk + M, ctx->num_sms);
+        ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + 2.0 * E * M * C) + 4.0 * E * r * C);
+        FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g], ctx->csplit_map[scale_idx], ga,
+                                 ctx->num_sms, st), "cache projection gemm");
+        ctx->launched();
+      }
+      const long long rc = static_cast<long long>(r) * C, rr = static_cast<long long>(r) * r, mc = static_cast<long long>(M) * C,
+                      mr = static_cast<long long>(M) * r;
+      auto sg = [&](bool tb, const float *A, const float *Bm, float *O, int m, int n, int k, long long lda, long long ldb, long long ldo,
+                    long long ao, long long as, long long bo, long long bs, long long oo, long long os, bool acc, const char *what) -> fvar_status {
+        ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * m * n * k * E, 4.0 * E * (static_cast<double>(m) * k + static_cast<double>(n) * k + static_cast<double>(m) * n));
+        FV_CUDA(ctx, launch_sgemm(tb, A, Bm, O, m, n, k, lda, ldb, ldo, ao, as, bo, bs, oo, os, E, acc, st), what);
+        ctx->launched();
+        return FVAR_OK;
+      };
+      float *G1 = ctx->lls_G, *G2 = ctx->lls_G + E * rr, *I1 = ctx->lls_Ginv, *I2 = ctx->lls_Ginv + E * rr;
+      float *T1 = ctx->lls_T, *T2 = ctx->lls_T + E * rc, *P1 = ctx->lls_P, *P2 = ctx->lls_P + E * mr;
+      if ((s = sg(true, ctx->lls_xhat, ctx->lls_xhat, G1, r, r, C, C, C, r, 0, rc, 0, rc, 0, rr, false, "gram 1")) != FVAR_OK) return s;
+      if ((s = sg(true, ctx->lls_chat, ctx->lls_chat, G2, r, r, C, C, C, r, 0, rc, 0, rc, 0, rr, false, "gram 2")) != FVAR_OK) return s;
+      ctx->prof_begin(FVAR_KCLASS_CONVERT, 2.0 * E * rr * r, 16.0 * E * rr);
+      FV_CUDA(ctx, launch_chol_inverse(ctx->lls_G, ctx->lls_Ginv, r, 2 * E, ctx->status, st), "gram inverse");
+      ctx->launched();
+      if ((s = sg(false, I1, ctx->xs, T1, r, C, r, r, C, C, 0, rr, 0, rc, 0, rc, false, "T1")) != FVAR_OK) return s;
+      if ((s = sg(false, I2, ctx->xs, T2, r, C, r, r, C, C, 0, rr, 0, rc, 0, rc, false, "T2")) != FVAR_OK) return s;
+      if ((s = sg(true, X_in, ctx->lls_xhat, P1, M, r, C, C, C, r, boff * mc, bmul * mc, 0, rc, 0, mr, false, "P1")) != FVAR_OK) return s;
+      if ((s = sg(true, ctx->cup, ctx->lls_chat, P2, M, r, C, C, C, r, boff * mc, bmul * mc, 0, rc, 0, mr, false, "P2")) != FVAR_OK) return s;
+      if ((s = sg(false, P1, T1, gout, M, C, r, r, C, C, 0, mr, 0, rc, boff * mc, bmul * mc, false, "restore 1")) != FVAR_OK) return s;
+      if ((s = sg(false, P2, T2, gout, M, C, r, r, C, C, 0, mr, 0, rc, boff * mc, bmul * mc, true, "restore 2")) != FVAR_OK) return s;
+      if (next_split) {
+        ctx->prof_begin(FVAR_KCLASS_CONVERT, 0.0, 8.0 * E * mc);
+        FV_CUDA(ctx, launch_split_rows(gout, boff * mc, bmul * mc, E, M, C, next_split, Mk, st), "split rows");
+        ctx->launched();
+      }
     }
     X_in = gout;
     ctx->last_rank[g] = r;
@@ -1171,7 +1255,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
   } else if (ctx->use_graphs && !ctx->prof_on && !pol->forced_indices) {
     std::string key;
     auto put = [&](long long v) { key.append(reinterpret_cast<const char *>(&v), sizeof(v)); };
-    put(scale_idx); put(B); put(E); put(prev_slot); put(cur_slot); put(ctx->cache_scale);
+    put(scale_idx); put(B); put(E); put(prev_slot); put(cur_slot); put(ctx->cache_scale); put(lls ? 1 : 0);
     put(sampled ? static_cast<long long>(reinterpret_cast<uintptr_t>(pol->sample_noise)) : 0);
     for (int g = 0; g < G; ++g) put(rank[g]);
     for (int blk = 0; blk < ctx->cfg.n_blocks; ++blk) put(ctx->len[blk]);
@@ -1219,6 +1303,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
   ctx->staged_scale = scale_idx;
   ctx->last_scale = scale_idx;
   ctx->last_E = E; ctx->last_M = M;
+  ctx->last_lls = lls;
   if (null_only) ctx->null_only_seen = 1;
   return FVAR_OK;
 }
@@ -1309,7 +1394,7 @@ fvar_status fvar_kv_append(fvar_ctx *ctx, int scale_idx) {
 fvar_status fvar_get_indices(fvar_ctx *ctx, int group, int *idx_dev, int *count_host) {
   if (!ctx) return FVAR_EINVAL;
   if (group < 0 || group >= ctx->G || !idx_dev || !count_host) return fail(ctx, FVAR_EINVAL, "get_indices: bad arguments");
-  if (ctx->last_scale < 0 || ctx->last_rank[group] <= 0 || ctx->last_rank[group] >= ctx->last_M)
+  if (ctx->last_scale < 0 || ctx->last_lls || ctx->last_rank[group] <= 0 || ctx->last_rank[group] >= ctx->last_M)
     return fail(ctx, FVAR_ESTATE, "get_indices: the last step did not select rows for this group");
   const int r = ctx->last_rank[group];
   FV_CUDA(ctx, cudaMemcpyAsync(idx_dev, ctx->idx + static_cast<size_t>(group) * ctx->Bmax * ctx->Mmax,

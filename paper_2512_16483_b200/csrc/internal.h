@@ -179,6 +179,18 @@ cudaError_t launch_up_accumulate(const bf16 *Z, const int *codes, int B, int h0,
 cudaError_t launch_cfg_combine(const bf16 *pair, int pairs, long long per_elem, float s, bf16 *out, cudaStream_t st);
 // dup: every element is written twice, [2B][h1 * w1][C] (the two branches of a CFG pair).
 cudaError_t launch_down_area(const float *F, int B, int h0, int w0, int h1, int w1, int C, bf16 *tokens, bool dup, cudaStream_t st);
+// LLS restoration (lls.cu): fp32 products, the inverse of an r x r Gram matrix through its Cholesky factor, and the
+// two-term bf16 split of fp32 rows.  Ranks up to kLlsMaxRank (the factor lives in one CTA's shared memory).
+constexpr int kLlsMaxRank = 192;
+cudaError_t lls_prepare();
+// out[z] (+)= A[z] B[z]^T (trans_b: B stored [n][k]) or A[z] B[z] (B stored [k][n]); pitches and batch strides in floats.
+cudaError_t launch_sgemm(bool trans_b, const float *A, const float *B, float *out, int m, int n, int k, long long lda, long long ldb,
+                         long long ldo, long long a_off, long long a_stride, long long b_off, long long b_stride, long long o_off,
+                         long long o_stride, int batch, bool accumulate, cudaStream_t st);
+cudaError_t launch_chol_inverse(const float *G, float *Ginv, int r, int count, unsigned *status, cudaStream_t st);
+cudaError_t launch_split_rows(const float *x, long long x_off, long long x_stride, int E, int M, int C, bf16 *xsplit, int mk,
+                              cudaStream_t st);
+
 // Self-test of the bounded wait: one CTA waits on an mbarrier nobody signals with a budget of `cycles`, flags the
 // status word and returns.
 cudaError_t launch_wait_selftest(long long cycles, unsigned *status, cudaStream_t st);

@@ -8,7 +8,7 @@ import torch
 
 import synth_inputs as si
 from oracle import fvar_oracle as orc
-from helpers import assert_close, assert_out_close, bf16_to_numpy, to_bf16_cuda, weights_to_cuda
+from helpers import assert_close, assert_out_close, bf16_to_numpy, rel_err, to_bf16_cuda, weights_to_cuda
 
 pytestmark = pytest.mark.gpu
 
@@ -492,3 +492,69 @@ def test_pipelined_host_entry_point_matches_the_synchronous_one(fv):
     for a, b in zip(results["sync"], results["async"]):
         assert torch.equal(a, b)
     assert float(results["async"][-1].float().abs().sum()) > 0
+
+
+# ----------------------------------------------------------------------------- LLS restoration (Eq. "lstsq", App. A.3)
+
+@pytest.mark.parametrize("r,cfg", [(32, "pair"), (128, "null_only"), (160, "pair")])
+def test_lls_restoration_step(fv, r, cfg):
+    """One VAR-d16-shaped block group (two blocks) at the last scale with the rows restored by the least-squares
+    matrices instead of RTR: F_k^o = (W_hat + W^{o,cache}) F_r^o, against the oracle's fp64 solve, at the block-output
+    bar (the restoration is linear in the block output and runs in fp32; measured 0.5e-2 .. 1.4e-2 x RMS)."""
+    shp = si.shape_var_d16(n_blocks=2, blocks_per_group=2)
+    B, k, M = 2, 9, 256
+    p = Pair(fv, shp, seed=120 + r, B=B)
+    p.prefill(k)
+    p.set_projections(k, [r])
+    toks = si.make_tokens(120 + r, B, M, 1024, "spread")
+    ref = p.oracle.scale_step(toks, k, orc.Policy("lowrank_rtr", cfg, rank_per_group=[r], restore="lls"))
+    out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY if cfg == "null_only" else fv.CFG_PAIR,
+                           rank_per_group=[r], restore=fv.RESTORE_LLS)
+    p.check_ok()
+    els = [1] if cfg == "null_only" else [0, 1]
+    g32 = p.gpu.get_group_output(0, M).cpu().numpy()[els]
+    e, c = rel_err(g32, np.stack([p.oracle.group_cache[0][b] for b in els]))
+    print("LLS r=%d %s: max-abs/RMS %.3e cosine %.6f" % (r, cfg, e, c))
+    assert e <= 2e-2 and c >= 0.999, (e, c)
+    assert_out_close(bf16_to_numpy(out), ref, what="LLS step r=%d" % r)
+    with pytest.raises(fv.FvarError):
+        p.gpu.get_indices(0, len(els), M)                   # LLS chooses no index set
+    p.gpu.kv_append(k)
+    p.oracle.kv_append(k)
+    assert p.gpu.cache_len(1) == 424 + r == p.oracle.cache_len(1, 1)
+    if r == 160:                                            # the upsampled 13 x 13 cache has rank <= 169 < 170
+        p.gpu.restore_loaded()
+        p.set_projections(k, [170])
+        with pytest.raises(fv.FvarError) as ei:
+            p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, rank_per_group=[170], restore=fv.RESTORE_LLS)
+        assert ei.value.status == fv.EINVAL
+
+
+def test_lls_restoration_two_groups_and_limits(fv):
+    """Two block groups in sequence (the second projects the first one's restored rows), and the rank limit.  An LLS
+    group's output is spanned by its r block-output rows, so the next group's rank may not be larger (its projection
+    would not have full row rank): ranks 40 then 24."""
+    shp = si.shape_tiny(n_blocks=2, blocks_per_group=1, width=128, n_heads=2, head_dim=64, ffn_dim=256, scales=(2, 4, 8, 16))
+    B = 2
+    p = Pair(fv, shp, seed=130, B=B, std=0.05)
+    Ms = shp.tokens_per_scale()
+    for k in (0, 1, 2):
+        toks = si.make_tokens(130, B, Ms[k], 128)
+        _step_both(p, toks, k, mode=fv.DENSE)
+        p.gpu.kv_append(k)
+        p.oracle.kv_append(k)
+    ranks = [40, 24]
+    p.set_projections(3, ranks)
+    toks = si.make_tokens(130, B, 256, 128, "spread")
+    ref = p.oracle.scale_step(toks, 3, orc.Policy("lowrank_rtr", "pair", rank_per_group=ranks, restore="lls"))
+    out = p.gpu.scale_step(to_bf16_cuda(toks), 3, mode=fv.LOWRANK_RTR, rank_per_group=ranks, restore=fv.RESTORE_LLS)
+    p.check_ok()
+    for g in range(2):
+        e, c = rel_err(p.gpu.get_group_output(g, 256).cpu().numpy(), np.stack(p.oracle.group_cache[g]))
+        print("LLS group %d: max-abs/RMS %.3e cosine %.6f" % (g, e, c))
+        assert e <= 2e-2 * np.sqrt(g + 1.0) and c >= 0.999, (g, e, c)
+    assert_out_close(bf16_to_numpy(out), ref, what="LLS two groups", max_rel=2e-2 * np.sqrt(2.0))
+    p.set_projections(3, [200, 24])
+    with pytest.raises(fv.FvarError) as ei:
+        p.gpu.scale_step(to_bf16_cuda(toks), 3, mode=fv.LOWRANK_RTR, rank_per_group=[200, 24], restore=fv.RESTORE_LLS)
+    assert ei.value.status == fv.EUNSUPPORTED
