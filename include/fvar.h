@@ -239,10 +239,12 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx);
  * not depend on timing.  When allowed, the picker splits only reductions of K >= 4096 whose tiles would
  * leave more than half of the SMs idle.  Measured: +2 % on the Infinity-shaped late scales, -5 % on the
  * VAR-d16 ones, hence off by default.
- * FVAR_OPT_SKINNY_MAX_ROWS (default 64; 0 .. 512): GEMMs of a step with at most this many rows
- * R = B_eff * r take the weight-streaming form (the weights are the M side of the MMA, the K range of a
- * 128-feature tile is spread over a thread-block cluster that reduces through distributed shared memory),
- * which is bound by reading the weights once; 0 never uses it.
+ * FVAR_OPT_SKINNY_MAX_ROWS (default 512; 0 .. 512): cap on the rows R = B_eff * r up to which a GEMM of the
+ * step may take the weight-streaming form (the library's own rule picks it per GEMM: up to 32 rows for wide
+ * outputs, up to 128 / 336 rows for outputs of at most 2048 features with a short / long reduction).  In that
+ * form the weights are the M side of the MMA and the K range of a 128-feature tile is spread over a
+ * thread-block cluster that reduces through distributed shared memory; it is bound by reading the weights
+ * once.  0 never uses it.
  * FVAR_OPT_WAIT_KCYCLES (default 0 = about half a second): budget, in thousands of clock cycles, of every
  * bounded wait inside the step's kernels; a wait that runs out sets FVAR_ETIMEOUT (fvar_poll_status). */
 enum { FVAR_OPT_CUDA_GRAPHS = 0, FVAR_OPT_GEMM_MAX_SPLITS = 1, FVAR_OPT_SKINNY_MAX_ROWS = 2, FVAR_OPT_WAIT_KCYCLES = 3 };

@@ -357,7 +357,7 @@ fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk
 // A operand from one of the library's activation buffers: a single row tile takes the shortest box
 // that covers its rows.
 fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int blk, int wid, GemmArgs &g, const char *what) {
-  if (g.nbatch == 1 && g.R <= ctx->skinny_max_rows && gemm_skinny_supported(epi, g.R, g.N, g.K)) {
+  if (g.nbatch == 1 && g.R <= ctx->skinny_max_rows && g.R <= gemm_skinny_row_limit(g.N, g.K) && gemm_skinny_supported(epi, g.R, g.N, g.K)) {
     // few rows: bound by streaming the weights once, so the weights take the M side of the MMA and the K range
     // of every 128-feature tile is spread over a cluster (gemm_skinny.cu)
     const int S = gemm_skinny_pick_splits(g.N, g.K, 0);
@@ -581,7 +581,7 @@ fvar_status fvar_init(const fvar_weights *weights, const fvar_cfg *cfg, void *wo
   c->loaded_len = -1; c->loaded_cache_scale = -1;
   c->prof_on = false; c->ev_used = 0;
   c->max_splits = 1;
-  c->skinny_max_rows = 64;
+  c->skinny_max_rows = 512;
   c->wait_cycles = 0;
   c->use_graphs = cudaStreamCreateWithFlags(&c->cap_st, cudaStreamNonBlocking) == cudaSuccess &&
                   cudaStreamCreateWithFlags(&c->cap_st2, cudaStreamNonBlocking) == cudaSuccess &&

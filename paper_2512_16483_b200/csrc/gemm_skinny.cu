@@ -366,6 +366,15 @@ bool gemm_skinny_supported(int epi, int R, int N, int K) {
   return epi != EPI_ARGMAX && R >= 1 && R <= 512 && N % 8 == 0 && K % 8 == 0 && N >= 8;
 }
 
+// Up to how many rows the weight-streaming form beats the row-tiled kernels (measured on B200, Infinity-2B-shaped
+// GEMMs): with few output features the row-tiled kernels have too few tiles to fill the SMs and each CTA walks all
+// of K, so the K split over a cluster wins up to a few hundred rows, longer for a long reduction; with many
+// features the row-tiled kernels already cover the SMs and win from 64 rows on.
+int gemm_skinny_row_limit(int N, int K) {
+  if (N <= 2048) return K >= 4096 ? 336 : 128;
+  return 32;
+}
+
 // K ranges per 128-feature tile: the split whose slowest CTA walks the fewest K blocks, waves of resident
 // clusters counted; among equals the smallest.  forced > 0 takes that split when it is launchable.
 int gemm_skinny_pick_splits(int N, int K, int forced) {

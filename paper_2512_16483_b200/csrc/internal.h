@@ -104,6 +104,7 @@ GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_cluster
 // a 128-feature tile is split over a cluster of `splits` CTAs that reduce through distributed shared memory.
 // tmA: box {64, a.sk_rp} over the activation rows; tmW: box {64, 128} over the weight rows.
 bool gemm_skinny_supported(int epi, int R, int N, int K);
+int gemm_skinny_row_limit(int N, int K);                      // rows up to which this form is the faster one
 int gemm_skinny_pick_splits(int N, int K, int forced);      // 0: not launchable on this device
 void gemm_skinny_shape(GemmArgs &a);      // needs a.R, a.K and a.splits
 bool gemm_skinny_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows, int nk);
