@@ -75,7 +75,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int kv_per = (nkv_total + splits - 1) / splits;
   const int jb0 = sp * kv_per;                                    // first key block of this CTA
   const int nkv = min(kv_per, nkv_total - jb0);                   // >= 1: the host sizes splits so
-  const int ntiles = (p.r - qt * 2 * kQRows > kQRows) ? 2 : 1;     // query tiles this CTA really has
+  const int tpc = p.tiles_per_cta == 1 ? 1 : 2;                   // query tiles a CTA takes: two, or one when CTAs are scarce
+  const int q0 = qt * tpc * kQRows;                               // first query row of this CTA within its element
+  const int ntiles = (tpc == 2 && p.r - q0 > kQRows) ? 2 : 1;     // query tiles this CTA really has
 
   if (threadIdx.x == 0) {
     abort_flag = 0;
@@ -111,7 +113,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (lane == 0) {
       // ---------------------------------------------------------------- TMA producer
       mbar_expect_tx(q_full, ntiles * Cfg::kTileBytes);
-      const int qrow0 = e * p.r + qt * 2 * kQRows;
+      const int qrow0 = e * p.r + q0;
       for (int t = 0; t < ntiles; ++t)
 #pragma unroll
         for (int a = 0; a < D / 64; ++a)
@@ -303,7 +305,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       final_ok = ok && __all_sync(0xffffffffu, mbar_wait(o_full(t), (nkv - 1) & 1u, p.status, &abort_flag, wb));
       if (final_ok && splits == 1) {
         tc_fence_after();
-        const int rib = qt * 2 * kQRows + t * kQRows + row_local;
+        const int rib = q0 + t * kQRows + row_local;
         bf16 *dst = p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D;
         const float inv_l = 1.0f / l_run;
 #pragma unroll 1
@@ -367,7 +369,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       const float c = p.scale_log2;
       for (int tt = 0; tt < ntiles; ++tt) {
-        const int rows_valid = min(kQRows, p.r - qt * 2 * kQRows - tt * kQRows);
+        const int rows_valid = min(kQRows, p.r - q0 - tt * kQRows);
         const int rpr = (rows_valid + splits - 1) / splits;        // this CTA merges rows [lo, hi) of the tile
         const int lo = sp * rpr, hi = min(rows_valid, lo + rpr);
         for (int row = lo + st / G; row < hi; row += 256 / G) {
@@ -388,7 +390,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
               o.x = fmaf(w, v.x, o.x); o.y = fmaf(w, v.y, o.y); o.z = fmaf(w, v.z, o.z); o.w = fmaf(w, v.w, o.w);
             }
           const float inv_l = 1.0f / l_all;
-          const int rib = qt * 2 * kQRows + tt * kQRows + row;
+          const int rib = q0 + tt * kQRows + row;
           __nv_bfloat162 h0 = __floats2bfloat162_rn(o.x * inv_l, o.y * inv_l), h1 = __floats2bfloat162_rn(o.z * inv_l, o.w * inv_l);
           *reinterpret_cast<uint2 *>(p.out + (static_cast<long long>(e) * p.r + rib) * (p.H * D) + h * D + d4) =
               make_uint2(*reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1));
@@ -432,7 +434,8 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   const int splits = a.kv_splits > 1 ? a.kv_splits : 1;
   if (splits > 8) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((a.r + 2 * kQRows - 1) / (2 * kQRows) * splits, a.H, a.B_eff);
+  const int rows_cta = (a.tiles_per_cta == 1 ? 1 : 2) * kQRows;
+  cfg.gridDim = dim3((a.r + rows_cta - 1) / rows_cta * splits, a.H, a.B_eff);
   cfg.blockDim = dim3(kAttnThreads);
   cfg.dynamicSmemBytes = Cfg::kSmemBytes;
   cfg.stream = st;
@@ -448,18 +451,28 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
   return cudaLaunchKernelEx(&cfg, attention_kernel<D>, tmQ, tmK, tmV, a);
 }
 
-int attention_pick_splits(int B_eff, int H, int r, int D, int L, int num_sms) {
-  (void)D;
-  const int qtiles = (r + 2 * kQRows - 1) / (2 * kQRows);
-  const long long ctas = static_cast<long long>(qtiles) * H * B_eff;
+// Launch shape of an attention call: query tiles per CTA (two: each K / V block feeds two tiles, the softmax of one
+// overlapping the MMAs of the other; one: twice the CTAs when they would not fill the SMs) and key ranges per query
+// tile group (a cluster of at most 8 CTAs, each range at least four key blocks long).
+void attention_plan(int B_eff, int H, int r, int L, int num_sms, int *tiles_per_cta, int *kv_splits) {
   const int nkv = (L + kKeys - 1) / kKeys;
-  if (ctas * 2 > num_sms || nkv < 8) return 1;            // enough CTAs already, or too few key blocks to share
-  int splits = static_cast<int>(num_sms / ctas);
-  if (splits > nkv / 4) splits = nkv / 4;                  // at least four key blocks per range
-  if (splits > 8) splits = 8;                              // a portable cluster
-  if (splits < 2) return 1;
-  const int per = (nkv + splits - 1) / splits;
-  return (nkv + per - 1) / per;                            // every range gets at least one block
+  const long long pairs = static_cast<long long>((r + 2 * kQRows - 1) / (2 * kQRows)) * H * B_eff;
+  const long long singles = static_cast<long long>((r + kQRows - 1) / kQRows) * H * B_eff;
+  *tiles_per_cta = (r > kQRows && pairs * 2 <= num_sms) ? 1 : 2;
+  const long long ctas = *tiles_per_cta == 1 ? singles : pairs;
+  int splits = 1;
+  if (ctas * 2 <= num_sms && nkv >= 8) {
+    splits = static_cast<int>(num_sms / ctas);
+    if (splits > nkv / 4) splits = nkv / 4;                  // at least four key blocks per range (measured: finer is slower)
+    if (splits > 8) splits = 8;
+    if (splits >= 2) {
+      const int per = (nkv + splits - 1) / splits;
+      splits = (nkv + per - 1) / per;                        // every range gets at least one block
+    } else {
+      splits = 1;
+    }
+  }
+  *kv_splits = splits;
 }
 
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,

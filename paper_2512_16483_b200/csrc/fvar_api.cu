@@ -1115,7 +1115,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
       {
         AttnArgs aa{E, H, r, D, L_prev + r, ctx->L_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1};
         aa.wait_cycles = ctx->wait_cycles;
-        aa.kv_splits = attention_pick_splits(E, H, r, D, L_prev + r, ctx->num_sms);
+        attention_plan(E, H, r, L_prev + r, ctx->num_sms, &aa.tiles_per_cta, &aa.kv_splits);
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * (L_prev + r) * C, 4.0 * E * (L_prev + r) * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->kmap[blk], ctx->vmap[blk], aa, st), "attention");
         ctx->launched();
@@ -1141,6 +1141,7 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
         if ((s = run_gemm(ctx, EPI_BF16, ctx->y_map, blk, W_CQ, gq, "cross q gemm")) != FVAR_OK) return s;
         AttnArgs aa{E, H, r, D, ctx->cfg.ctx_len, ctx->ctx_cap, bmul, boff, ctx->a, scale_log2, ctx->status, 1};
         aa.wait_cycles = ctx->wait_cycles;
+        attention_plan(E, H, r, ctx->cfg.ctx_len, ctx->num_sms, &aa.tiles_per_cta, &aa.kv_splits);
         ctx->prof_begin(FVAR_KCLASS_ATTENTION, 4.0 * E * r * ctx->cfg.ctx_len * C, 4.0 * E * ctx->cfg.ctx_len * C + 4.0 * E * r * C);
         FV_CUDA(ctx, launch_attention(ctx->q_map, ctx->ckmap[blk], ctx->cvmap[blk], aa, st), "cross attention");
         ctx->launched();
@@ -1545,7 +1546,7 @@ fvar_status fvar_attention(const void *q, const void *Kc, const void *Vt, int B,
   int dev = 0, sms = 0;
   FK_CUDA(cudaGetDevice(&dev), "get device");
   FK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "device attribute");
-  a.kv_splits = attention_pick_splits(B, H, r, D, L, sms);
+  attention_plan(B, H, r, L, sms, &a.tiles_per_cta, &a.kv_splits);
   if (!a.status) return kfail(FVAR_ECUDA, "attention: status word");
   FK_CUDA(launch_attention(tq, tk, tv, a, static_cast<cudaStream_t>(stream)), "attention");
   return FVAR_OK;
