@@ -2,6 +2,8 @@
 
     python microbench.py gemm        # FVAR_GEMM_BLOCK_N=64|128|256 forces a width, FVAR_GEMM_PAIR=0|1 the launch form
     python microbench.py skinny      # the weight-streaming form on the Infinity-2B-shaped late GEMMs
+    python microbench.py skinny_one R N K [S]  # eight launches of that form on one shape (for ncu)
+    python microbench.py attention_one B H D r L   # four attention launches on one shape (for ncu)
     python microbench.py gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
     python microbench.py attention
     python microbench.py memory      # score, LayerNorm + modulate, restoration fill, selection
@@ -95,6 +97,33 @@ def skinny():
                 R, N, K, auto, sk, N * K * 2 / sk / 1e3, 2 * R * N * K / sk / 1e6), flush=True)
 
 
+def skinny_one():
+    """A few launches of the weight-streaming form over rotating weight copies (for a profiler): R N K [ranges]."""
+    lib = fv.load_library()
+    R, N, K = (int(x) for x in sys.argv[2:5])
+    S = int(sys.argv[5]) if len(sys.argv) > 5 else 0
+    A = torch.randn(R, K, device="cuda").bfloat16()
+    Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(8)]
+    out = torch.empty(R, N, device="cuda", dtype=torch.float32)
+    for W in Ws:
+        assert lib.fvar_gemm_bf16_form(A.data_ptr(), W.data_ptr(), None, R, N, K, fv.GEMM_SKINNY, S, out.data_ptr(),
+                                       torch.cuda.current_stream().cuda_stream) == 0
+    torch.cuda.synchronize()
+    print("launched 8 weight-streaming GEMMs R=%d N=%d K=%d" % (R, N, K))
+
+
+def attention_one():
+    """A few launches of the attention kernel over rotating caches (for a profiler): B H D r L."""
+    B, H, D, r, L = (int(x) for x in sys.argv[2:7])
+    Lc = (L + 127) // 128 * 128
+    q = torch.randn(B, r, H * D, device="cuda").bfloat16()
+    caches = [(torch.randn(B, H, Lc, D, device="cuda").bfloat16(), torch.randn(B, H, D, Lc, device="cuda").bfloat16()) for _ in range(4)]
+    for Kc, Vt in caches:
+        fv.fvar_attention(q, Kc, Vt, L)
+    torch.cuda.synchronize()
+    print("launched 4 attention calls B=%d H=%d D=%d r=%d L=%d" % (B, H, D, r, L))
+
+
 def gemmk():
     lib = fv.load_library()
     tag = "PAIR=%s BN=%s" % (os.environ.get("FVAR_GEMM_PAIR", "model"), os.environ.get("FVAR_GEMM_BLOCK_N", "model"))
@@ -182,4 +211,5 @@ def transition():
 
 if __name__ == "__main__":
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
-    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition, "skinny": skinny}[which]()
+    {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition, "skinny": skinny,
+     "skinny_one": skinny_one, "attention_one": attention_one}[which]()
