@@ -353,12 +353,14 @@ fvar_status fvar_gemm_bf16_wt(const void *A, const void *Wt, const void *bias, i
  * pick the width for the given form.  The transformer block of the step is the workload's own
  * definition (the paper only names it a "VAR block", Sec. 3.1), so this is a kernel-level entry for
  * tests and tuning.  FVAR_GEMM_SKINNY: the weight-streaming form for R <= 512 (see FVAR_OPT_SKINNY_MAX_ROWS);
- * block_n is then the number of K ranges per 128-feature tile, 1 .. 8, or 0 to let the library pick.
+ * block_n is then the number of K ranges per 128-feature tile, 1 .. 8, or 0 to let the library pick.  FVAR_GEMM_KSPLIT:
+ * 128 x 128 output tiles (rows on the M side, any R) whose K range is spread over a cluster in the same way.
  * FVAR_EINVAL for a form / width the problem does not allow. */
 #define FVAR_GEMM_AUTO 0
 #define FVAR_GEMM_SINGLE 1
 #define FVAR_GEMM_PAIR 2
 #define FVAR_GEMM_SKINNY 3
+#define FVAR_GEMM_KSPLIT 4
 fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
                                 int block_n, float *out, void *stream);
 

@@ -124,6 +124,18 @@ def attention_one():
     print("launched 4 attention calls B=%d H=%d D=%d r=%d L=%d" % (B, H, D, r, L))
 
 
+def ksplit():
+    """128 x 128 tiles with the K range over a cluster against the picked form and the weight-streaming form."""
+    lib = fv.load_library()
+    for R in (111, 170, 256, 336, 410, 479):
+        for N, K in ((2048, 2048), (2048, 8192), (6144, 2048), (8192, 2048)):
+            auto = _gemm_form_graph_us(lib, R, N, K, fv.GEMM_AUTO, 0)
+            sk = _gemm_form_graph_us(lib, R, N, K, fv.GEMM_SKINNY, 0)
+            ks = _gemm_form_graph_us(lib, R, N, K, fv.GEMM_KSPLIT, 0)
+            print("R=%d N=%d K=%d: picked %.2f us | weight-streaming %.2f us | 128x128 cluster-split %.2f us (%.0f TFLOP/s)" % (
+                R, N, K, auto, sk, ks, 2 * R * N * K / ks / 1e6), flush=True)
+
+
 def gemmk():
     lib = fv.load_library()
     tag = "PAIR=%s BN=%s" % (os.environ.get("FVAR_GEMM_PAIR", "model"), os.environ.get("FVAR_GEMM_BLOCK_N", "model"))
@@ -212,4 +224,4 @@ def transition():
 if __name__ == "__main__":
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
     {"gemm": gemm, "gemmk": gemmk, "attention": attention, "memory": memory, "transition": transition, "skinny": skinny,
-     "skinny_one": skinny_one, "attention_one": attention_one}[which]()
+     "ksplit": ksplit, "skinny_one": skinny_one, "attention_one": attention_one}[which]()

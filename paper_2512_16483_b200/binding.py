@@ -21,7 +21,7 @@ CFG_PAIR, CFG_NULL_ONLY = 0, 1
 SELECT_TOPR, SELECT_SAMPLE = 0, 1
 RESTORE_RTR, RESTORE_LLS = 0, 1
 OPT_CUDA_GRAPHS, OPT_GEMM_MAX_SPLITS, OPT_SKINNY_MAX_ROWS, OPT_WAIT_KCYCLES = 0, 1, 2, 3
-GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR, GEMM_SKINNY = 0, 1, 2, 3
+GEMM_AUTO, GEMM_SINGLE, GEMM_PAIR, GEMM_SKINNY, GEMM_KSPLIT = 0, 1, 2, 3, 4
 KCLASSES = ("gemm", "attention", "ln_modulate", "row_scores", "select_topr", "rtr_fill", "convert")
 STATUS_NAMES = ("FVAR_OK", "FVAR_EINVAL", "FVAR_ENOMEM", "FVAR_ESTATE", "FVAR_ECUDA", "FVAR_ETIMEOUT",
                 "FVAR_EUNSUPPORTED")

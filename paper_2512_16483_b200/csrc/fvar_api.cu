@@ -357,7 +357,8 @@ fvar_status run_gemm_map(fvar_ctx *ctx, int epi, const CUtensorMap &tmA, int blk
 // A operand from one of the library's activation buffers: a single row tile takes the shortest box
 // that covers its rows.
 fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int blk, int wid, GemmArgs &g, const char *what) {
-  if (g.nbatch == 1 && g.R <= ctx->skinny_max_rows && g.R <= gemm_skinny_row_limit(g.N, g.K) && gemm_skinny_supported(epi, g.R, g.N, g.K)) {
+  if (g.nbatch == 1 && g.R <= ctx->skinny_max_rows && g.R <= gemm_skinny_row_limit(g.N, g.K) && !gemm_ksplit_wins(g.R, g.N, g.K) &&
+      gemm_skinny_supported(epi, g.R, g.N, g.K)) {
     // few rows: bound by streaming the weights once, so the weights take the M side of the MMA and the K range
     // of every 128-feature tile is spread over a cluster (gemm_skinny.cu)
     const int S = gemm_skinny_pick_splits(g.N, g.K, 0);
@@ -379,6 +380,27 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int 
     g.splits = 1;
   }
   g.pf_ptr = nullptr;
+  if (g.nbatch == 1 && ctx->skinny_max_rows > 0 && gemm_ksplit_wins(g.R, g.N, g.K) && epi != EPI_ARGMAX && g.N % 8 == 0) {
+    // a few hundred rows, narrow output: 128 x 128 tiles with the K range spread over a cluster (gemm_skinny.cu, ROWS)
+    g.sk_tiles_m = (g.R + 127) / 128;
+    const int S = gemm_skinny_pick_splits(g.N, g.K, 0, g.sk_tiles_m);
+    g.splits = S;
+    gemm_skinny_shape(g);
+    CUtensorMap tmA, tmW;
+    if (S > 0 && g.sk_stages >= 1 && gemm_skinny_map(&tmA, maps.base, maps.rows, maps.cols, maps.cols, 128, g.sk_nk) &&
+        gemm_skinny_map(&tmW, ctx->w[wid][blk], g.N, g.K, g.K, 128, g.sk_nk)) {
+      g.status = ctx->status;
+      g.wait_cycles = ctx->wait_cycles;
+      ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * g.R * g.N * g.K,
+                      2.0 * (static_cast<double>(g.N) * g.K + static_cast<double>(g.R) * g.K) +
+                          (epi == EPI_F32 || epi == EPI_RESID ? 4.0 : 2.0) * g.R * g.N);
+      FV_CUDA(ctx, launch_gemm_skinny(epi, tmA, tmW, g, ctx->launch_st), what);
+      ctx->launched();
+      return FVAR_OK;
+    }
+    g.sk_tiles_m = 0;
+    g.splits = 1;
+  }
   int t = 3;
   if (g.nbatch == 1 && g.R <= 64) t = g.R <= 16 ? 0 : (g.R <= 32 ? 1 : 2);
   g.a_box_rows = 16 << t;
@@ -1452,14 +1474,18 @@ fvar_status fvar_ln_modulate(const float *x, int R, int C, int rows_per_batch, c
 fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, int R, int N, int K, int form,
                                 int block_n, float *out, void *stream) {
   if (!A || !W || !out || R <= 0 || N <= 0 || K <= 0 || K % 8) return kfail(FVAR_EINVAL, "gemm: bad arguments");
-  if (form != FVAR_GEMM_AUTO && form != FVAR_GEMM_SINGLE && form != FVAR_GEMM_PAIR && form != FVAR_GEMM_SKINNY)
+  if (form != FVAR_GEMM_AUTO && form != FVAR_GEMM_SINGLE && form != FVAR_GEMM_PAIR && form != FVAR_GEMM_SKINNY && form != FVAR_GEMM_KSPLIT)
     return kfail(FVAR_EINVAL, "gemm: bad form");
-  if (form == FVAR_GEMM_SKINNY) {
-    if (!gemm_skinny_supported(EPI_F32, R, N, K)) return kfail(FVAR_EINVAL, "gemm: the weight-streaming form needs R <= 512, N % 8 == 0");
-    if (block_n < 0 || block_n > 8) return kfail(FVAR_EINVAL, "gemm: the weight-streaming form takes 0 .. 8 K ranges");
-    const int S = gemm_skinny_pick_splits(N, K, block_n);
+  if (form == FVAR_GEMM_SKINNY || form == FVAR_GEMM_KSPLIT) {
+    const int tiles_m = form == FVAR_GEMM_KSPLIT ? (R + 127) / 128 : 0;
+    if (form == FVAR_GEMM_SKINNY && !gemm_skinny_supported(EPI_F32, R, N, K))
+      return kfail(FVAR_EINVAL, "gemm: the weight-streaming form needs R <= 512, N % 8 == 0");
+    if (N % 8) return kfail(FVAR_EINVAL, "gemm: the cluster-split forms need N % 8 == 0");
+    if (block_n < 0 || block_n > 8) return kfail(FVAR_EINVAL, "gemm: the cluster-split forms take 0 .. 8 K ranges");
+    const int S = gemm_skinny_pick_splits(N, K, block_n, tiles_m);
     if (S <= 0) return kfail(FVAR_EINVAL, "gemm: this number of K ranges is not launchable for the problem");
     GemmArgs g = gemm_args(R, N, K);
+    g.sk_tiles_m = tiles_m;
     g.splits = S;
     gemm_skinny_shape(g);
     CUtensorMap ta, tw;

@@ -107,7 +107,11 @@ __device__ __forceinline__ void skinny_store(const GemmArgs &p, float4 acc, int 
 }
 
 // tmA: the activation rows [R][K], box of sk_rp rows; tmW: the weight rows [N][K], box of 128 rows (gemm_skinny_map).
-template <int EPI>
+// ROWS = false: the form described at the top (weights on the M side, all rows on the N side).  ROWS = true: the same
+// pipeline, K split and cluster reduction for 128 x 128 output tiles with the rows back on the M side -- for a few
+// hundred rows and a narrow output, where the row-tiled kernels have too few tiles to fill the SMs and each of their
+// CTAs walks all of K; cluster c then owns tile (row tile c % sk_tiles_m, feature tile c / sk_tiles_m).
+template <int EPI, bool ROWS>
 __global__ void __launch_bounds__(kSkinnyThreads, 1)
 gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                    const __grid_constant__ GemmArgs p) {
@@ -126,7 +130,9 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   const long long wb = wait_budget(p.wait_cycles);
   const int S = p.splits > 1 ? p.splits : 1;                 // cluster size = K ranges per tile
   const int sp = static_cast<int>(cluster_ctarank());
-  const int tile = static_cast<int>(cluster_id_x());
+  const int cid = static_cast<int>(cluster_id_x());
+  const int tile = ROWS ? cid / p.sk_tiles_m : cid;          // 128-feature tile
+  const int row0 = ROWS ? (cid % p.sk_tiles_m) * kBlockM : 0;  // first row of the tile (ROWS)
   const int nstages = p.sk_stages, rp = p.sk_rp, rc = p.sk_rows_chunk, nchunks = p.sk_nchunks;
   const int rp32 = (rp + 31) & ~31;                          // TMEM columns between the accumulators of two chunks
   const int nk = p.sk_nk;                                   // K blocks per pipeline stage (one TMA instruction per operand)
@@ -150,8 +156,8 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   auto load_a = [&](int i) {
     const uint32_t dst = ring + (i % nstages) * stage_bytes + w_stage;
     for (int ch = 0; ch < nchunks; ++ch) {
-      if (nk > 1) tma_load_3d(dst + ch * nk * a_bytes, &tmA, full_bar(i % nstages), 0, ch * rc, kb0 + i * nk);
-      else tma_load_2d(dst + ch * a_bytes, &tmA, full_bar(i % nstages), (kb0 + i) * kBlockK, ch * rc);
+      if (nk > 1) tma_load_3d(dst + ch * nk * a_bytes, &tmA, full_bar(i % nstages), 0, row0 + ch * rc, kb0 + i * nk);
+      else tma_load_2d(dst + ch * a_bytes, &tmA, full_bar(i % nstages), (kb0 + i) * kBlockK, row0 + ch * rc);
     }
   };
   const int pre = min(nstages, nst);
@@ -238,8 +244,12 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         for (int kk = 0; kk < kvalid; ++kk) {
 #pragma unroll
           for (int k = 0; k < kBlockK / 16; ++k) {
-            umma_bf16(tmem_base, dw + 2 * k, da0 + 2 * k, idesc, acc);
-            if (nchunks > 1) umma_bf16(tmem_base + rp32, dw + 2 * k, da0 + da1_off + 2 * k, idesc, acc);
+            if (ROWS) {
+              umma_bf16(tmem_base, da0 + 2 * k, dw + 2 * k, idesc, acc);       // rows x features
+            } else {
+              umma_bf16(tmem_base, dw + 2 * k, da0 + 2 * k, idesc, acc);       // features x rows
+              if (nchunks > 1) umma_bf16(tmem_base + rp32, dw + 2 * k, da0 + da1_off + 2 * k, idesc, acc);
+            }
             acc = 1u;
           }
           dw += kSkinnyWAtom >> 4;
@@ -262,19 +272,38 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
   // Every thread of every CTA of the cluster passes the same cluster barriers; warps 2-9 do the work.
   const int et = static_cast<int>(threadIdx.x) - 64;         // 0 .. 255 in the epilogue warps
   const uint32_t red = ring;                                   // fp32 [rows of the chunk][128 features]; the ring is free by now
+  // parked tile: [row][128 features] fp32; ROWS pads a row to 132 floats so that the 16-byte writes of the 32 lanes
+  // (one row each) do not collide
+  constexpr uint32_t kPitch = ROWS ? 528u : 512u;
   for (int ch = 0; ch < nchunks; ++ch) {
-    const int rows_ch = min(rc, p.R - ch * rc);
+    const int rows_ch = ROWS ? min(kBlockM, p.R - row0) : min(rc, p.R - ch * rc);
     if (warp >= 2 && ok) {
       const int quad = warp & 3, cg = (warp - 2) >> 2;
       const uint32_t taddr = tmem_base + ch * rp32 + (static_cast<uint32_t>(quad * 32) << 16);
-      for (int c = cg; c * 32 < rows_ch; c += kEpiColGroups) {
-        uint32_t acc[32];
-        tmem_ld32(taddr + c * 32, acc);
-        tmem_ld_wait();
-        const uint32_t dst = red + static_cast<uint32_t>(c * 32) * 512u + static_cast<uint32_t>(quad * 32 + lane) * 4u;
+      if (ROWS) {
+        const int row_local = quad * 32 + lane;              // TMEM lane = row of the tile, columns = features
+        for (int c = cg; c < kBlockM / 32; c += kEpiColGroups) {
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+          if (row_local < rows_ch) {
+            const uint32_t dst = red + static_cast<uint32_t>(row_local) * kPitch + static_cast<uint32_t>(c * 32) * 4u;
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (c * 32 + i < rows_ch) asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + i * 512u), "r"(acc[i]) : "memory");
+            for (int q = 0; q < 8; ++q)
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + q * 16u), "r"(acc[q * 4]), "r"(acc[q * 4 + 1]),
+                           "r"(acc[q * 4 + 2]), "r"(acc[q * 4 + 3]) : "memory");
+          }
+        }
+      } else {
+        for (int c = cg; c * 32 < rows_ch; c += kEpiColGroups) {   // TMEM lane = feature, columns = rows
+          uint32_t acc[32];
+          tmem_ld32(taddr + c * 32, acc);
+          tmem_ld_wait();
+          const uint32_t dst = red + static_cast<uint32_t>(c * 32) * 512u + static_cast<uint32_t>(quad * 32 + lane) * 4u;
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i < rows_ch) asm volatile("st.shared.b32 [%0], %1;" ::"r"(dst + i * 512u), "r"(acc[i]) : "memory");
+        }
       }
     }
     tc_fence_before();
@@ -288,7 +317,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 #pragma unroll
         for (int t = 0; t < 8; ++t) peer[t] = mapa_shared(red, static_cast<uint32_t>(t < S ? t : 0));
         for (int jj = lo + (et >> 5); jj < hi; jj += 8) {
-          const uint32_t off = static_cast<uint32_t>(jj) * 512u + static_cast<uint32_t>(n4) * 4u;
+          const uint32_t off = static_cast<uint32_t>(jj) * kPitch + static_cast<uint32_t>(n4) * 4u;
           float4 sum = ld_dsmem_f4(peer[0] + off);
 #pragma unroll
           for (int t = 1; t < 8; ++t)
@@ -296,7 +325,7 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
               const float4 v = ld_dsmem_f4(peer[t] + off);
               sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
             }
-          skinny_store<EPI>(p, sum, ch * rc + jj, n);
+          skinny_store<EPI>(p, sum, row0 + ch * rc + jj, n);
         }
       }
     }
@@ -313,19 +342,19 @@ gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------ host
-template <int EPI>
+template <int EPI, bool ROWS>
 struct SkinnyState {
   static bool ready;
   static int max_clusters[9];        // resident clusters of size S (0: not launchable)
 };
-template <int EPI> bool SkinnyState<EPI>::ready = false;
-template <int EPI> int SkinnyState<EPI>::max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+template <int EPI, bool ROWS> bool SkinnyState<EPI, ROWS>::ready = false;
+template <int EPI, bool ROWS> int SkinnyState<EPI, ROWS>::max_clusters[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
 
-template <int EPI>
+template <int EPI, bool ROWS>
 static cudaError_t skinny_prepare_one() {
-  using St = SkinnyState<EPI>;
+  using St = SkinnyState<EPI, ROWS>;
   if (St::ready) return cudaSuccess;
-  cudaError_t err = cudaFuncSetAttribute(gemm_skinny_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkinnySmemBytes);
+  cudaError_t err = cudaFuncSetAttribute(gemm_skinny_kernel<EPI, ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSkinnySmemBytes);
   if (err != cudaSuccess) return err;
   int dev = 0, sms = 0;
   if ((err = cudaGetDevice(&dev)) != cudaSuccess) return err;
@@ -343,7 +372,7 @@ static cudaError_t skinny_prepare_one() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_skinny_kernel<EPI>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_skinny_kernel<EPI, ROWS>, &cfg) != cudaSuccess) {
       cudaGetLastError();            // this cluster size is not launchable here: leave it at 0
       n = 0;
     }
@@ -354,11 +383,16 @@ static cudaError_t skinny_prepare_one() {
 }
 
 cudaError_t gemm_skinny_prepare() {
-  cudaError_t e = skinny_prepare_one<EPI_F32>();
-  if (e == cudaSuccess) e = skinny_prepare_one<EPI_BF16>();
-  if (e == cudaSuccess) e = skinny_prepare_one<EPI_GELU_BF16>();
-  if (e == cudaSuccess) e = skinny_prepare_one<EPI_QKV>();
-  if (e == cudaSuccess) e = skinny_prepare_one<EPI_RESID>();
+  cudaError_t e = skinny_prepare_one<EPI_F32, false>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_BF16, false>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_GELU_BF16, false>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_QKV, false>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_RESID, false>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_F32, true>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_BF16, true>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_GELU_BF16, true>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_QKV, true>();
+  if (e == cudaSuccess) e = skinny_prepare_one<EPI_RESID, true>();
   return e;
 }
 
@@ -371,16 +405,25 @@ bool gemm_skinny_supported(int epi, int R, int N, int K) {
 // of K, so the K split over a cluster wins up to a few hundred rows, longer for a long reduction; with many
 // features the row-tiled kernels already cover the SMs and win from 64 rows on.
 int gemm_skinny_row_limit(int N, int K) {
-  if (N <= 2048) return K >= 4096 ? 336 : 128;
+  if (N <= 2048) return K >= 4096 ? 384 : 64;               // 65 .. 256 rows go to the 128 x 128 cluster-split mode first
   return 32;
 }
 
-// K ranges per 128-feature tile: the split whose slowest CTA walks the fewest K blocks, waves of resident
-// clusters counted; among equals the smallest.  forced > 0 takes that split when it is launchable.
-int gemm_skinny_pick_splits(int N, int K, int forced) {
+// Whether the 128 x 128-tile mode (rows on the M side, K split over a cluster) beats the row-tiled kernels: set from
+// measurements; see the cost note in gemm_skinny_row_limit.
+bool gemm_ksplit_wins(int R, int N, int K) {
+  if (N > 2048 || R <= 64) return false;                     // wide outputs fill the SMs without a K split; few rows stream weights
+  if (R <= 256) return true;                                 // one or two row tiles: 7 - 15 us against 9 - 25 us row-tiled
+  return K >= 4096 && R > 384 && R <= 512;                   // four row tiles over a long reduction: 22 us against 25 us
+}
+
+// K ranges per tile (128 features x all rows, or x 128 rows when row_tiles > 0 row tiles are given): the split whose
+// slowest CTA walks the fewest K blocks, waves of resident clusters counted; among equals the smallest.  forced > 0
+// takes that split when it is launchable.
+int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles) {
   if (gemm_skinny_prepare() != cudaSuccess) return 0;
-  const int *mc = SkinnyState<EPI_RESID>::max_clusters;
-  const int tiles = (N + kBlockM - 1) / kBlockM, num_kb = (K + kBlockK - 1) / kBlockK;
+  const int *mc = row_tiles > 0 ? SkinnyState<EPI_RESID, true>::max_clusters : SkinnyState<EPI_RESID, false>::max_clusters;
+  const int tiles = (N + kBlockM - 1) / kBlockM * (row_tiles > 0 ? row_tiles : 1), num_kb = (K + kBlockK - 1) / kBlockK;
   int best = 0;
   long long best_cost = 0;
   for (int s = 1; s <= 8; ++s) {
@@ -395,13 +438,13 @@ int gemm_skinny_pick_splits(int N, int K, int forced) {
   return best;
 }
 
-template <int EPI>
+template <int EPI, bool ROWS>
 static cudaError_t skinny_launch_one(const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, cudaStream_t st) {
-  cudaError_t err = skinny_prepare_one<EPI>();
+  cudaError_t err = skinny_prepare_one<EPI, ROWS>();
   if (err != cudaSuccess) return err;
   const int S = a.splits > 1 ? a.splits : 1;
-  if (S > 8 || SkinnyState<EPI>::max_clusters[S] <= 0) return cudaErrorInvalidValue;
-  const int tiles = (a.N + kBlockM - 1) / kBlockM;
+  if (S > 8 || SkinnyState<EPI, ROWS>::max_clusters[S] <= 0) return cudaErrorInvalidValue;
+  const int tiles = (a.N + kBlockM - 1) / kBlockM * (ROWS ? a.sk_tiles_m : 1);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(tiles * S);
   cfg.blockDim = dim3(kSkinnyThreads);
@@ -416,11 +459,19 @@ static cudaError_t skinny_launch_one(const CUtensorMap &tmA, const CUtensorMap &
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<EPI>, tmA, tmW, a);
+  return cudaLaunchKernelEx(&cfg, gemm_skinny_kernel<EPI, ROWS>, tmA, tmW, a);
 }
 
 // Fills the chunking fields of `a` for R rows (R <= 512): rows per chunk, padded MMA width, stage count.
 void gemm_skinny_shape(GemmArgs &a) {
+  if (a.sk_tiles_m > 0) {                    // 128 x 128 tiles: two K blocks of each operand per stage, three stages
+    a.sk_nchunks = 1; a.sk_rows_chunk = kBlockM; a.sk_rp = kBlockM; a.sk_small = 0;
+    const int num_kb = (a.K + kBlockK - 1) / kBlockK, S = a.splits > 1 ? a.splits : 1;
+    a.sk_nk = (a.K % kBlockK == 0 && (num_kb + S - 1) / S >= 2) ? 2 : 1;
+    a.sk_stages = kSkinnyRing / (a.sk_nk * 2 * kSkinnyWAtom);
+    if (a.sk_stages > kSkinnyMaxStages) a.sk_stages = kSkinnyMaxStages;
+    return;
+  }
   a.sk_nchunks = a.R > 256 ? 2 : 1;
   a.sk_rows_chunk = a.sk_nchunks == 1 ? a.R : (((a.R + 1) / 2 + 15) & ~15);
   a.sk_rp = (a.sk_rows_chunk + 15) & ~15;
@@ -453,13 +504,25 @@ bool gemm_skinny_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t K
 // tmA / tmW: gemm_skinny_map over the activation rows (box of a.sk_rp rows) and the weight rows (box of 128 rows).
 // a.splits = cluster size, set before gemm_skinny_shape.
 cudaError_t launch_gemm_skinny(int epi, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, cudaStream_t st) {
-  if (a.nbatch != 1 || a.w_mn_major || !gemm_skinny_supported(epi, a.R, a.N, a.K) || a.sk_stages < 1) return cudaErrorInvalidValue;
+  if (a.nbatch != 1 || a.w_mn_major || a.sk_stages < 1 || epi == EPI_ARGMAX || a.N % 8 || a.K % 8 ||
+      (a.sk_tiles_m <= 0 && !gemm_skinny_supported(epi, a.R, a.N, a.K)))
+    return cudaErrorInvalidValue;
+  if (a.sk_tiles_m > 0) {
+    switch (epi) {
+      case EPI_F32: return skinny_launch_one<EPI_F32, true>(tmA, tmW, a, st);
+      case EPI_BF16: return skinny_launch_one<EPI_BF16, true>(tmA, tmW, a, st);
+      case EPI_GELU_BF16: return skinny_launch_one<EPI_GELU_BF16, true>(tmA, tmW, a, st);
+      case EPI_QKV: return skinny_launch_one<EPI_QKV, true>(tmA, tmW, a, st);
+      case EPI_RESID: return skinny_launch_one<EPI_RESID, true>(tmA, tmW, a, st);
+    }
+    return cudaErrorInvalidValue;
+  }
   switch (epi) {
-    case EPI_F32: return skinny_launch_one<EPI_F32>(tmA, tmW, a, st);
-    case EPI_BF16: return skinny_launch_one<EPI_BF16>(tmA, tmW, a, st);
-    case EPI_GELU_BF16: return skinny_launch_one<EPI_GELU_BF16>(tmA, tmW, a, st);
-    case EPI_QKV: return skinny_launch_one<EPI_QKV>(tmA, tmW, a, st);
-    case EPI_RESID: return skinny_launch_one<EPI_RESID>(tmA, tmW, a, st);
+    case EPI_F32: return skinny_launch_one<EPI_F32, false>(tmA, tmW, a, st);
+    case EPI_BF16: return skinny_launch_one<EPI_BF16, false>(tmA, tmW, a, st);
+    case EPI_GELU_BF16: return skinny_launch_one<EPI_GELU_BF16, false>(tmA, tmW, a, st);
+    case EPI_QKV: return skinny_launch_one<EPI_QKV, false>(tmA, tmW, a, st);
+    case EPI_RESID: return skinny_launch_one<EPI_RESID, false>(tmA, tmW, a, st);
   }
   return cudaErrorInvalidValue;
 }

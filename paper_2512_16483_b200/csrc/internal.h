@@ -60,6 +60,7 @@ struct GemmArgs {
   // Weight-streaming form (gemm_skinny.cu; `splits` is then the cluster size): rows per column chunk, the padded
   // MMA width of a chunk, chunks (1 or 2) and pipeline stages -- filled by gemm_skinny_shape
   int sk_rows_chunk, sk_rp, sk_nchunks, sk_stages, sk_small, sk_nk;
+  int sk_tiles_m;          // > 0: the 128 x 128-tile mode of that kernel with this many row tiles (rows on the M side)
   // optional: weights the next GEMM of the chain will stream; every CTA asks L2 to prefetch its share
   const void *pf_ptr;
   unsigned long long pf_bytes;
@@ -104,8 +105,9 @@ GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_cluster
 // a 128-feature tile is split over a cluster of `splits` CTAs that reduce through distributed shared memory.
 // tmA: box {64, a.sk_rp} over the activation rows; tmW: box {64, 128} over the weight rows.
 bool gemm_skinny_supported(int epi, int R, int N, int K);
-int gemm_skinny_row_limit(int N, int K);                      // rows up to which this form is the faster one
-int gemm_skinny_pick_splits(int N, int K, int forced);      // 0: not launchable on this device
+int gemm_skinny_row_limit(int N, int K);
+bool gemm_ksplit_wins(int R, int N, int K);                   // the 128 x 128-tile cluster-split mode is the faster form                      // rows up to which this form is the faster one
+int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles = 0);      // 0: not launchable on this device
 void gemm_skinny_shape(GemmArgs &a);      // needs a.R, a.K and a.splits
 bool gemm_skinny_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows, int nk);
 cudaError_t launch_gemm_skinny(int epi, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, cudaStream_t st);

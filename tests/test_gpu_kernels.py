@@ -150,6 +150,28 @@ def test_gemm_bf16_weight_streaming_form(fv, R, N, K, splits):
     np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
 
 
+# The same K split over a cluster with 128 x 128 output tiles (rows on the M side): ragged rows, features and K, one to
+# four row tiles, every cluster size.
+@pytest.mark.parametrize("R,N,K", [(1, 128, 64), (130, 200, 136), (336, 2048, 2048), (257, 384, 520), (512, 256, 1024),
+                                   (410, 2048, 8192), (700, 128, 256)])
+@pytest.mark.parametrize("splits", [0, 1, 2, 3, 4, 6, 8])
+def test_gemm_bf16_cluster_split_tiles(fv, R, N, K, splits):
+    rng = np.random.default_rng(13 * R + N + K)
+    A = si.normal_bf16(rng, (R, K))
+    W = si.normal_bf16(rng, (N, K), 0.05)
+    b = si.normal_bf16(rng, (N,))
+    num_kb = -(-K // 64)
+    if splits and -(-num_kb // -(-num_kb // splits)) != splits:
+        with pytest.raises(fv.FvarError):
+            fv.fvar_gemm_bf16_form(to_bf16_cuda(A), to_bf16_cuda(W), to_bf16_cuda(b), fv.GEMM_KSPLIT, splits)
+        return
+    got = fv.fvar_gemm_bf16_form(to_bf16_cuda(A), to_bf16_cuda(W), to_bf16_cuda(b), fv.GEMM_KSPLIT, splits).cpu().numpy()
+    _poll(fv)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T + b.astype(np.float64)
+    tol = 1e-5 * (np.abs(A).astype(np.float64) @ np.abs(W).astype(np.float64).T).max() + 1e-6
+    np.testing.assert_allclose(got, ref, atol=tol, rtol=0)
+
+
 @pytest.mark.parametrize("R,N,K", [(128, 64, 64), (300, 200, 136), (1000, 1024, 512), (130, 1920, 344), (64, 2048, 8192)])
 @pytest.mark.parametrize("block_n", [0, 64, 128, 256])
 def test_gemm_bf16_second_operand_transposed(fv, R, N, K, block_n):
