@@ -9,7 +9,8 @@ dense path with both CFG branches; R < 4096 is the method: null-prompt branch on
 blocks on R rows, restoration.  The method has one knob, the number of rows r that go through the blocks,
 so the keep ratios {0.75, 0.5, 0.25} and the ranks {64, 32, 16} of the sweep are all values of R.
 Prints one markdown table row per point: ms per step, tokens/s, speed-up over the dense path of the same
-batch, TFLOP/s and fraction of the measured sustained bf16 peak of the GEMM class, TFLOP/s of attention.
+batch, the roofline that binds the step (HBM below the ridge, tensor above), the fraction of it reached and the
+floor it implies.
 """
 from __future__ import annotations
 
@@ -40,19 +41,19 @@ def main():
     args = ap.parse_args()
     ranks = [int(v) for v in args.ranks.split(",")]
     batches = [int(v) for v in args.batches.split(",")]
-    print("| B (pairs) | R | mode | ms / step | tokens/s | vs dense | GEMM TFLOP/s (frac) | attention TFLOP/s | SM MHz, reasons |")
-    print("|---|---|---|---|---|---|---|---|---|")
+    print("| B (pairs) | R | mode | ms / step | tokens/s | vs dense | bound | roofline frac | floor ms | SM MHz, reasons |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
     for B in batches:
         dense_ms = None
         for R in ranks:
             d = run_point(R, B, args.steps)
-            c = d["roofline"]["classes"]
+            rf = d["roofline"]
             if R == 4096:
                 dense_ms = d["ms_per_step"]
-            print("| %d (%d) | %d | %s | %.2f | %.3g | %s | %.0f (%.2f) | %.0f | %s %s |" % (
+            print("| %d (%d) | %d | %s | %.2f | %.3g | %s | %s | %.2f | %.2f | %s %s |" % (
                 B, B // 2, R, "dense, both branches" if R == 4096 else "null branch, RP + RTR", d["ms_per_step"], d["value"],
-                "%.1fx" % (dense_ms / d["ms_per_step"]) if dense_ms else "-", c["gemm"]["tflops"], d["roofline"]["frac"],
-                c["attention"]["tflops"], d["clocks"]["sm_mhz"], ",".join(d["clocks"]["reasons"]) or "none"), flush=True)
+                "%.1fx" % (dense_ms / d["ms_per_step"]) if dense_ms else "-", rf["bound"], rf["frac"], rf["floor_ms_per_step"],
+                d["clocks"]["sm_mhz"], ",".join(d["clocks"]["reasons"]) or "none"), flush=True)
 
 
 if __name__ == "__main__":

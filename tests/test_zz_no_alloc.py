@@ -26,8 +26,15 @@ def test_static_selection_matches_two_call_form_twice():
         ref_idx, ref_inv = fv.fvar_select_topr(fv.fvar_row_scores(x), r)
         idx = torch.full((B, r), -5, dtype=torch.int32, device="cuda")
         inv = torch.full((B, M), -5, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         fv.fvar_select_rows_static(x, r, idx, inv)
         torch.cuda.synchronize()
+        # nothing was allocated: not through torch, and (from the second call on, once the kernels' code is loaded)
+        # not behind its back either
+        assert torch.cuda.memory_allocated() == held
+        if seed == 12:
+            assert torch.cuda.mem_get_info()[0] >= free
         assert torch.equal(idx, ref_idx) and torch.equal(inv, ref_inv)
         assert bool((idx[:, 1:] > idx[:, :-1]).all())
 
