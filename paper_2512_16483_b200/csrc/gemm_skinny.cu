@@ -9,10 +9,10 @@
 // reduces a 1/S slice of the rows over all S partials through distributed shared memory, in rank order
 // (the sum does not depend on timing), and applies the epilogue.  Nothing goes through global scratch.
 //
-// A TMA tile load costs the SM's copy unit about the same time whatever its size (measured: ~550 cycles per
-// instruction even for L2 hits, instructions hardly overlapping), so a pipeline stage covers several K blocks
-// fetched by ONE instruction per operand: the operands are described as 3-D tensors {64 K elements, rows, K / 64}
-// and a box {64, rows, nk} lands as nk consecutive 128-byte-swizzled K-major tiles.
+// A pipeline stage covers up to four 64-wide K blocks fetched by ONE TMA instruction per operand: the operands are
+// described as 3-D tensors {64 K elements, rows, K / 64} and a box {64, rows, nk} lands as nk consecutive
+// 128-byte-swizzled K-major tiles (fewer barrier round trips per byte; in a load-only probe the bytes per instruction
+// set the throughput of a single SM's copy unit).
 //
 // Roles: warp 0 feeds the stage ring with TMA (the weight halves of the first stages are requested before
 // griddepcontrol.wait: weights never depend on the preceding kernel), warp 1 issues the MMAs into TMEM,
