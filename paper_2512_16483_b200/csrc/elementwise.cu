@@ -208,6 +208,39 @@ cudaError_t launch_copy_indices(const int *forced, int B, int M, int r, int ld_f
 constexpr int kLnThreads = 128;
 constexpr int kLnMaxVec = 8;                    // 8 x (8 elements) x 128 threads = 8192 columns
 
+// Normalises, modulates (or scales by gamma) and stores one group of 8 consecutive elements of a row: group g of
+// the row whose values are in v, statistics mean / rstd; shift and scale at float offset voff, y row at yr.
+__device__ __forceinline__ void ln_store_group(const float (&v)[8], float mean, float rstd, const bf16 *__restrict__ gamma,
+                                               const float *__restrict__ scale, const float *__restrict__ shift, long long voff,
+                                               int g, bf16 *__restrict__ yr) {
+  float o[8];
+  if (gamma != nullptr) {
+    const uint4 gu = __ldg(reinterpret_cast<const uint4 *>(gamma) + g);
+    const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&gu);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 gf = __bfloat1622float2(gh[i]);
+      o[2 * i] = (v[2 * i] - mean) * rstd * gf.x;
+      o[2 * i + 1] = (v[2 * i + 1] - mean) * rstd * gf.y;
+    }
+  } else {
+    const float4 *sc = reinterpret_cast<const float4 *>(scale + voff) + 2 * g;
+    const float4 *sh = reinterpret_cast<const float4 *>(shift + voff) + 2 * g;
+    const float4 s0 = __ldg(sc), s1 = __ldg(sc + 1), h0 = __ldg(sh), h1 = __ldg(sh + 1);
+    const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const float shv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = fmaf((v[i] - mean) * rstd, 1.0f + scv[i], shv[i]);
+  }
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+    w[i] = *reinterpret_cast<uint32_t *>(&h2);
+  }
+  reinterpret_cast<uint4 *>(yr)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 __global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__restrict__ x, RowMap xmap, int rows,
                                                                  int C, const float *__restrict__ shift,
                                                                  const float *__restrict__ scale,
@@ -263,32 +296,7 @@ __global__ void __launch_bounds__(kLnThreads) ln_modulate_kernel(const float *__
   for (int t = 0; t < kLnMaxVec; ++t) {
     const int g = threadIdx.x + t * kLnThreads;
     if (g < nvec) {
-      float o[8];
-      if (gamma != nullptr) {
-        const uint4 gu = __ldg(reinterpret_cast<const uint4 *>(gamma) + g);
-        const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&gu);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 gf = __bfloat1622float2(gh[i]);
-          o[2 * i] = (v[t][2 * i] - mean) * rstd * gf.x;
-          o[2 * i + 1] = (v[t][2 * i + 1] - mean) * rstd * gf.y;
-        }
-      } else {
-        const float4 *sc = reinterpret_cast<const float4 *>(scale + voff) + 2 * g;
-        const float4 *sh = reinterpret_cast<const float4 *>(shift + voff) + 2 * g;
-        const float4 s0 = __ldg(sc), s1 = __ldg(sc + 1), h0 = __ldg(sh), h1 = __ldg(sh + 1);
-        const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        const float shv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] = fmaf((v[t][i] - mean) * rstd, 1.0f + scv[i], shv[i]);
-      }
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-        w[i] = *reinterpret_cast<uint32_t *>(&h2);
-      }
-      reinterpret_cast<uint4 *>(yr)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+      ln_store_group(v[t], mean, rstd, gamma, scale, shift, voff, g, yr);
     }
   }
 }
@@ -340,32 +348,7 @@ __global__ void __launch_bounds__(256) ln_modulate_warp_kernel(const float *__re
   for (int t = 0; t < T; ++t) {
     const int g = lane + t * 32;
     if (g < nvec) {
-      float o[8];
-      if (gamma != nullptr) {
-        const uint4 gu = __ldg(reinterpret_cast<const uint4 *>(gamma) + g);
-        const __nv_bfloat162 *gh = reinterpret_cast<const __nv_bfloat162 *>(&gu);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 gf = __bfloat1622float2(gh[i]);
-          o[2 * i] = (v[t][2 * i] - mean) * rstd * gf.x;
-          o[2 * i + 1] = (v[t][2 * i + 1] - mean) * rstd * gf.y;
-        }
-      } else {
-        const float4 *sc = reinterpret_cast<const float4 *>(scale + voff) + 2 * g;
-        const float4 *sh = reinterpret_cast<const float4 *>(shift + voff) + 2 * g;
-        const float4 s0 = __ldg(sc), s1 = __ldg(sc + 1), h0 = __ldg(sh), h1 = __ldg(sh + 1);
-        const float scv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        const float shv[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) o[i] = fmaf((v[t][i] - mean) * rstd, 1.0f + scv[i], shv[i]);
-      }
-      uint32_t w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-        w[i] = *reinterpret_cast<uint32_t *>(&h2);
-      }
-      reinterpret_cast<uint4 *>(yr)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+      ln_store_group(v[t], mean, rstd, gamma, scale, shift, voff, g, yr);
     }
   }
 }
@@ -403,11 +386,8 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
   if (inv != nullptr && inv[static_cast<long long>(e) * M1 + i] >= 0) return;
   const int b = e * bmul + boff;
   const int y = i / w1, xq = i - y * w1;
-  const float sy = fmaxf((y + 0.5f) * (static_cast<float>(h0) / h1) - 0.5f, 0.f);
-  const float sx = fmaxf((xq + 0.5f) * (static_cast<float>(w0) / w1) - 0.5f, 0.f);
-  const int y0 = min(static_cast<int>(sy), h0 - 1), x0 = min(static_cast<int>(sx), w0 - 1);
-  const int y1 = min(y0 + 1, h0 - 1), x1 = min(x0 + 1, w0 - 1);
-  const float fy = sy - y0, fx = sx - x0;
+  const BilinearTap tap = bilinear_tap(y, xq, h0, w0, h1, w1);
+  const int y0 = tap.y0, y1 = tap.y1, x0 = tap.x0, x1 = tap.x1;
   const float *src = prev + static_cast<long long>(b) * h0 * w0 * C;
   const float4 *p00 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y0) * w0 + x0) * C);
   const float4 *p01 = reinterpret_cast<const float4 *>(src + (static_cast<long long>(y0) * w0 + x1) * C);
@@ -416,7 +396,7 @@ __global__ void __launch_bounds__(256) rtr_fill_kernel(const float *__restrict__
   float4 *dst = reinterpret_cast<float4 *>(out + (static_cast<long long>(b) * M1 + i) * C);
   uint2 *hi_dst = xsplit ? reinterpret_cast<uint2 *>(xsplit + (static_cast<long long>(e) * 2 * mk + i) * C) : nullptr;
   const long long lo_off = static_cast<long long>(mk) * C / 4;      // in 4-element groups
-  const float w00 = (1.f - fy) * (1.f - fx), w01 = (1.f - fy) * fx, w10 = fy * (1.f - fx), w11 = fy * fx;
+  const float w00 = tap.w00, w01 = tap.w01, w10 = tap.w10, w11 = tap.w11;
 #pragma unroll 4
   for (int c = threadIdx.x & 31; c < C / 4; c += 32) {
     const float4 a = __ldg(p00 + c), bq = __ldg(p01 + c), cq = __ldg(p10 + c), d = __ldg(p11 + c);

@@ -16,6 +16,23 @@ struct RowMap {
   int bmul, boff, rpb;
 };
 
+// Bilinear upsampling (Eq. "upcache", Eq. "var_upf"): source cell and weights of target cell (y, x) on an (h1, w1) grid
+// read from an (h0, w0) grid -- half-pixel centres, source coordinate clamped at 0, neighbours clamped at the edge.
+struct BilinearTap {
+  int y0, y1, x0, x1;
+  float w00, w01, w10, w11;
+};
+__host__ __device__ inline BilinearTap bilinear_tap(int y, int x, int h0, int w0, int h1, int w1) {
+  const float sy = fmaxf((y + 0.5f) * (static_cast<float>(h0) / h1) - 0.5f, 0.f);
+  const float sx = fmaxf((x + 0.5f) * (static_cast<float>(w0) / w1) - 0.5f, 0.f);
+  BilinearTap t;
+  t.y0 = min(static_cast<int>(sy), h0 - 1); t.x0 = min(static_cast<int>(sx), w0 - 1);
+  t.y1 = min(t.y0 + 1, h0 - 1); t.x1 = min(t.x0 + 1, w0 - 1);
+  const float fy = sy - t.y0, fx = sx - t.x0;
+  t.w00 = (1.f - fy) * (1.f - fx); t.w01 = (1.f - fy) * fx; t.w10 = fy * (1.f - fx); t.w11 = fy * fx;
+  return t;
+}
+
 enum EpiMode { EPI_F32 = 0, EPI_BF16 = 1, EPI_GELU_BF16 = 2, EPI_QKV = 3, EPI_RESID = 4, EPI_ARGMAX = 5 };
 
 struct GemmArgs {

@@ -70,17 +70,14 @@ __global__ void __launch_bounds__(256) up_accumulate_kernel(const bf16 *__restri
   if (gw >= static_cast<long long>(B) * M1) return;
   const int b = static_cast<int>(gw / M1), i = static_cast<int>(gw - static_cast<long long>(b) * M1);
   const int y = i / w1, xq = i - y * w1;
-  const float sy = fmaxf((y + 0.5f) * (static_cast<float>(h0) / h1) - 0.5f, 0.f);
-  const float sx = fmaxf((xq + 0.5f) * (static_cast<float>(w0) / w1) - 0.5f, 0.f);
-  const int y0 = min(static_cast<int>(sy), h0 - 1), x0 = min(static_cast<int>(sx), w0 - 1);
-  const int y1 = min(y0 + 1, h0 - 1), x1 = min(x0 + 1, w0 - 1);
-  const float fy = sy - y0, fx = sx - x0;
+  const BilinearTap tap = bilinear_tap(y, xq, h0, w0, h1, w1);
+  const int y0 = tap.y0, y1 = tap.y1, x0 = tap.x0, x1 = tap.x1;
   const int *cb = codes + static_cast<long long>(b) * h0 * w0;
   const uint4 *p00 = reinterpret_cast<const uint4 *>(Z + static_cast<long long>(__ldg(cb + y0 * w0 + x0)) * C);
   const uint4 *p01 = reinterpret_cast<const uint4 *>(Z + static_cast<long long>(__ldg(cb + y0 * w0 + x1)) * C);
   const uint4 *p10 = reinterpret_cast<const uint4 *>(Z + static_cast<long long>(__ldg(cb + y1 * w0 + x0)) * C);
   const uint4 *p11 = reinterpret_cast<const uint4 *>(Z + static_cast<long long>(__ldg(cb + y1 * w0 + x1)) * C);
-  const float w00 = (1.f - fy) * (1.f - fx), w01 = (1.f - fy) * fx, w10 = fy * (1.f - fx), w11 = fy * fx;
+  const float w00 = tap.w00, w01 = tap.w01, w10 = tap.w10, w11 = tap.w11;
   float4 *dst = reinterpret_cast<float4 *>(F + (static_cast<long long>(b) * M1 + i) * C);
   for (int g = threadIdx.x & 31; g < C / 8; g += 32) {
     const uint4 a = __ldg(p00 + g), bq = __ldg(p01 + g), cq = __ldg(p10 + g), d = __ldg(p11 + g);
