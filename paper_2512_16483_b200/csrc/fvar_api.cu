@@ -361,7 +361,7 @@ fvar_status run_gemm(fvar_ctx *ctx, int epi, const fvar_ctx::ActMaps &maps, int 
       gemm_skinny_supported(epi, g.R, g.N, g.K)) {
     // few rows: bound by streaming the weights once, so the weights take the M side of the MMA and the K range
     // of every 128-feature tile is spread over a cluster (gemm_skinny.cu)
-    const int S = gemm_skinny_pick_splits(g.N, g.K, 0);
+    const int S = gemm_skinny_pick_splits(g.N, g.K, 0, 0, g.R <= 64);
     g.splits = S;
     gemm_skinny_shape(g);
     CUtensorMap tmA, tmW;
@@ -1482,7 +1482,7 @@ fvar_status fvar_gemm_bf16_form(const void *A, const void *W, const void *bias, 
       return kfail(FVAR_EINVAL, "gemm: the weight-streaming form needs R <= 512, N % 8 == 0");
     if (N % 8) return kfail(FVAR_EINVAL, "gemm: the cluster-split forms need N % 8 == 0");
     if (block_n < 0 || block_n > 8) return kfail(FVAR_EINVAL, "gemm: the cluster-split forms take 0 .. 8 K ranges");
-    const int S = gemm_skinny_pick_splits(N, K, block_n, tiles_m);
+    const int S = gemm_skinny_pick_splits(N, K, block_n, tiles_m, tiles_m == 0 && R <= 64);
     if (S <= 0) return kfail(FVAR_EINVAL, "gemm: this number of K ranges is not launchable for the problem");
     GemmArgs g = gemm_args(R, N, K);
     g.sk_tiles_m = tiles_m;

@@ -405,7 +405,7 @@ bool gemm_skinny_supported(int epi, int R, int N, int K) {
 // of K, so the K split over a cluster wins up to a few hundred rows, longer for a long reduction; with many
 // features the row-tiled kernels already cover the SMs and win from 64 rows on.
 int gemm_skinny_row_limit(int N, int K) {
-  if (N <= 2048) return K >= 4096 ? 384 : 64;               // 65 .. 256 rows go to the 128 x 128 cluster-split mode first
+  if (N <= 2048) return 64;                                  // from 65 rows on the 128 x 128 cluster-split mode is the faster one
   return 32;
 }
 
@@ -414,25 +414,29 @@ int gemm_skinny_row_limit(int N, int K) {
 bool gemm_ksplit_wins(int R, int N, int K) {
   if (N > 2048 || R <= 64) return false;                     // wide outputs fill the SMs without a K split; few rows stream weights
   if (R <= 256) return true;                                 // one or two row tiles: 7 - 15 us against 9 - 25 us row-tiled
-  return K >= 4096 && R > 384 && R <= 512;                   // four row tiles over a long reduction: 22 us against 25 us
+  return K >= 4096 && R <= 512;                              // three or four row tiles over a long reduction: 22 us against 25 us
 }
 
 // K ranges per tile (128 features x all rows, or x 128 rows when row_tiles > 0 row tiles are given): the split whose
-// slowest CTA walks the fewest K blocks, waves of resident clusters counted; among equals the smallest.  forced > 0
-// takes that split when it is launchable.
-int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles) {
+// slowest CTA walks the fewest K blocks while all clusters are resident at once.  Measured on B200: clusters of 7 or 8
+// and grids above about 0.9 of the SMs (odd cluster sizes do not pack the GPCs) fall into a second wave and cost 1.5 -
+// 2x, whatever the occupancy query says; the small form fits two CTAs per SM.  forced > 0 takes that split when it is
+// launchable.
+int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles, int small_form) {
   if (gemm_skinny_prepare() != cudaSuccess) return 0;
   const int *mc = row_tiles > 0 ? SkinnyState<EPI_RESID, true>::max_clusters : SkinnyState<EPI_RESID, false>::max_clusters;
   const int tiles = (N + kBlockM - 1) / kBlockM * (row_tiles > 0 ? row_tiles : 1), num_kb = (K + kBlockK - 1) / kBlockK;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int capacity = (small_form ? 2 : 1) * sms * 9 / 10;
   int best = 0;
   long long best_cost = 0;
   for (int s = 1; s <= 8; ++s) {
     if (mc[s] <= 0 || (forced > 0 && s != forced)) continue;
     const int kbps = (num_kb + s - 1) / s;
     if ((num_kb + kbps - 1) / kbps != s) continue;          // some range would be empty
-    if (s > 1 && kbps < 2 && forced <= 0) continue;
-    const long long waves = (tiles + mc[s] - 1) / mc[s];
-    const long long cost = waves * (kbps + 3);               // a wave costs its K blocks plus about three blocks' worth of fixed time
+    if (forced <= 0 && s > 1 && (kbps < 2 || s > 6 || tiles * s > capacity)) continue;
+    const long long cost = 10ll * (kbps + 3) + s;            // K blocks of the slowest CTA plus fixed time; smaller clusters on ties
     if (best == 0 || cost < best_cost) { best = s; best_cost = cost; }
   }
   return best;

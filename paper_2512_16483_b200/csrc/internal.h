@@ -124,7 +124,7 @@ GemmPlan gemm_plan(int R, int nbatch, int N, int K, int num_sms, int max_cluster
 bool gemm_skinny_supported(int epi, int R, int N, int K);
 int gemm_skinny_row_limit(int N, int K);
 bool gemm_ksplit_wins(int R, int N, int K);                   // the 128 x 128-tile cluster-split mode is the faster form                      // rows up to which this form is the faster one
-int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles = 0);      // 0: not launchable on this device
+int gemm_skinny_pick_splits(int N, int K, int forced, int row_tiles = 0, int small_form = 0);      // 0: not launchable on this device
 void gemm_skinny_shape(GemmArgs &a);      // needs a.R, a.K and a.splits
 bool gemm_skinny_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t K, uint64_t ld, uint32_t box_rows, int nk);
 cudaError_t launch_gemm_skinny(int epi, const CUtensorMap &tmA, const CUtensorMap &tmW, const GemmArgs &a, cudaStream_t st);
