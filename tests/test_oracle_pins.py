@@ -698,3 +698,60 @@ def test_lls_step_structure():
         assert np.linalg.matrix_rank(o.group_cache[g][1], tol=1e-8) <= r       # M rows spanned by the r block-output rows
     o.kv_append(2)
     assert o.cache_len(0, 1) == 4 + 9 + r and o.cache_len(0, 0) == 4 + 9
+
+
+# ----------------------------------------------------------------------------- wiring of the stateful oracle
+
+def test_sample_noise_is_indexed_by_group_then_computed_element_then_row():
+    """Oracle.scale_step under sampled selection: group g of computed element e (here the null-prompt elements b = 1, 3)
+    uses sample_noise[g][e].  Rebuilt outside the class from the group inputs it leaves behind."""
+    shp = si.shape_tiny(n_blocks=3, blocks_per_group=1, width=64, n_heads=1, head_dim=64, ffn_dim=128, scales=(2, 3, 4))
+    o = orc.Oracle(si.make_weights(51, shp, 0.05), shp.n_heads, 1, shp.hw(), shp.ln_eps)
+    B, r = 4, 5
+    o.set_cond(si.make_cond(51, B, 64))
+    for k in (0, 1):
+        o.scale_step(si.make_tokens(51, B, shp.tokens_per_scale()[k], 64), k, orc.Policy("dense"))
+        o.kv_append(k)
+    for g in range(3):
+        o.set_projection(2, g, si.make_projection(51, 2, g, 16, r))
+    toks = si.make_tokens(51, B, 16, 64, "spread")
+    noise = si.make_sample_noise(51, 2, 3, 2, 16)                       # [G = 3][E = 2][M = 16]
+    o.scale_step(toks, 2, orc.Policy("lowrank_rtr", "null_only", rank_per_group=[r] * 3, sample_noise=noise))
+    for e, b in enumerate((1, 3)):
+        X = toks[b].astype(np.float64)
+        for g in range(3):
+            want = orc.select_top_r(orc.sampling_keys(orc.row_scores(X, np.float32), noise[g][e]), r)
+            assert np.array_equal(o.last_indices[e][g], want), (e, g)
+            X = o.group_cache[g][b]                                     # the next group's input
+    # the lists really depend on the noise slice: another slice gives another list somewhere
+    assert any(not np.array_equal(o.last_indices[0][g], o.last_indices[1][g]) for g in range(3))
+
+
+def test_context_weight_rows_are_keys_then_values():
+    """set_cond splits w_ckv [2C][ctx_width] into keys (first C rows) and values (last C rows).  With the value rows
+    zeroed the cross-attention adds exactly nothing; with the key rows zeroed its scores are all equal, so it adds
+    the mean value row through W_co."""
+    shp = si.shape_tiny(n_blocks=1, width=64, n_heads=1, head_dim=64, ffn_dim=128, scales=(2,), cross=True, ctx_len=6)
+    w = si.make_weights(52, shp, 0.05)
+    cond, ctx = si.make_cond(52, 1, 64), si.make_context(52, 1, 6, 64)
+    toks = si.make_tokens(52, 1, 4, 64)
+
+    def run(wts):
+        o = orc.Oracle(wts, 1, 1, shp.hw(), shp.ln_eps)
+        o.set_cond(cond, ctx)
+        return o.scale_step(toks, 0, orc.Policy("dense"))[0]
+
+    no_values = [dict(w[0], w_ckv=np.concatenate([w[0]["w_ckv"][:64], np.zeros_like(w[0]["w_ckv"][64:])]))]
+    no_cross = [dict(w[0], w_co=np.zeros_like(w[0]["w_co"]))]
+    np.testing.assert_allclose(run(no_values), run(no_cross), rtol=0, atol=1e-12)
+    no_keys = [dict(w[0], w_ckv=np.concatenate([np.zeros_like(w[0]["w_ckv"][:64]), w[0]["w_ckv"][64:]]))]
+    # uniform scores: the cross-attention output of every row is mean_t(ctx_t W_v^T) W_co^T, independent of the query
+    add = (ctx[0].astype(np.float64) @ w[0]["w_ckv"][64:].astype(np.float64).T).mean(axis=0) @ w[0]["w_co"].astype(np.float64).T
+    o = orc.Oracle(no_keys, 1, 1, shp.hw(), shp.ln_eps)
+    o.set_cond(cond, ctx)
+    x = toks[0].astype(np.float64)
+    o.ada[0][0].reshape(6, -1)[5] = 0.0                                  # gate2 = 0
+    got, _, _ = orc.block_forward(x, o.ada[0][0], o.w[0], np.zeros((0, 64)), np.zeros((0, 64)), 1, shp.ln_eps, o.cross_kv[0][0])
+    ref, _, _ = orc.block_forward(x, o.ada[0][0], dict(o.w[0], w_co=np.zeros((64, 64))), np.zeros((0, 64)), np.zeros((0, 64)), 1,
+                                  shp.ln_eps, o.cross_kv[0][0])
+    np.testing.assert_allclose(got - ref, np.broadcast_to(add, got.shape), rtol=1e-9, atol=1e-12)
