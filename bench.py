@@ -66,19 +66,22 @@ LOOP_GUIDANCE = 3.0
 
 def resolve_workload(name):
     """A named workload, or a point of the last-scale sweep on the Infinity-2B shape:
-    `infinity2b_last_r<R>_b<B>` = only the 64 x 64 scale (4096 queries over a cache pre-filled with 6425 rows),
+    `infinity2b_last_[lls_]r<R>_b<B>` = only the 64 x 64 scale (4096 queries over a cache pre-filled with 6425 rows),
     batch B, every block group at rank R.  R < 4096 runs the method (null-prompt branch only, RP + RTR);
     R = 4096 is the unpruned dense path with both CFG branches."""
     import re
     if name in WORKLOADS:
         return WORKLOADS[name]
-    m = re.fullmatch(r"infinity2b_last_r(\d+)_b(\d+)", name)
+    m = re.fullmatch(r"infinity2b_last_(lls_)?r(\d+)_b(\d+)", name)
     if not m:
-        raise SystemExit("unknown workload %r (named: %s; or infinity2b_last_r<R>_b<B>)" % (name, ", ".join(sorted(WORKLOADS))))
-    R, B = int(m.group(1)), int(m.group(2))
+        raise SystemExit("unknown workload %r (named: %s; or infinity2b_last_[lls_]r<R>_b<B>)" % (name, ", ".join(sorted(WORKLOADS))))
+    lls, R, B = bool(m.group(1)), int(m.group(2)), int(m.group(3))
     if not (1 <= R <= 4096) or B < 1 or (R < 4096 and B % 2):
         raise SystemExit("need 1 <= R <= 4096 and a batch of whole CFG pairs")
-    return dict(shape="inf2b", B=B, first_late=12, keep=("rank", R), null_only=R < 4096)
+    if lls and R > 192:
+        raise SystemExit("the LLS restoration takes ranks up to 192")
+    # `lls_`: the same step with the rows restored by the least-squares matrices (Eq. "lstsq") instead of RTR
+    return dict(shape="inf2b", B=B, first_late=12, keep=("rank", R), null_only=R < 4096, restore="lls" if lls else "rtr")
 
 
 def scale_plan(wl, shp):
@@ -242,7 +245,7 @@ def oracle_leg(wl, steps, warmup):
             if r < Ms[k]:
                 o.set_projection(k, g, si.make_projection(SEED, k, g, Ms[k], r))
         pols[k] = orc.Policy("lowrank_rtr" if late else "dense", "null_only" if wl["null_only"] else "pair",
-                             rank_per_group=ranks if late else None)
+                             rank_per_group=ranks if late else None, restore=wl.get("restore", "rtr"))
     E = B // 2 if wl["null_only"] else B
     tokens_per_step = E * sum(Ms[k] for k in plan_full)       # skipped scales deliver their positions too
     last_dt = [0.0]
@@ -315,7 +318,7 @@ def main():
     config = {"workload": args.workload, "shape": wl["shape"], "batch": wl["B"],
               "late_scale_sides": list(make_shape(wl["shape"]).scales[wl["first_late"]:]),
               "keep": "rank %d" % wl["keep"][1] if isinstance(wl["keep"], tuple) else wl["keep"],
-              "cfg": "null_only" if wl["null_only"] else "pair",
+              "cfg": "null_only" if wl["null_only"] else "pair", "restore": wl.get("restore", "rtr"),
               "l2": "inputs_exceed_l2 (the stack's weights, streamed every step, are larger than L2)",
               "parity_bar": ("Infinity-2B shape: max-abs error <= 3e-2 x output RMS per block group (the stated 2e-2 is below what "
                              "rounding the FFN operands to bf16 alone costs at this shape, 1.6e-2; measured 2.1e-2), "
@@ -445,13 +448,15 @@ def main():
             feat_host.copy_(ctx.get_feature(B // 2, Ms[-1], shp.width), non_blocking=True)
             torch.cuda.synchronize()
 
+    restore = fv.RESTORE_LLS if wl.get("restore") == "lls" else fv.RESTORE_RTR
+
     def step_device():
         rewind()
         for k in late_scales:
             mode, ranks = modes[k]
             if mode == fv.SKIP:
                 continue
-            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks, out=outs[k])
+            ctx.scale_step(toks[k], k, mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks, out=outs[k], restore=restore)
             ctx.kv_append(k)
 
     def step_host():
@@ -460,7 +465,8 @@ def main():
             mode, ranks = modes[k]
             if mode == fv.SKIP:
                 continue
-            ctx.scale_step_host_async(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks)
+            ctx.scale_step_host_async(toks_host[k], k, outs_host[k], mode=mode, cfg_mode=cfg_at[k], rank_per_group=ranks,
+                                      restore=restore)
             ctx.kv_append(k)
         ctx.host_sync()                         # every result of the step is in host memory before the step counts
 

@@ -408,10 +408,10 @@ class Fvar:
         return out_host
 
     def scale_step_host_async(self, tokens_host: torch.Tensor, scale_idx: int, out_host: torch.Tensor, *, mode: int = DENSE,
-                              cfg_mode: int = CFG_PAIR, keep_ratio: float = 1.0, rank_per_group=None):
+                              cfg_mode: int = CFG_PAIR, keep_ratio: float = 1.0, rank_per_group=None, restore: int = RESTORE_RTR):
         """Pipelined host entry point: enqueues upload, step and download and returns; host_sync() waits for them."""
         assert not tokens_host.is_cuda and not out_host.is_cuda
-        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, None)
+        pol, _keep = self._policy(mode, cfg_mode, keep_ratio, rank_per_group, None, None, restore)
         self._check(self.lib.fvar_scale_step_host_async(self.ctx, tokens_host.data_ptr(), scale_idx, ct.byref(pol),
                                                         out_host.data_ptr()))
         return out_host
