@@ -13,7 +13,7 @@
 // TMEM round trip.  Keys at or beyond L are masked.  Every wait is bounded (see ptx.cuh).
 //
 // Few queries over a long cache (few CTAs, many key blocks): the key range is split over a thread-block cluster of
-// up to 8 CTAs.  Each parks its unnormalised (O, m, l) in its own shared memory; after a cluster barrier every
+// up to 6 CTAs.  Each parks its unnormalised (O, m, l) in its own shared memory; after a cluster barrier every
 // CTA merges a slice of the query rows over all ranges through distributed shared memory, in range order (the
 // result does not depend on timing), normalises and stores.  Nothing goes through global scratch.
 #include <math.h>
@@ -453,14 +453,19 @@ static cudaError_t launch_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, cons
 
 // Launch shape of an attention call: query tiles per CTA (two: each K / V block feeds two tiles, the softmax of one
 // overlapping the MMAs of the other; one: twice the CTAs when they would not fill the SMs) and key ranges per query
-// tile group (a cluster of at most 8 CTAs, each range at least four key blocks long).
+// tile group (a cluster of at most 6 CTAs, each range at least four key blocks long).
+// Largest cluster of key ranges.  Clusters of 7 or 8 CTAs (one CTA per SM here) do not pack the GPCs and part of the
+// grid falls into a second wave: measured in the step at the Infinity-2B shape, 8 -> 6 ranges took a block with r = 16
+// rows over 6.4 k keys from 110 to 100 us (5 ranges: 102, 4: 103).
+constexpr int kMaxRanges = 6;
+
 void attention_plan(int B_eff, int H, int r, int L, int num_sms, int *tiles_per_cta, int *kv_splits) {
   const int nkv = (L + kKeys - 1) / kKeys;
   auto ranges = [&](long long ctas) {                       // key ranges when `ctas` CTAs would run without a split
     if (ctas * 2 > num_sms || nkv < 8) return 1;            // enough CTAs already, or too few key blocks to share
     int s = static_cast<int>(num_sms / ctas);
     if (s > nkv / 4) s = nkv / 4;                           // at least four key blocks per range (measured: finer is slower)
-    if (s > 8) s = 8;                                       // a portable cluster
+    if (s > kMaxRanges) s = kMaxRanges;
     if (s < 2) return 1;
     const int per = (nkv + s - 1) / s;
     return (nkv + per - 1) / per;                           // every range gets at least one block

@@ -141,13 +141,13 @@ struct AttnArgs {
   bf16 *out;               // [B_eff * r][H * D]
   float scale_log2;        // log2(e) / sqrt(D)
   unsigned *status;
-  // kv_splits > 1: the key range is split over a cluster of that many CTAs (at most 8), merged through
+  // kv_splits > 1: the key range is split over a cluster of that many CTAs (at most 8 supported by the kernel; the planner uses up to 6), merged through
   // distributed shared memory
   int kv_splits;
   int tiles_per_cta;       // 1: one 128-row query tile per CTA; otherwise two
   long long wait_cycles;   // budget of every bounded wait (0: the default)
 };
-// Query tiles per CTA (1 or 2) and key ranges per launch (1 = no split; at most 8, a portable cluster).
+// Query tiles per CTA (1 or 2) and key ranges per launch (1 = no split; at most 6).
 void attention_plan(int B_eff, int H, int r, int L, int num_sms, int *tiles_per_cta, int *kv_splits);
 cudaError_t launch_attention(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                              const AttnArgs &a, cudaStream_t st);
