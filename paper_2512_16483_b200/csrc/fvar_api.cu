@@ -1099,7 +1099,13 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
       ga.ld_out = C;
       ga.status = ctx->status;
       ga.wait_cycles = ctx->wait_cycles;
-      const int bn = gemm_pick_block_n((r + 127) / 128 * E, C, Mk + M, ctx->num_sms);
+      // few row tiles over a long reduction (2 M rows of [hi ; lo]): the deterministic split-K of the row-tiled kernel
+      // puts more CTAs on it
+      int bn = 64, sp = 1;
+      gemm_pick_tile((r + 127) / 128 * E, C, Mk + M, ctx->num_sms, 4, kSplitScratchBytes, &bn, &sp);
+      ga.splits = sp;
+      ga.partial = ctx->split_partial;
+      ga.counters = ctx->split_counters;
       ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * r * C * M * E, 2.0 * (static_cast<double>(r) * M + 2.0 * E * M * C) + 4.0 * E * r * C);
       FV_CUDA(ctx, launch_gemm(EPI_F32, bn, ctx->qt_map[static_cast<size_t>(scale_idx) * G + g],
                                ctx->xsplit_map[scale_idx * 2 + (g & 1)], ga, ctx->num_sms, st), "projection gemm");
