@@ -51,7 +51,7 @@ enum { FVAR_RESTORE_RTR = 0, FVAR_RESTORE_LLS = 1 };               /* fvar_keep_
 /* Static shape of the block stack. */
 typedef struct {
   int n_blocks;          /* transformer blocks                                                */
-  int blocks_per_group;  /* RP / RTR are applied per block group ("at the block level", Sec. 3.3) */
+  int blocks_per_group;  /* RP / RTR are applied per block group (Sec. 3.3: block-level application) */
   int width;             /* C (the paper's d); multiple of 64                                 */
   int n_heads;           /* H                                                                 */
   int head_dim;          /* D: 64 or 128; H * D == C                                          */

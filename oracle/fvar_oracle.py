@@ -23,7 +23,7 @@ What the paper fixes and this file follows:
                                                           (Sec. 3.2; Algorithm 1)
   * rank schedule: ratio of min(M, d) per block chunk and late scale
                                                           (Eq. "low_rank_percent"; App. A.1 table)
-The paper gives no internals for "the VAR block"; the block below (AdaLN
+The paper gives no internals for its VAR block; the block below (AdaLN
 shift/scale/gate, multi-head attention over a multi-scale KV cache, tanh-GELU
 FFN, optional cross-attention) is the synthetic definition both sides use.
 
@@ -264,7 +264,7 @@ def scale_transition(F_prev: np.ndarray, F_o: np.ndarray, Z: np.ndarray, hw_k, h
 
 def cfg_combine(F_prompt: np.ndarray, F_null: np.ndarray, s: float) -> np.ndarray:
     """Classifier-free guidance on the two branches of a CFG pair: F_null + s (F_prompt - F_null).  s = 0 is
-    the null-prompt branch alone, which is what "setting the CFG to 0" in the fidelity-refinement stage means
+    the null-prompt branch alone, which is what a CFG of 0 in the fidelity-refinement stage amounts to
     (Sec. 3.3: CFG = 0 amounts to running the null text prompt alone)."""
     a, b = np.asarray(F_prompt, dtype=np.float64), np.asarray(F_null, dtype=np.float64)
     return b + s * (a - b)
@@ -295,7 +295,7 @@ def lls_restoration_matrix(F_r: np.ndarray, F_full: np.ndarray) -> np.ndarray:
 def lls_restore(F_r_out: np.ndarray, F_hat: np.ndarray, F_tilde: np.ndarray, Q: np.ndarray, cache_up: np.ndarray) -> np.ndarray:
     """The LLS restoration the paper tries before RTR (Sec. 3.3 RP, Eq. "lstsq"; App. A.3; Tab. "lowrank" row 5):
     F_k^o = W_r^o F_r^o with W_r^o ~ W_hat_r + W_r^{o,cache}.  W_hat_r restores the step's input from its projection
-    (F_tilde from F_hat = Q^T F_tilde).  W_r^{o,cache} is "obtained by solving the LLS problem" for the cached
+    (F_tilde from F_hat = Q^T F_tilde).  W_r^{o,cache} comes from a second least-squares problem posed on the cached
     counterpart feature; the paper does not name the r-row feature of that second problem -- read here as the
     projection of the cached feature by the same Q, Q^T Up(F_{k-1}^o), restored to Up(F_{k-1}^o).  The sum of the
     two matrices is taken as the paper writes it.  Both problems need their r-row feature of full row rank, so
