@@ -463,7 +463,7 @@ void attention_plan(int B_eff, int H, int r, int L, int num_sms, int *tiles_per_
   const int nkv = (L + kKeys - 1) / kKeys;
   auto ranges = [&](long long ctas) {                       // key ranges when `ctas` CTAs would run without a split
     if (ctas * 2 > num_sms || nkv < 8) return 1;            // enough CTAs already, or too few key blocks to share
-    int s = static_cast<int>(num_sms / ctas);
+    int s = static_cast<int>(num_sms * 9 / 10 / ctas);       // clusters do not pack the last tenth of the SMs (measured)
     if (s > nkv / 4) s = nkv / 4;                           // at least four key blocks per range (measured: finer is slower)
     if (s > kMaxRanges) s = kMaxRanges;
     if (s < 2) return 1;
@@ -474,7 +474,8 @@ void attention_plan(int B_eff, int H, int r, int L, int num_sms, int *tiles_per_
   const long long singles = static_cast<long long>((r + kQRows - 1) / kQRows) * H * B_eff;
   // One tile per CTA when the tile pairs alone would leave more than half of the SMs idle: a lone tile cannot hide its
   // softmax behind the other tile's MMAs, but twice the CTAs share the tensor work.  Measured in the step at the
-  // Infinity-2B shape: r = 170 over 6.6 k keys 150 -> 130 us per block, r = 218 over 2.7 k keys 123 -> 115.
+  // Infinity-2B shape: r = 170 over 6.6 k keys 150 -> 130 us per block, r = 218 over 2.7 k keys 123 -> 115; a model
+  // weighing 2 x 1800 cycles per key block of a pair against 2500 of a lone tile picked no better.
   const bool single = r > kQRows && pairs * 2 <= num_sms;
   *tiles_per_cta = single ? 1 : 2;
   *kv_splits = ranges(single ? singles : pairs);
