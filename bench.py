@@ -93,6 +93,10 @@ def scale_plan(wl, shp):
         keep = wl["keep"]
         if k < wl.get("dense_until", 0):
             plan[k] = [Ms[k]] * shp.n_groups
+        elif isinstance(keep, tuple) and wl.get("restore") == "lls":
+            # an LLS group's output is spanned by its r rows, so the next group projects a rank-r input: its rank
+            # steps down by 8 per group to keep the r x r Gram matrix of that projection well conditioned in fp32
+            plan[k] = [max(8, min(keep[1], Ms[k]) - 8 * g) for g in range(shp.n_groups)]
         elif isinstance(keep, tuple):
             plan[k] = [min(keep[1], Ms[k])] * shp.n_groups
         elif keep in ("table", "paper"):

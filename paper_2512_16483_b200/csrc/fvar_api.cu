@@ -1229,9 +1229,19 @@ static fvar_status scale_step_impl(fvar_ctx *ctx, const void *tokens, bool token
                       mr = static_cast<long long>(M) * r;
       auto sg = [&](bool tb, const float *A, const float *Bm, float *O, int m, int n, int k, long long lda, long long ldb, long long ldo,
                     long long ao, long long as, long long bo, long long bs, long long oo, long long os, bool acc, const char *what) -> fvar_status {
+        // few output tiles over a long reduction (the Gram matrices, F F_hat^T): cut K so that about all SMs work; the
+        // partial products go through the split-K scratch area and are added in a fixed order
+        const long long tiles = static_cast<long long>((m + 127) / 128) * ((n + 63) / 64) * E;
+        int ks = 1;
+        if (!acc && k >= 256 && tiles * 2 <= ctx->num_sms) {
+          ks = static_cast<int>(ctx->num_sms / tiles);
+          if (ks > k / 64) ks = k / 64;
+          while (ks > 1 && static_cast<size_t>(ks) * E * m * n * 4 > kSplitScratchBytes) --ks;
+        }
         ctx->prof_begin(FVAR_KCLASS_GEMM, 2.0 * m * n * k * E, 4.0 * E * (static_cast<double>(m) * k + static_cast<double>(n) * k + static_cast<double>(m) * n));
-        FV_CUDA(ctx, launch_sgemm(tb, A, Bm, O, m, n, k, lda, ldb, ldo, ao, as, bo, bs, oo, os, E, acc, st), what);
+        FV_CUDA(ctx, launch_sgemm(tb, A, Bm, O, m, n, k, lda, ldb, ldo, ao, as, bo, bs, oo, os, E, acc, st, ks, ctx->split_partial), what);
         ctx->launched();
+        if (ks > 1) ctx->launched();
         return FVAR_OK;
       };
       float *G1 = ctx->lls_G, *G2 = ctx->lls_G + E * rr, *I1 = ctx->lls_Ginv, *I2 = ctx->lls_Ginv + E * rr;

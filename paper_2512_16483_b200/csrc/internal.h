@@ -207,7 +207,7 @@ cudaError_t lls_prepare();
 // out[z] (+)= A[z] B[z]^T (trans_b: B stored [n][k]) or A[z] B[z] (B stored [k][n]); pitches and batch strides in floats.
 cudaError_t launch_sgemm(bool trans_b, const float *A, const float *B, float *out, int m, int n, int k, long long lda, long long ldb,
                          long long ldo, long long a_off, long long a_stride, long long b_off, long long b_stride, long long o_off,
-                         long long o_stride, int batch, bool accumulate, cudaStream_t st);
+                         long long o_stride, int batch, bool accumulate, cudaStream_t st, int ksplit = 1, float *scratch = nullptr);
 cudaError_t launch_chol_inverse(const float *G, float *Ginv, int r, int count, unsigned *status, cudaStream_t st);
 cudaError_t launch_split_rows(const float *x, long long x_off, long long x_stride, int E, int M, int C, bf16 *xsplit, int mk,
                               cudaStream_t st);
