@@ -97,7 +97,8 @@ typedef struct {
                                  F_r^o, W_hat the least-squares map from Q^T F back to the group's input F, W^{o,cache}
                                  the same for the upsampled cached group output (this library's reading: its r-row
                                  feature is its projection by the same Q).  No index set is chosen; r <= 192 per
-                                 group (FVAR_EUNSUPPORTED beyond).  fp32 arithmetic; a Gram matrix that is not
+                                 group (FVAR_EUNSUPPORTED beyond) and r <= the tokens of the cached scale (FVAR_EINVAL);
+                                 a group's output then has rank r, so the next group should use a smaller r.  fp32 arithmetic; a Gram matrix that is not
                                  positive definite is reported as FVAR_EINVAL by fvar_poll_status.                  */
 } fvar_keep_policy;
 
