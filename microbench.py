@@ -1,10 +1,10 @@
 """Stand-alone timings of the library's kernels through the C ABI (CUDA events, one GPU).
 
-    python microbench.py gemm        # FVAR_GEMM_BLOCK_N=64|128|256 forces a width, FVAR_GEMM_PAIR=0|1 the launch form
+    python microbench.py gemm [single|pair <64|128|256>]   # the library's choice, or a given launch form and tile width
     python microbench.py skinny      # the weight-streaming form on the Infinity-2B-shaped late GEMMs
     python microbench.py skinny_one R N K [S]  # eight launches of that form on one shape (for ncu)
     python microbench.py attention_one B H D r L   # four attention launches on one shape (for ncu)
-    python microbench.py gemmk       # the same over K at fixed R x N: fixed cost and cost per K step
+    python microbench.py gemmk [single|pair <width>]       # the same over K at fixed R x N: fixed cost and cost per K step
     python microbench.py attention
     python microbench.py memory      # score, LayerNorm + modulate, restoration fill, selection
     python microbench.py transition  # between two scale steps: codeword search, Up-accumulate, Down
@@ -14,7 +14,6 @@ that host launch cost does not enter the time.
 """
 from __future__ import annotations
 
-import os
 import sys
 
 import torch
@@ -35,34 +34,24 @@ def _time(fn, n=20, warm=3):
     return e0.elapsed_time(e1) * 1e3 / n          # microseconds
 
 
-def _gemm_graph_us(lib, R, N, K):
-    ncopy = max(2, min(32, int(300e6 // (N * K * 2))))
-    A = torch.randn(R, K, device="cuda").bfloat16()
-    Ws = [torch.randn(N, K, device="cuda").bfloat16() * 0.02 for _ in range(ncopy)]
-    out = torch.empty(R, N, device="cuda", dtype=torch.float32)
-
-    def call(i):
-        lib.fvar_gemm_bf16(A.data_ptr(), Ws[i % ncopy].data_ptr(), None, R, N, K, out.data_ptr(),
-                           torch.cuda.current_stream().cuda_stream)
-    for i in range(ncopy):
-        call(i)
-    torch.cuda.synchronize()
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g):
-        for i in range(ncopy):
-            call(i)
-    return _time(g.replay, n=5, warm=1) / ncopy
+def _form_args():
+    """Optional launch form after the sub-command: `single|pair <tile width>`; default: the library's cost model."""
+    if len(sys.argv) > 3 and sys.argv[2] in ("single", "pair"):
+        return (fv.GEMM_SINGLE if sys.argv[2] == "single" else fv.GEMM_PAIR), int(sys.argv[3]), "%s %s" % (sys.argv[2], sys.argv[3])
+    return fv.GEMM_AUTO, 0, "picked"
 
 
 def gemm():
     lib = fv.load_library()
-    bn = os.environ.get("FVAR_GEMM_BLOCK_N", "auto")
+    form, block_n, bn = _form_args()
     shapes = [(1024, 3072, 1024), (1024, 1024, 1024), (1024, 4096, 1024), (1024, 1024, 4096), (400, 3072, 1024),
               (16, 2048, 2048), (16, 2048, 8192), (336, 8192, 2048), (4096, 4096, 1024), (8192, 8192, 2048),
               (16384, 4096, 4096)]
     for R, N, K in shapes:
-        us = _gemm_graph_us(lib, R, N, K)
-        print("BN=%s R=%d N=%d K=%d: %.2f us  %.1f TFLOP/s  weights %.0f GB/s" % (
+        if form == fv.GEMM_PAIR and R <= 128:
+            continue                                     # a single row tile has no partner
+        us = _gemm_form_graph_us(lib, R, N, K, form, block_n)
+        print("form %s R=%d N=%d K=%d: %.2f us  %.1f TFLOP/s  weights %.0f GB/s" % (
             bn, R, N, K, us, 2 * R * N * K / us / 1e6, N * K * 2 / us / 1e3))
 
 
@@ -138,10 +127,10 @@ def ksplit():
 
 def gemmk():
     lib = fv.load_library()
-    tag = "PAIR=%s BN=%s" % (os.environ.get("FVAR_GEMM_PAIR", "model"), os.environ.get("FVAR_GEMM_BLOCK_N", "model"))
+    form, block_n, tag = _form_args()
     for R, N in [(1024, 3072), (1024, 1024), (4096, 4096)]:
-        res = ["K=%d: %.2f us" % (K, _gemm_graph_us(lib, R, N, K)) for K in (128, 256, 512, 1024, 2048, 4096)]
-        print(tag, "R=%d N=%d |" % (R, N), "  ".join(res), flush=True)
+        res = ["K=%d: %.2f us" % (K, _gemm_form_graph_us(lib, R, N, K, form, block_n)) for K in (128, 256, 512, 1024, 2048, 4096)]
+        print("form", tag, "R=%d N=%d |" % (R, N), "  ".join(res), flush=True)
 
 
 def attention():
