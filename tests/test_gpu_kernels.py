@@ -298,3 +298,25 @@ def test_row_keys_and_sampled_selection(fv, B, M, C):
     # a key is one correctly rounded fp32 division of the kernel's own score
     s_gpu = fv.fvar_row_scores(torch.from_numpy(x).cuda()).cpu().numpy()
     assert np.array_equal(got, (s_gpu / noise).astype(np.float32))
+
+
+# ----------------------------------------------------------------------------- run-to-run determinism of the cluster reductions
+
+def test_cluster_reductions_are_bit_stable(fv):
+    """The K split of the cluster GEMMs and the key split of attention add their partial results in rank order, so
+    repeated launches on the same operands give the same bits."""
+    rng = np.random.default_rng(77)
+    A = to_bf16_cuda(si.normal_bf16(rng, (170, 8192)))
+    W = to_bf16_cuda(si.normal_bf16(rng, (2048, 8192), 0.05))
+    for form in (fv.GEMM_SKINNY, fv.GEMM_KSPLIT):
+        first = fv.fvar_gemm_bf16_form(A, W, None, form, 0).clone()
+        for _ in range(3):
+            assert torch.equal(first, fv.fvar_gemm_bf16_form(A, W, None, form, 0))
+    B, H, D, r, L, L_cap = 1, 16, 128, 170, 6595, 6656
+    q = to_bf16_cuda(si.normal_bf16(rng, (B, r, H * D)))
+    Kc = to_bf16_cuda(si.normal_bf16(rng, (B, H, L_cap, D)))
+    Vt = to_bf16_cuda(si.normal_bf16(rng, (B, H, D, L_cap)))
+    first = fv.fvar_attention(q, Kc, Vt, L).clone()
+    for _ in range(3):
+        assert torch.equal(first, fv.fvar_attention(q, Kc, Vt, L))
+    _poll(fv)
