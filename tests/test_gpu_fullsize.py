@@ -241,3 +241,24 @@ def test_infinity_group_last_scale_small_ranks(fv, B):
         p.gpu.restore_loaded()
         p.oracle.load_group_cache(k - 1, gc)
         p.oracle.load_kv(*si.make_kv_prefill(5000 + B, 4, B, 6425, 2048))
+
+
+def test_infinity_group_last_scale_lls_restoration(fv):
+    """The LLS restoration variant (Eq. "lstsq", App. A.3) on one Infinity-2B-shaped block group at the last scale:
+    4096 rows restored from r = 64 block-output rows by the two least-squares matrices, against the oracle's fp64 solve."""
+    shp = si.shape_infinity_2b(n_blocks=4, blocks_per_group=4)
+    B, k, r = 2, 12, 64
+    p = Pair(fv, shp, seed=66, B=B)
+    p.prefill(k)
+    p.set_projections(k, [r])
+    toks = si.make_tokens(66, B, 4096, 2048, "spread")
+    ref = p.oracle.scale_step(toks, k, orc.Policy("lowrank_rtr", "null_only", rank_per_group=[r], restore="lls"))
+    out = p.gpu.scale_step(to_bf16_cuda(toks), k, mode=fv.LOWRANK_RTR, cfg_mode=fv.CFG_NULL_ONLY, rank_per_group=[r],
+                           restore=fv.RESTORE_LLS)
+    p.check_ok()
+    e, c = rel_err(p.gpu.get_group_output(0, 4096).cpu().numpy()[1], p.oracle.group_cache[0][1])
+    print("Infinity-shaped LLS group: max-abs/RMS %.3e cosine %.6f" % (e, c))
+    assert e <= 2e-2 and c >= 0.999, (e, c)                  # measured 0.8e-2: the stated bar holds here
+    assert_out_close(bf16_to_numpy(out), ref, what="Infinity-shaped group, LLS")
+    p.gpu.kv_append(k)
+    assert [p.gpu.cache_len(b) for b in range(4)] == [6425 + r] * 4
