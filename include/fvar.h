@@ -241,9 +241,9 @@ fvar_status fvar_restore_loaded(fvar_ctx *ctx);
  * leave more than half of the SMs idle.  Measured: +2 % on the Infinity-shaped late scales, -5 % on the
  * VAR-d16 ones, hence off by default.
  * FVAR_OPT_SKINNY_MAX_ROWS (default 512; 0 .. 512): cap on the rows R = B_eff * r up to which a GEMM of the
- * step may take the weight-streaming form (the library's own rule picks it per GEMM: up to 32 rows for wide
- * outputs, up to 64 rows for outputs of at most 2048 features, which from 65 rows on take 128 x 128 tiles with the
- * same K split: up to 256 rows, up to 512 with a reduction of 4096 or more).  In that
+ * step may take one of the cluster-split forms (the library's own rule picks per GEMM: the weight-streaming form up
+ * to 32 rows for wide outputs; 128 x 128 tiles with the same K split for outputs of at most 2048 features up to 256
+ * rows, up to 512 with a reduction of 4096 or more).  In that
  * form the weights are the M side of the MMA and the K range of a 128-feature tile is spread over a
  * thread-block cluster that reduces through distributed shared memory; it is bound by reading the weights
  * once.  0 never uses it.

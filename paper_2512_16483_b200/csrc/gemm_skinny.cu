@@ -400,21 +400,22 @@ bool gemm_skinny_supported(int epi, int R, int N, int K) {
   return epi != EPI_ARGMAX && R >= 1 && R <= 512 && N % 8 == 0 && K % 8 == 0 && N >= 8;
 }
 
-// Up to how many rows the weight-streaming form beats the row-tiled kernels (measured on B200, Infinity-2B-shaped
-// GEMMs): with few output features the row-tiled kernels have too few tiles to fill the SMs and each CTA walks all
-// of K, so the K split over a cluster wins up to a few hundred rows, longer for a long reduction; with many
-// features the row-tiled kernels already cover the SMs and win from 64 rows on.
+// Which of the two cluster-split modes, if any, beats the row-tiled kernels -- set from measurements in the step on B200
+// (Infinity-2B-shaped GEMMs).  Narrow outputs (at most 2048 features: out-proj, cross-attention projections, fc2) have
+// too few tiles to fill the SMs row-tiled and each CTA walks all of K: the 128 x 128-tile mode with the K range over a
+// cluster wins for every row count up to 256, up to 512 with a long reduction (fc2: 25 -> 13 - 22 us).  It also beats
+// the weight-streaming form there, down to 16 rows (a block at r = 16: 94.5 -> 90.6 us, at r = 59: 107.8 -> 100.3).
+// Wide outputs (QKV, fc1) fill the SMs row-tiled from 33 rows on; below, the weight-streaming form wins (15.5 -> 7.8 us
+// at R = 16) and the 128 x 128 mode does not (90.6 -> 93.9 us per block).
 int gemm_skinny_row_limit(int N, int K) {
-  if (N <= 2048) return 64;                                  // from 65 rows on the 128 x 128 cluster-split mode is the faster one
+  (void)N; (void)K;
   return 32;
 }
 
-// Whether the 128 x 128-tile mode (rows on the M side, K split over a cluster) beats the row-tiled kernels: set from
-// measurements; see the cost note in gemm_skinny_row_limit.
 bool gemm_ksplit_wins(int R, int N, int K) {
-  if (N > 2048 || R <= 64) return false;                     // wide outputs fill the SMs without a K split; few rows stream weights
-  if (R <= 256) return true;                                 // one or two row tiles: 7 - 15 us against 9 - 25 us row-tiled
-  return K >= 4096 && R <= 512;                              // three or four row tiles over a long reduction: 22 us against 25 us
+  if (N > 2048) return false;
+  if (R <= 256) return true;
+  return K >= 4096 && R <= 512;
 }
 
 // K ranges per tile (128 features x all rows, or x 128 rows when row_tiles > 0 row tiles are given): the split whose
